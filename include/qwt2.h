@@ -1,0 +1,170 @@
+/*
+ * qwt2.h -- C ABI of libqwt2: CWAC-fused quantized linear layer and CWAC calibration
+ *           (QwT-v2, "channel-wise affine compensation") for NVIDIA B200 (sm_100a).
+ *
+ * General rules
+ *   - Plain C.  No exceptions, no abort, nothing is printed.  Every call returns qwt_status.
+ *   - Unless a parameter is marked HOST, every data pointer is a CUDA DEVICE pointer owned by the
+ *     caller.  The library never frees caller memory and (except the *_host calls) never allocates
+ *     device memory and never synchronises: work is enqueued on `stream` (a cudaStream_t passed as
+ *     void*, NULL = the legacy default stream) and outputs are valid once that stream reaches the
+ *     end of the call.
+ *   - Matrices are row-major with the last index contiguous.
+ *   - Argument errors are found on the host before anything is launched.
+ *   - Inputs are assumed finite; NaN/Inf behaviour is unspecified.  Outputs must not alias inputs.
+ *   - Calls may run concurrently on different streams if their workspaces are distinct.
+ */
+#ifndef QWT2_H_
+#define QWT2_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef int32_t qwt_status;
+enum {
+  QWT_OK = 0,
+  QWT_ERR_NULL = 1,        /* a required pointer is NULL */
+  QWT_ERR_SHAPE = 2,       /* non-positive or overflowing dimension */
+  QWT_ERR_ALIGN = 3,       /* base pointer or leading dimension not aligned as required */
+  QWT_ERR_UNSUPPORTED = 4, /* dimension not a required multiple, unknown enum value */
+  QWT_ERR_WORKSPACE = 5,   /* workspace too small */
+  QWT_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed; see qwt_last_cuda_error */
+  QWT_ERR_TIMEOUT = 7,     /* a bounded device-side wait gave up (reported by qwt_qlinear_check_status) */
+  QWT_ERR_ARCH = 8         /* current device is not compute capability 10.x */
+};
+
+/* weight storage */
+enum { QWT_W_INT8 = 0,         /* [N, K] int8 codes in [-127, 127] */
+       QWT_W_INT4_PACKED = 1   /* [N, K/2] bytes, two's-complement nibbles, element 2j low, 2j+1 high */ };
+
+/* output stage of the forward call */
+enum { QWT_OUT_INT8_PER_TOKEN = 0, /* int8 codes [M, N] + float y_scale[M] (dynamic per-token absmax) */
+       QWT_OUT_BF16 = 1,           /* bfloat16 [M, N], round to nearest even */
+       QWT_OUT_FP32 = 2,           /* float [M, N]: the compensated real-valued output z */
+       QWT_OUT_INT32_ACC = 3       /* int32 [M, N]: raw integer accumulators (verification) */ };
+
+const char* qwt_version(void);
+const char* qwt_status_string(qwt_status s);
+/* CUDA error code of the most recent QWT_ERR_CUDA on the calling thread (0 if none). */
+qwt_status qwt_last_cuda_error(int* cuda_err /*HOST out*/);
+
+/* ---------------------------------------------------------------------------------------------
+ * CWAC calibration -- Section 3.3, Eq. 3-5.
+ * For every output channel c the least-squares line through the calibration pairs
+ *     (q_out[r, c], fp_out[r, c]),  r = 0..rows-1:
+ *     a[c] = Cov(fp_out[:,c], q_out[:,c]) / Var(q_out[:,c]),   b[c] = E[fp_out[:,c]] - a[c] E[q_out[:,c]].
+ * fp_out is the full-precision module output Y_full, q_out the quantized module's output Y_quant
+ * on the same calibration tokens.
+ *
+ * The kernels make ONE pass over the two matrices and reduce them to five numbers per channel,
+ * stats = double[5 * channels] laid out as [n | sum q | sum f | sum q*f | sum q*q] (each `channels`
+ * long).  Eq. 4-5 are functions of exactly these, so calibration can be streamed batch by batch
+ * (qwt_cwac_stats_accumulate per batch, qwt_cwac_solve at the end) or done in one call
+ * (qwt_cwac_calibrate = zero stats in workspace + accumulate + solve).
+ *
+ * Degenerate channel (Var(q) <= 1e-12 * E[q^2], e.g. a constant column or rows == 1): every
+ * (a, b = E[f] - a E[q]) minimises Eq. 3; a = 1 is returned.
+ *
+ *   fp_out, q_out : float [rows, ld], ld >= channels, ld % 4 == 0, base 16-byte aligned
+ *   a, b          : float [channels] out
+ *   n_degenerate  : int32 out (single value), may be NULL
+ *   workspace     : >= qwt_cwac_workspace_bytes(rows, channels) bytes, 256-byte aligned
+ * Errors: NULL, SHAPE (rows < 1, channels < 1, ld < channels), ALIGN, WORKSPACE, ARCH, CUDA.
+ * Results are bitwise reproducible for fixed (rows, channels, ld).
+ */
+size_t qwt_cwac_workspace_bytes(int64_t rows, int32_t channels);
+qwt_status qwt_cwac_calibrate(const float* fp_out, const float* q_out, int64_t rows, int32_t channels,
+                              int64_t ld, float* a, float* b, int32_t* n_degenerate,
+                              void* workspace, size_t workspace_bytes, void* stream);
+/* stats += statistics of this batch.  The caller zeroes stats (5*channels doubles) before the first batch. */
+qwt_status qwt_cwac_stats_accumulate(const float* fp_out, const float* q_out, int64_t rows, int32_t channels,
+                                     int64_t ld, double* stats, void* workspace, size_t workspace_bytes,
+                                     void* stream);
+/* Closed form of Eq. 4-5 from the statistics (float64 arithmetic, float32 results). */
+qwt_status qwt_cwac_solve(const double* stats, int32_t channels, float* a, float* b, int32_t* n_degenerate,
+                          void* stream);
+/* Calibration with HOST matrices: fp_out/q_out are host pointers (pinned memory recommended); they are
+ * streamed to the device in row chunks through `staging` (device, >= qwt_cwac_host_staging_bytes) while
+ * earlier chunks are reduced.  a, b, n_degenerate are HOST outputs, valid on return (the call waits). */
+size_t qwt_cwac_host_staging_bytes(int64_t rows, int32_t channels);
+qwt_status qwt_cwac_calibrate_host(const float* fp_out /*HOST*/, const float* q_out /*HOST*/, int64_t rows,
+                                   int32_t channels, int64_t ld, float* a /*HOST*/, float* b /*HOST*/,
+                                   int32_t* n_degenerate /*HOST, may be NULL*/,
+                                   void* staging, size_t staging_bytes, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Fold -- Section 3.4, Eq. 9-11.  CWAC is absorbed into the layer's requantization parameters:
+ * alpha joins the multiplier (Eq. 11, M' = alpha S_x S_W / S_r), beta joins the additive term.
+ * With per-token S_x and S_r that are only known at run time the static parts are
+ *     fscale[n] = a[n] * w_scale[n],     fbias[n] = a[n] * bias[n] + b[n]
+ * (CWAC acts on the module output, which includes the layer bias).
+ *   w_scale [n] float (S_W); bias [n] float or NULL (= 0); a, b [n] float or both NULL (= 1, 0)
+ *   fscale, fbias [n] float out.
+ * Errors: NULL (w_scale, fscale, fbias; or exactly one of a, b), SHAPE (n < 1), ARCH, CUDA.
+ */
+qwt_status qwt_cwac_fold(const float* w_scale, const float* bias, const float* a, const float* b, int32_t n,
+                         float* fscale, float* fbias, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Forward -- Section 3.4, Eq. 6-11 with all zero-points 0 (symmetric codes).
+ *     acc[m, n] = sum_k X[m, k] * W[n, k]                       (int8 x int8 -> int32, exact; the W_q x_q of Eq. 7)
+ *     z[m, n]   = fma((float)acc[m, n] * x_scale[m], fscale[n], fbias[n])      (Eq. 9 after the fold)
+ *   QWT_OUT_INT8_PER_TOKEN: y_scale[m] = max_n |z[m, n]| / 127;  Y[m, n] = clip(rne(z / y_scale[m]), -127, 127)
+ *                           (Eq. 1-2 applied to the output with zero-point 0: the 1/S_r of Eq. 10-11, per token);
+ *                           a row of zeros gives y_scale 0 and codes 0.
+ *   QWT_OUT_BF16 / FP32   : Y = z rounded to bfloat16 / as is.       QWT_OUT_INT32_ACC: Y = acc.
+ *
+ *   X [M, K] int8; x_scale [M] float (may be NULL for INT32_ACC)
+ *   W [N, K] int8, or [N, K/2] packed int4 (expanded to int8 on chip)
+ *   fscale, fbias [N] float (may be NULL for INT32_ACC)
+ *   Y [M, N] of the output type; y_scale [M] float out, INT8 mode only (else NULL)
+ *   K % 16 == 0 (int8) or K % 32 == 0 (packed int4); X, W, Y bases 16-byte aligned;
+ *   N % 16 == 0 (int8 out), N % 8 == 0 (bf16), N % 4 == 0 (fp32 / int32).
+ *   workspace >= qwt_qlinear_workspace_bytes(...), 256-byte aligned; its content is scratch
+ *   (a status word, per-row maxima, per-strip counters) that the call re-initialises itself.
+ * Errors: NULL, SHAPE, ALIGN, UNSUPPORTED, WORKSPACE, ARCH, CUDA.  Device-side waits are bounded; if one
+ * gives up the kernel records it in the workspace status word and exits; qwt_qlinear_check_status
+ * reports that as QWT_ERR_TIMEOUT.
+ */
+size_t qwt_qlinear_workspace_bytes(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode);
+qwt_status qwt_qlinear_cwac_forward(const int8_t* X, const float* x_scale, const void* W, int32_t wfmt,
+                                    const float* fscale, const float* fbias, int32_t M, int32_t N, int32_t K,
+                                    int32_t out_mode, void* Y, float* y_scale,
+                                    void* workspace, size_t workspace_bytes, void* stream);
+/* Waits for `stream`, then reads the status word of a forward workspace.  QWT_OK or QWT_ERR_TIMEOUT.
+ * device_status (HOST out, may be NULL) receives the raw word (0 = clean). */
+qwt_status qwt_qlinear_check_status(const void* workspace, void* stream, int32_t* device_status);
+/* Forward with HOST activations: X, x_scale are host inputs, Y, y_scale host outputs (pinned memory
+ * recommended); W, fscale, fbias stay DEVICE resident (they are model parameters).  `staging` is device
+ * scratch >= qwt_qlinear_host_staging_bytes(...).  The call copies in, runs the same kernel, copies out
+ * and waits for the stream, so the outputs are valid on return. */
+size_t qwt_qlinear_host_staging_bytes(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode);
+qwt_status qwt_qlinear_cwac_forward_host(const int8_t* X /*HOST*/, const float* x_scale /*HOST*/, const void* W,
+                                         int32_t wfmt, const float* fscale, const float* fbias, int32_t M,
+                                         int32_t N, int32_t K, int32_t out_mode, void* Y /*HOST*/,
+                                         float* y_scale /*HOST*/, void* staging, size_t staging_bytes,
+                                         void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Support: symmetric row-wise quantizer -- Eq. 1-2 with zero-point 0 and signed codes.
+ *     scale[r] = max_c |X[r, c]| / qmax;   Xq[r, c] = clip(rne(X[r, c] / scale[r]), -qmax, qmax)
+ * Per-token activations: X = activations, qmax = 127.  Per-channel weights: X = W [N, K], qmax = 127 or 7.
+ *   X float [rows, ld] (ld >= cols); Xq int8 [rows, cols]; scale float [rows].  A zero row gives scale 0, codes 0.
+ * qwt_pack_int4: codes int8 [rows, cols] in [-8, 7], cols even -> packed [rows, cols/2].
+ */
+qwt_status qwt_quantize_rows_i8(const float* X, int64_t rows, int32_t cols, int64_t ld, int32_t qmax,
+                                int8_t* Xq, float* scale, void* stream);
+qwt_status qwt_pack_int4(const int8_t* codes, int64_t rows, int32_t cols, uint8_t* packed, void* stream);
+
+/* Kernels launched by this library on the calling thread since the last reset (for launch accounting). */
+int64_t qwt_launch_count(void);
+void qwt_launch_count_reset(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* QWT2_H_ */

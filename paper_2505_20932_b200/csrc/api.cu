@@ -1,0 +1,386 @@
+// extern "C" entry points of libqwt2: argument validation on the host, then kernel launches.
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <string.h>
+
+#include <mutex>
+
+#include "qwt2_internal.h"
+
+namespace qwt {
+
+static thread_local int tl_cuda_error = 0;
+static thread_local int64_t tl_launches = 0;
+
+void set_cuda_error(int err) { tl_cuda_error = err; }
+void count_launch(int n) { tl_launches += n; }
+
+qwt_status current_device(DeviceInfo* out) {
+  static std::mutex mu;
+  static DeviceInfo cache[64];
+  static bool have[64] = {false};
+  int dev = 0;
+  QWT_CUDA_TRY(cudaGetDevice(&dev));
+  std::lock_guard<std::mutex> lock(mu);
+  if (dev < 0 || dev >= 64) return QWT_ERR_ARCH;
+  if (!have[dev]) {
+    DeviceInfo d{};
+    d.device = dev;
+    QWT_CUDA_TRY(cudaDeviceGetAttribute(&d.sm_count, cudaDevAttrMultiProcessorCount, dev));
+    QWT_CUDA_TRY(cudaDeviceGetAttribute(&d.cc_major, cudaDevAttrComputeCapabilityMajor, dev));
+    QWT_CUDA_TRY(cudaDeviceGetAttribute(&d.cc_minor, cudaDevAttrComputeCapabilityMinor, dev));
+    QWT_CUDA_TRY(cudaDeviceGetAttribute(&d.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev));
+    cache[dev] = d;
+    have[dev] = true;
+  }
+  *out = cache[dev];
+  if (out->cc_major != 10) return QWT_ERR_ARCH;
+  return QWT_OK;
+}
+
+static inline cudaStream_t as_stream(void* s) { return static_cast<cudaStream_t>(s); }
+
+static qwt_status check_calib_args(const float* fp_out, const float* q_out, int64_t rows, int32_t channels,
+                                   int64_t ld) {
+  if (fp_out == nullptr || q_out == nullptr) return QWT_ERR_NULL;
+  if (rows < 1 || channels < 1 || ld < channels) return QWT_ERR_SHAPE;
+  if (!aligned(fp_out, 16) || !aligned(q_out, 16) || (ld % 4) != 0) return QWT_ERR_ALIGN;
+  return QWT_OK;
+}
+
+qwt_status launch_cwac_reduce(const void* workspace, const CwacPlan& plan, int32_t channels, int64_t rows,
+                              double* stats_io, float* a, float* b, int32_t* n_degenerate, cudaStream_t st);
+
+}  // namespace qwt
+
+using namespace qwt;
+
+extern "C" {
+
+const char* qwt_version(void) { return "qwt2-b200 0.1 (sm_100a)"; }
+
+const char* qwt_status_string(qwt_status s) {
+  switch (s) {
+    case QWT_OK: return "ok";
+    case QWT_ERR_NULL: return "required pointer is NULL";
+    case QWT_ERR_SHAPE: return "invalid dimension";
+    case QWT_ERR_ALIGN: return "pointer or leading dimension not aligned";
+    case QWT_ERR_UNSUPPORTED: return "unsupported size multiple or enum value";
+    case QWT_ERR_WORKSPACE: return "workspace too small or misaligned";
+    case QWT_ERR_CUDA: return "CUDA call failed";
+    case QWT_ERR_TIMEOUT: return "device-side wait timed out";
+    case QWT_ERR_ARCH: return "device is not compute capability 10.x";
+    default: return "unknown status";
+  }
+}
+
+qwt_status qwt_last_cuda_error(int* cuda_err) {
+  if (cuda_err == nullptr) return QWT_ERR_NULL;
+  *cuda_err = tl_cuda_error;
+  return QWT_OK;
+}
+
+int64_t qwt_launch_count(void) { return tl_launches; }
+void qwt_launch_count_reset(void) { tl_launches = 0; }
+
+// ------------------------------------------------------------------------------------------------ calibration
+
+size_t qwt_cwac_workspace_bytes(int64_t rows, int32_t channels) {
+  if (rows < 1 || channels < 1) return 0;
+  return cwac_plan(rows, channels, 148).partial_bytes;
+}
+
+qwt_status qwt_cwac_calibrate(const float* fp_out, const float* q_out, int64_t rows, int32_t channels, int64_t ld,
+                              float* a, float* b, int32_t* n_degenerate, void* workspace, size_t workspace_bytes,
+                              void* stream) {
+  qwt_status s = check_calib_args(fp_out, q_out, rows, channels, ld);
+  if (s != QWT_OK) return s;
+  if (a == nullptr || b == nullptr || workspace == nullptr) return QWT_ERR_NULL;
+  const CwacPlan plan = cwac_plan(rows, channels, 148);
+  if (workspace_bytes < plan.partial_bytes || !aligned(workspace, 256)) return QWT_ERR_WORKSPACE;
+  DeviceInfo dev;
+  if ((s = current_device(&dev)) != QWT_OK) return s;
+  if ((s = launch_cwac_stats(fp_out, q_out, rows, channels, ld, nullptr, workspace, plan, as_stream(stream))) != QWT_OK)
+    return s;
+  return launch_cwac_reduce(workspace, plan, channels, rows, nullptr, a, b, n_degenerate, as_stream(stream));
+}
+
+qwt_status qwt_cwac_stats_accumulate(const float* fp_out, const float* q_out, int64_t rows, int32_t channels,
+                                     int64_t ld, double* stats, void* workspace, size_t workspace_bytes,
+                                     void* stream) {
+  qwt_status s = check_calib_args(fp_out, q_out, rows, channels, ld);
+  if (s != QWT_OK) return s;
+  if (stats == nullptr || workspace == nullptr) return QWT_ERR_NULL;
+  const CwacPlan plan = cwac_plan(rows, channels, 148);
+  if (workspace_bytes < plan.partial_bytes || !aligned(workspace, 256)) return QWT_ERR_WORKSPACE;
+  DeviceInfo dev;
+  if ((s = current_device(&dev)) != QWT_OK) return s;
+  if ((s = launch_cwac_stats(fp_out, q_out, rows, channels, ld, nullptr, workspace, plan, as_stream(stream))) != QWT_OK)
+    return s;
+  return launch_cwac_reduce(workspace, plan, channels, rows, stats, nullptr, nullptr, nullptr, as_stream(stream));
+}
+
+qwt_status qwt_cwac_solve(const double* stats, int32_t channels, float* a, float* b, int32_t* n_degenerate,
+                          void* stream) {
+  if (stats == nullptr || a == nullptr || b == nullptr) return QWT_ERR_NULL;
+  if (channels < 1) return QWT_ERR_SHAPE;
+  DeviceInfo dev;
+  qwt_status s = current_device(&dev);
+  if (s != QWT_OK) return s;
+  return launch_cwac_solve(stats, channels, a, b, n_degenerate, as_stream(stream));
+}
+
+// Host-matrix calibration: rows are cut into chunks; chunk i is copied into one of two staging slots while
+// chunk i-1 is reduced.  Staging layout: [stats 5*C doubles][out a,b,n_deg][2 slots x (fp, q) chunk][partials].
+namespace {
+struct HostCalibLayout {
+  int64_t chunk_rows;
+  size_t off_stats, off_out, off_slot[2], slot_bytes, off_ws, ws_bytes, total;
+};
+HostCalibLayout host_calib_layout(int64_t rows, int32_t channels) {
+  HostCalibLayout L{};
+  const int64_t target_bytes = 64ll << 20;   // per matrix per slot
+  int64_t cr = target_bytes / ((int64_t)channels * 4);
+  if (cr < 128) cr = 128;
+  if (cr > rows) cr = rows;
+  L.chunk_rows = cr;
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  size_t off = 0;
+  L.off_stats = off; off += up((size_t)5 * channels * 8);
+  L.off_out = off; off += up((size_t)2 * channels * 4 + 16);
+  L.slot_bytes = up((size_t)cr * channels * 4);
+  for (int i = 0; i < 2; ++i) { L.off_slot[i] = off; off += 2 * L.slot_bytes; }
+  L.ws_bytes = cwac_plan(cr, channels, 148).partial_bytes;
+  L.off_ws = off; off += up(L.ws_bytes);
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+size_t qwt_cwac_host_staging_bytes(int64_t rows, int32_t channels) {
+  if (rows < 1 || channels < 1) return 0;
+  return host_calib_layout(rows, channels).total;
+}
+
+qwt_status qwt_cwac_calibrate_host(const float* fp_out, const float* q_out, int64_t rows, int32_t channels,
+                                   int64_t ld, float* a, float* b, int32_t* n_degenerate, void* staging,
+                                   size_t staging_bytes, void* stream) {
+  if (fp_out == nullptr || q_out == nullptr || a == nullptr || b == nullptr || staging == nullptr) return QWT_ERR_NULL;
+  if (rows < 1 || channels < 1 || ld < channels) return QWT_ERR_SHAPE;
+  if ((channels % 4) != 0) return QWT_ERR_ALIGN;   // staged rows are packed with ld = channels
+  const HostCalibLayout L = host_calib_layout(rows, channels);
+  if (staging_bytes < L.total || !aligned(staging, 256)) return QWT_ERR_WORKSPACE;
+  DeviceInfo dev;
+  qwt_status s = current_device(&dev);
+  if (s != QWT_OK) return s;
+  cudaStream_t st = as_stream(stream);
+  uint8_t* base = static_cast<uint8_t*>(staging);
+  double* stats = reinterpret_cast<double*>(base + L.off_stats);
+  float* d_a = reinterpret_cast<float*>(base + L.off_out);
+  float* d_b = d_a + channels;
+  int32_t* d_nd = reinterpret_cast<int32_t*>(d_b + channels);
+
+  // a second stream carries the copies so that they overlap the reduction of the previous chunk
+  cudaStream_t copy_st;
+  cudaEvent_t copied[2], reduced[2];
+  QWT_CUDA_TRY(cudaStreamCreateWithFlags(&copy_st, cudaStreamNonBlocking));
+  for (int i = 0; i < 2; ++i) {
+    cudaEventCreateWithFlags(&copied[i], cudaEventDisableTiming);
+    cudaEventCreateWithFlags(&reduced[i], cudaEventDisableTiming);
+  }
+  qwt_status rc = QWT_OK;
+  cudaEvent_t start;
+  cudaEventCreateWithFlags(&start, cudaEventDisableTiming);
+  auto cleanup = [&]() {
+    cudaStreamSynchronize(copy_st);
+    cudaStreamDestroy(copy_st);
+    for (int i = 0; i < 2; ++i) { cudaEventDestroy(copied[i]); cudaEventDestroy(reduced[i]); }
+    cudaEventDestroy(start);
+  };
+#define QWT_HC_TRY(expr) do { cudaError_t _e = (expr); if (_e != cudaSuccess) { set_cuda_error((int)_e); rc = QWT_ERR_CUDA; goto done; } } while (0)
+  {
+    QWT_HC_TRY(cudaMemsetAsync(stats, 0, (size_t)5 * channels * 8, st));
+    QWT_HC_TRY(cudaEventRecord(start, st));
+    QWT_HC_TRY(cudaStreamWaitEvent(copy_st, start, 0));
+    int64_t r0 = 0;
+    for (int i = 0; r0 < rows; ++i, r0 += L.chunk_rows) {
+      const int slot = i & 1;
+      const int64_t nr = (rows - r0 < L.chunk_rows) ? rows - r0 : L.chunk_rows;
+      float* d_fp = reinterpret_cast<float*>(base + L.off_slot[slot]);
+      float* d_q = reinterpret_cast<float*>(base + L.off_slot[slot] + L.slot_bytes);
+      if (i >= 2) QWT_HC_TRY(cudaStreamWaitEvent(copy_st, reduced[slot], 0));
+      QWT_HC_TRY(cudaMemcpy2DAsync(d_fp, (size_t)channels * 4, fp_out + r0 * ld, (size_t)ld * 4, (size_t)channels * 4,
+                                   (size_t)nr, cudaMemcpyHostToDevice, copy_st));
+      QWT_HC_TRY(cudaMemcpy2DAsync(d_q, (size_t)channels * 4, q_out + r0 * ld, (size_t)ld * 4, (size_t)channels * 4,
+                                   (size_t)nr, cudaMemcpyHostToDevice, copy_st));
+      QWT_HC_TRY(cudaEventRecord(copied[slot], copy_st));
+      QWT_HC_TRY(cudaStreamWaitEvent(st, copied[slot], 0));
+      const CwacPlan plan = cwac_plan(nr, channels, 148);
+      if ((rc = launch_cwac_stats(d_fp, d_q, nr, channels, channels, nullptr, base + L.off_ws, plan, st)) != QWT_OK) goto done;
+      if ((rc = launch_cwac_reduce(base + L.off_ws, plan, channels, nr, stats, nullptr, nullptr, nullptr, st)) != QWT_OK) goto done;
+      QWT_HC_TRY(cudaEventRecord(reduced[slot], st));
+    }
+    if ((rc = launch_cwac_solve(stats, channels, d_a, d_b, d_nd, st)) != QWT_OK) goto done;
+    QWT_HC_TRY(cudaMemcpyAsync(a, d_a, (size_t)channels * 4, cudaMemcpyDeviceToHost, st));
+    QWT_HC_TRY(cudaMemcpyAsync(b, d_b, (size_t)channels * 4, cudaMemcpyDeviceToHost, st));
+    if (n_degenerate != nullptr) QWT_HC_TRY(cudaMemcpyAsync(n_degenerate, d_nd, 4, cudaMemcpyDeviceToHost, st));
+    QWT_HC_TRY(cudaStreamSynchronize(st));
+  }
+done:
+#undef QWT_HC_TRY
+  cleanup();
+  return rc;
+}
+
+// ------------------------------------------------------------------------------------------------ fold
+
+qwt_status qwt_cwac_fold(const float* w_scale, const float* bias, const float* a, const float* b, int32_t n,
+                         float* fscale, float* fbias, void* stream) {
+  if (w_scale == nullptr || fscale == nullptr || fbias == nullptr) return QWT_ERR_NULL;
+  if ((a == nullptr) != (b == nullptr)) return QWT_ERR_NULL;
+  if (n < 1) return QWT_ERR_SHAPE;
+  DeviceInfo dev;
+  qwt_status s = current_device(&dev);
+  if (s != QWT_OK) return s;
+  return launch_cwac_fold(w_scale, bias, a, b, n, fscale, fbias, as_stream(stream));
+}
+
+// ------------------------------------------------------------------------------------------------ forward
+
+static qwt_status check_forward_args(const void* X, const float* x_scale, const void* W, int32_t wfmt,
+                                     const float* fscale, const float* fbias, int32_t M, int32_t N, int32_t K,
+                                     int32_t out_mode, const void* Y, const float* y_scale, bool host_io) {
+  if (X == nullptr || W == nullptr || Y == nullptr) return QWT_ERR_NULL;
+  if (wfmt != QWT_W_INT8 && wfmt != QWT_W_INT4_PACKED) return QWT_ERR_UNSUPPORTED;
+  if (out_mode < QWT_OUT_INT8_PER_TOKEN || out_mode > QWT_OUT_INT32_ACC) return QWT_ERR_UNSUPPORTED;
+  if (out_mode != QWT_OUT_INT32_ACC && (x_scale == nullptr || fscale == nullptr || fbias == nullptr))
+    return QWT_ERR_NULL;
+  if (out_mode == QWT_OUT_INT8_PER_TOKEN && y_scale == nullptr) return QWT_ERR_NULL;
+  if (M < 1 || N < 1 || K < 1) return QWT_ERR_SHAPE;
+  if ((int64_t)M * (int64_t)N >= (int64_t)1 << 40) return QWT_ERR_SHAPE;
+  if (K > 131072) return QWT_ERR_SHAPE;   // 127^2 * K must stay below 2^31
+  const int kmul = wfmt == QWT_W_INT8 ? 16 : 32;
+  if (K % kmul != 0) return QWT_ERR_UNSUPPORTED;
+  const int nmul = out_mode == QWT_OUT_INT8_PER_TOKEN ? 16 : (out_mode == QWT_OUT_BF16 ? 8 : 4);
+  if (N % nmul != 0) return QWT_ERR_UNSUPPORTED;
+  if (!aligned(W, 16)) return QWT_ERR_ALIGN;
+  if (!host_io && (!aligned(X, 16) || !aligned(Y, 16))) return QWT_ERR_ALIGN;
+  return QWT_OK;
+}
+
+size_t qwt_qlinear_workspace_bytes(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode) {
+  if (M < 1 || N < 1 || K < 1) return 0;
+  DeviceInfo dev{};
+  dev.sm_count = 148;
+  QlinearPlan plan;
+  if (qlinear_plan(M, N, K, wfmt, out_mode, dev, &plan) != QWT_OK) return 0;
+  return plan.ws_total;
+}
+
+qwt_status qwt_qlinear_cwac_forward(const int8_t* X, const float* x_scale, const void* W, int32_t wfmt,
+                                    const float* fscale, const float* fbias, int32_t M, int32_t N, int32_t K,
+                                    int32_t out_mode, void* Y, float* y_scale, void* workspace,
+                                    size_t workspace_bytes, void* stream) {
+  qwt_status s = check_forward_args(X, x_scale, W, wfmt, fscale, fbias, M, N, K, out_mode, Y, y_scale, false);
+  if (s != QWT_OK) return s;
+  if (workspace == nullptr) return QWT_ERR_NULL;
+  DeviceInfo dev{};
+  dev.sm_count = 148;
+  QlinearPlan plan;
+  if ((s = qlinear_plan(M, N, K, wfmt, out_mode, dev, &plan)) != QWT_OK) return s;
+  if (workspace_bytes < plan.ws_total || !aligned(workspace, 256)) return QWT_ERR_WORKSPACE;
+  DeviceInfo real;
+  if ((s = current_device(&real)) != QWT_OK) return s;
+  if (real.sm_count < plan.grid) return QWT_ERR_ARCH;   // the persistent grid must be co-resident
+  return launch_qlinear(X, x_scale, W, wfmt, fscale, fbias, M, N, K, out_mode, Y, y_scale, workspace, plan,
+                        as_stream(stream));
+}
+
+qwt_status qwt_qlinear_check_status(const void* workspace, void* stream, int32_t* device_status) {
+  if (workspace == nullptr) return QWT_ERR_NULL;
+  QWT_CUDA_TRY(cudaStreamSynchronize(as_stream(stream)));
+  uint32_t word = 0;
+  QWT_CUDA_TRY(cudaMemcpy(&word, workspace, sizeof(word), cudaMemcpyDeviceToHost));
+  if (device_status != nullptr) *device_status = (int32_t)word;
+  return word == 0 ? QWT_OK : QWT_ERR_TIMEOUT;
+}
+
+namespace {
+struct HostFwdLayout {
+  size_t off_x, off_xs, off_y, off_ys, off_ws, total;
+  size_t x_bytes, y_bytes;
+};
+HostFwdLayout host_fwd_layout(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode) {
+  HostFwdLayout L{};
+  auto up = [](size_t x) { return (x + 255) / 256 * 256; };
+  const size_t esz = out_mode == QWT_OUT_INT8_PER_TOKEN ? 1 : (out_mode == QWT_OUT_BF16 ? 2 : 4);
+  L.x_bytes = (size_t)M * K;
+  L.y_bytes = (size_t)M * N * esz;
+  size_t off = 0;
+  L.off_x = off; off += up(L.x_bytes);
+  L.off_xs = off; off += up((size_t)M * 4);
+  L.off_y = off; off += up(L.y_bytes);
+  L.off_ys = off; off += up((size_t)M * 4);
+  L.off_ws = off; off += up(qwt_qlinear_workspace_bytes(M, N, K, wfmt, out_mode));
+  L.total = off;
+  return L;
+}
+}  // namespace
+
+size_t qwt_qlinear_host_staging_bytes(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode) {
+  if (M < 1 || N < 1 || K < 1) return 0;
+  return host_fwd_layout(M, N, K, wfmt, out_mode).total;
+}
+
+qwt_status qwt_qlinear_cwac_forward_host(const int8_t* X, const float* x_scale, const void* W, int32_t wfmt,
+                                         const float* fscale, const float* fbias, int32_t M, int32_t N, int32_t K,
+                                         int32_t out_mode, void* Y, float* y_scale, void* staging,
+                                         size_t staging_bytes, void* stream) {
+  qwt_status s = check_forward_args(X, x_scale, W, wfmt, fscale, fbias, M, N, K, out_mode, Y, y_scale, true);
+  if (s != QWT_OK) return s;
+  if (staging == nullptr) return QWT_ERR_NULL;
+  const HostFwdLayout L = host_fwd_layout(M, N, K, wfmt, out_mode);
+  if (staging_bytes < L.total || !aligned(staging, 256)) return QWT_ERR_WORKSPACE;
+  cudaStream_t st = as_stream(stream);
+  uint8_t* base = static_cast<uint8_t*>(staging);
+  int8_t* d_x = reinterpret_cast<int8_t*>(base + L.off_x);
+  float* d_xs = reinterpret_cast<float*>(base + L.off_xs);
+  void* d_y = base + L.off_y;
+  float* d_ys = reinterpret_cast<float*>(base + L.off_ys);
+  QWT_CUDA_TRY(cudaMemcpyAsync(d_x, X, L.x_bytes, cudaMemcpyHostToDevice, st));
+  if (x_scale != nullptr) QWT_CUDA_TRY(cudaMemcpyAsync(d_xs, x_scale, (size_t)M * 4, cudaMemcpyHostToDevice, st));
+  s = qwt_qlinear_cwac_forward(d_x, x_scale ? d_xs : nullptr, W, wfmt, fscale, fbias, M, N, K, out_mode, d_y,
+                               out_mode == QWT_OUT_INT8_PER_TOKEN ? d_ys : nullptr, base + L.off_ws,
+                               L.total - L.off_ws, st);
+  if (s != QWT_OK) return s;
+  QWT_CUDA_TRY(cudaMemcpyAsync(Y, d_y, L.y_bytes, cudaMemcpyDeviceToHost, st));
+  if (out_mode == QWT_OUT_INT8_PER_TOKEN)
+    QWT_CUDA_TRY(cudaMemcpyAsync(y_scale, d_ys, (size_t)M * 4, cudaMemcpyDeviceToHost, st));
+  QWT_CUDA_TRY(cudaStreamSynchronize(st));
+  return QWT_OK;
+}
+
+// ------------------------------------------------------------------------------------------------ support
+
+qwt_status qwt_quantize_rows_i8(const float* X, int64_t rows, int32_t cols, int64_t ld, int32_t qmax, int8_t* Xq,
+                                float* scale, void* stream) {
+  if (X == nullptr || Xq == nullptr || scale == nullptr) return QWT_ERR_NULL;
+  if (rows < 1 || cols < 1 || ld < cols || rows > (int64_t)8 * 2147483647) return QWT_ERR_SHAPE;
+  if (qmax < 1 || qmax > 127) return QWT_ERR_UNSUPPORTED;
+  DeviceInfo dev;
+  qwt_status s = current_device(&dev);
+  if (s != QWT_OK) return s;
+  return launch_quantize_rows(X, rows, cols, ld, qmax, Xq, scale, as_stream(stream));
+}
+
+qwt_status qwt_pack_int4(const int8_t* codes, int64_t rows, int32_t cols, uint8_t* packed, void* stream) {
+  if (codes == nullptr || packed == nullptr) return QWT_ERR_NULL;
+  if (rows < 1 || cols < 2) return QWT_ERR_SHAPE;
+  if ((cols % 2) != 0) return QWT_ERR_UNSUPPORTED;
+  DeviceInfo dev;
+  qwt_status s = current_device(&dev);
+  if (s != QWT_OK) return s;
+  return launch_pack_int4(codes, rows, cols, packed, as_stream(stream));
+}
+
+}  // extern "C"

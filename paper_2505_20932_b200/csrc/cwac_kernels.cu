@@ -1,0 +1,318 @@
+// CWAC calibration (Section 3.3, Eq. 3-5), fold (Section 3.4, Eq. 9-11) and the symmetric
+// row quantizer (Eq. 1-2 with zero-point 0).  All kernels here are bandwidth bound.
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "qwt2_internal.h"
+
+namespace qwt {
+
+// ------------------------------------------------------------------------------------------------
+// Statistics pass.
+//
+// Grid = (column slabs of 128 channels) x (row chunks).  A block is 32 x 8 threads: a warp reads one
+// row's 128 channels of q and of f as two coalesced 512-byte requests (16 bytes per lane); the eight
+// warps of the block walk eight rows at a time.  Every thread owns 4 channels and keeps, for each of
+// them, four running sums of the values *shifted by the chunk's first row* (dq = q - q0, df = f - f0):
+//     sum dq, sum df, sum dq*df, sum dq*dq.
+// The sums run in FP32 for FLUSH rows and are then added to FP64 accumulators, so FP32 only ever adds
+// a handful of terms of the size of the channel's spread (the shift removes the mean), which keeps the
+// variance and covariance accurate for channels whose mean is far from zero.  At the end of the chunk
+// the shifted sums are turned back into raw sums in FP64 and written as one partial per (chunk, sum,
+// channel).  No atomics: a second kernel adds the partials in chunk order, so results are reproducible.
+// ------------------------------------------------------------------------------------------------
+constexpr int kStatsTX = 32;
+constexpr int kStatsTY = 8;
+constexpr int kStatsThreads = kStatsTX * kStatsTY;
+constexpr int kSlabChannels = kStatsTX * 4;
+constexpr int kFlushRows = 16;   // rows per thread between FP32 -> FP64 flushes
+constexpr int kBatchRows = 4;    // rows per thread whose loads are issued together
+
+__device__ __forceinline__ float4 ld_stream(const float* p) {
+  return __ldcs(reinterpret_cast<const float4*>(p));
+}
+
+__global__ void __launch_bounds__(kStatsThreads)
+cwac_stats_kernel(const float* __restrict__ fp_out, const float* __restrict__ q_out, int64_t rows, int channels,
+                  int64_t ld, int64_t chunk_rows, double* __restrict__ partial, int cpad) {
+  const int tx = threadIdx.x & (kStatsTX - 1);
+  const int ty = threadIdx.x / kStatsTX;
+  const int c0 = blockIdx.x * kSlabChannels + tx * 4;
+  const int64_t r0 = (int64_t)blockIdx.y * chunk_rows;
+  const int64_t r1 = (r0 + chunk_rows < rows) ? r0 + chunk_rows : rows;
+  // c0 + 3 may pass `channels`, but ld % 4 == 0 and ld >= channels keep the 16-byte load inside the row
+  const bool active = c0 < channels;
+
+  float kq[4] = {0.f, 0.f, 0.f, 0.f}, kf[4] = {0.f, 0.f, 0.f, 0.f};
+  if (active) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(q_out + r0 * ld + c0));
+    const float4 b = __ldg(reinterpret_cast<const float4*>(fp_out + r0 * ld + c0));
+    kq[0] = a.x; kq[1] = a.y; kq[2] = a.z; kq[3] = a.w;
+    kf[0] = b.x; kf[1] = b.y; kf[2] = b.z; kf[3] = b.w;
+  }
+
+  double acc[16];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) acc[i] = 0.0;
+
+  if (active) {
+    const float* qp = q_out + c0;
+    const float* fp = fp_out + c0;
+    for (int64_t rb = r0 + ty; rb < r1; rb += (int64_t)kStatsTY * kFlushRows) {
+      float s[16];
+#pragma unroll
+      for (int i = 0; i < 16; ++i) s[i] = 0.f;
+#pragma unroll
+      for (int g = 0; g < kFlushRows / kBatchRows; ++g) {
+        float4 qv[kBatchRows], fv[kBatchRows];
+#pragma unroll
+        for (int i = 0; i < kBatchRows; ++i) {
+          const int64_t r = rb + (int64_t)(g * kBatchRows + i) * kStatsTY;
+          if (r < r1) {
+            qv[i] = ld_stream(qp + r * ld);
+            fv[i] = ld_stream(fp + r * ld);
+          } else {  // shifted value 0: contributes nothing
+            qv[i] = make_float4(kq[0], kq[1], kq[2], kq[3]);
+            fv[i] = make_float4(kf[0], kf[1], kf[2], kf[3]);
+          }
+        }
+#pragma unroll
+        for (int i = 0; i < kBatchRows; ++i) {
+          const float qa[4] = {qv[i].x, qv[i].y, qv[i].z, qv[i].w};
+          const float fa[4] = {fv[i].x, fv[i].y, fv[i].z, fv[i].w};
+#pragma unroll
+          for (int j = 0; j < 4; ++j) {
+            const float dq = qa[j] - kq[j];
+            const float df = fa[j] - kf[j];
+            s[0 + j] += dq;
+            s[4 + j] += df;
+            s[8 + j] = fmaf(dq, df, s[8 + j]);
+            s[12 + j] = fmaf(dq, dq, s[12 + j]);
+          }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < 16; ++i) acc[i] += (double)s[i];
+    }
+  }
+
+  // block reduction over the 8 row lanes, in a fixed order
+  __shared__ double red[kStatsTY][16][kStatsTX];
+  __shared__ float shift_q[kSlabChannels], shift_f[kSlabChannels];
+#pragma unroll
+  for (int i = 0; i < 16; ++i) red[ty][i][tx] = acc[i];
+  if (ty == 0) {
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      shift_q[tx * 4 + j] = kq[j];
+      shift_f[tx * 4 + j] = kf[j];
+    }
+  }
+  __syncthreads();
+  if (threadIdx.x < kSlabChannels) {
+    const int ch = threadIdx.x;           // channel inside the slab
+    const int ltx = ch >> 2, j = ch & 3;
+    const int c = blockIdx.x * kSlabChannels + ch;
+    double sd[4];
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      double t = 0.0;
+#pragma unroll
+      for (int y = 0; y < kStatsTY; ++y) t += red[y][s * 4 + j][ltx];
+      sd[s] = t;
+    }
+    const double nb = (double)(r1 - r0);
+    const double Kq = (double)shift_q[ch], Kf = (double)shift_f[ch];
+    // raw sums from the shifted ones
+    const double Sq = sd[0] + nb * Kq;
+    const double Sf = sd[1] + nb * Kf;
+    const double Sqf = sd[2] + Kf * sd[0] + Kq * sd[1] + nb * Kq * Kf;
+    const double Sqq = sd[3] + 2.0 * Kq * sd[0] + nb * Kq * Kq;
+    double* out = partial + (size_t)blockIdx.y * 4 * cpad + c;
+    out[0 * (size_t)cpad] = Sq;
+    out[1 * (size_t)cpad] = Sf;
+    out[2 * (size_t)cpad] = Sqf;
+    out[3 * (size_t)cpad] = Sqq;
+  }
+}
+
+// Closed form of Eq. 4-5 from the five sums of one channel.
+__device__ __forceinline__ void cwac_solve_channel(double n, double Sq, double Sf, double Sqf, double Sqq,
+                                                   float* a, float* b, int* degenerate) {
+  const double mq = Sq / n, mf = Sf / n;
+  const double msq = Sqq / n;
+  const double var = msq - mq * mq;
+  const double cov = Sqf / n - mq * mf;
+  double alpha;
+  if (var <= 1e-12 * msq) {   // constant column / single row: every alpha minimises Eq. 3, take 1
+    alpha = 1.0;
+    *degenerate = 1;
+  } else {
+    alpha = cov / var;
+    *degenerate = 0;
+  }
+  *a = (float)alpha;
+  *b = (float)(mf - alpha * mq);
+}
+
+// Adds the partials in chunk order.  stats_io (may be NULL): running statistics to update.
+// a, b (may be NULL): solve after the reduction (one-shot calibration).
+__global__ void __launch_bounds__(128)
+cwac_reduce_kernel(const double* __restrict__ partial, int chunks, int cpad, int channels, double n_rows,
+                   double* __restrict__ stats_io, float* __restrict__ a, float* __restrict__ b,
+                   int* __restrict__ n_degenerate) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= channels) return;
+  double s[4] = {0.0, 0.0, 0.0, 0.0};
+  for (int k = 0; k < chunks; ++k) {
+    const double* p = partial + (size_t)k * 4 * cpad + c;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) s[i] += p[(size_t)i * cpad];
+  }
+  double n = n_rows;
+  if (stats_io != nullptr) {
+    n += stats_io[c];
+#pragma unroll
+    for (int i = 0; i < 4; ++i) s[i] += stats_io[(size_t)(i + 1) * channels + c];
+    stats_io[c] = n;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) stats_io[(size_t)(i + 1) * channels + c] = s[i];
+  }
+  if (a != nullptr) {
+    int deg;
+    cwac_solve_channel(n, s[0], s[1], s[2], s[3], &a[c], &b[c], &deg);
+    if (deg && n_degenerate != nullptr) atomicAdd(n_degenerate, 1);
+  }
+}
+
+__global__ void __launch_bounds__(128)
+cwac_solve_kernel(const double* __restrict__ stats, int channels, float* __restrict__ a, float* __restrict__ b,
+                  int* __restrict__ n_degenerate) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= channels) return;
+  int deg;
+  cwac_solve_channel(stats[c], stats[(size_t)channels + c], stats[2 * (size_t)channels + c],
+                     stats[3 * (size_t)channels + c], stats[4 * (size_t)channels + c], &a[c], &b[c], &deg);
+  if (deg && n_degenerate != nullptr) atomicAdd(n_degenerate, 1);
+}
+
+// Eq. 11: the static part of the multiplier and the additive term.
+__global__ void __launch_bounds__(256)
+cwac_fold_kernel(const float* __restrict__ w_scale, const float* __restrict__ bias, const float* __restrict__ a,
+                 const float* __restrict__ b, int n, float* __restrict__ fscale, float* __restrict__ fbias) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const float ai = a ? a[i] : 1.0f;
+  const float bi = b ? b[i] : 0.0f;
+  const float bs = bias ? bias[i] : 0.0f;
+  fscale[i] = ai * w_scale[i];
+  fbias[i] = fmaf(ai, bs, bi);
+}
+
+// Eq. 1-2 with zero-point 0: one warp per row, two passes over the row (the second hits cache).
+__global__ void __launch_bounds__(256)
+quantize_rows_kernel(const float* __restrict__ X, int64_t rows, int cols, int64_t ld, float qmax,
+                     int8_t* __restrict__ Xq, float* __restrict__ scale) {
+  const int lane = threadIdx.x & 31;
+  const int64_t r = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= rows) return;
+  const float* x = X + r * ld;
+  float m = 0.f;
+  for (int c = lane; c < cols; c += 32) m = fmaxf(m, fabsf(x[c]));
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+  const float s = __fdiv_rn(m, qmax);
+  if (lane == 0) scale[r] = s;
+  int8_t* q = Xq + r * (int64_t)cols;
+  if (s > 0.f) {
+    for (int c = lane; c < cols; c += 32) {
+      float v = rintf(__fdiv_rn(x[c], s));
+      v = fminf(fmaxf(v, -qmax), qmax);
+      q[c] = (int8_t)(int)v;
+    }
+  } else {
+    for (int c = lane; c < cols; c += 32) q[c] = 0;
+  }
+}
+
+__global__ void __launch_bounds__(256)
+pack_int4_kernel(const int8_t* __restrict__ codes, int64_t n_bytes, uint8_t* __restrict__ packed) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_bytes) return;
+  const int lo = codes[2 * i], hi = codes[2 * i + 1];
+  packed[i] = (uint8_t)((lo & 0xF) | ((hi & 0xF) << 4));
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+
+CwacPlan cwac_plan(int64_t rows, int32_t channels, int /*sm_count*/) {
+  // The plan is a function of the shape only, so that the workspace size and the summation order
+  // (hence the bits of the result) do not depend on the device.  1184 = 148 SMs x 8 resident blocks.
+  CwacPlan p;
+  p.slabs = (channels + kSlabChannels - 1) / kSlabChannels;
+  p.cpad = p.slabs * kSlabChannels;
+  const int64_t target_blocks = 1184;
+  int64_t chunks = (target_blocks + p.slabs - 1) / p.slabs;
+  const int64_t min_chunk = (int64_t)kStatsTY * kFlushRows;     // at least one full flush per thread
+  int64_t max_chunks = (rows + min_chunk - 1) / min_chunk;
+  if (chunks > max_chunks) chunks = max_chunks;
+  if (chunks < 1) chunks = 1;
+  int64_t chunk_rows = (rows + chunks - 1) / chunks;
+  chunk_rows = (chunk_rows + kStatsTY - 1) / kStatsTY * kStatsTY;
+  p.chunk_rows = chunk_rows;
+  p.chunks = (int)((rows + chunk_rows - 1) / chunk_rows);
+  p.partial_bytes = (size_t)p.chunks * 4 * p.cpad * sizeof(double);
+  return p;
+}
+
+qwt_status launch_cwac_stats(const float* fp_out, const float* q_out, int64_t rows, int32_t channels, int64_t ld,
+                             double* /*unused*/, void* workspace, const CwacPlan& plan, cudaStream_t st) {
+  dim3 grid(plan.slabs, plan.chunks);
+  cwac_stats_kernel<<<grid, kStatsThreads, 0, st>>>(fp_out, q_out, rows, channels, ld, plan.chunk_rows,
+                                                    static_cast<double*>(workspace), plan.cpad);
+  QWT_LAUNCH_CHECK();
+  return QWT_OK;
+}
+
+qwt_status launch_cwac_reduce(const void* workspace, const CwacPlan& plan, int32_t channels, int64_t rows,
+                              double* stats_io, float* a, float* b, int32_t* n_degenerate, cudaStream_t st) {
+  if (a != nullptr && n_degenerate != nullptr) QWT_CUDA_TRY(cudaMemsetAsync(n_degenerate, 0, sizeof(int32_t), st));
+  cwac_reduce_kernel<<<(channels + 127) / 128, 128, 0, st>>>(static_cast<const double*>(workspace), plan.chunks,
+                                                             plan.cpad, channels, (double)rows, stats_io, a, b,
+                                                             n_degenerate);
+  QWT_LAUNCH_CHECK();
+  return QWT_OK;
+}
+
+qwt_status launch_cwac_solve(const double* stats, int32_t channels, float* a, float* b, int32_t* n_degenerate,
+                             cudaStream_t st) {
+  if (n_degenerate != nullptr) QWT_CUDA_TRY(cudaMemsetAsync(n_degenerate, 0, sizeof(int32_t), st));
+  cwac_solve_kernel<<<(channels + 127) / 128, 128, 0, st>>>(stats, channels, a, b, n_degenerate);
+  QWT_LAUNCH_CHECK();
+  return QWT_OK;
+}
+
+qwt_status launch_cwac_fold(const float* w_scale, const float* bias, const float* a, const float* b, int32_t n,
+                            float* fscale, float* fbias, cudaStream_t st) {
+  cwac_fold_kernel<<<(n + 255) / 256, 256, 0, st>>>(w_scale, bias, a, b, n, fscale, fbias);
+  QWT_LAUNCH_CHECK();
+  return QWT_OK;
+}
+
+qwt_status launch_quantize_rows(const float* X, int64_t rows, int32_t cols, int64_t ld, int32_t qmax, int8_t* Xq,
+                                float* scale, cudaStream_t st) {
+  const int rows_per_block = 8;
+  const int64_t blocks = (rows + rows_per_block - 1) / rows_per_block;
+  quantize_rows_kernel<<<(unsigned)blocks, rows_per_block * 32, 0, st>>>(X, rows, cols, ld, (float)qmax, Xq, scale);
+  QWT_LAUNCH_CHECK();
+  return QWT_OK;
+}
+
+qwt_status launch_pack_int4(const int8_t* codes, int64_t rows, int32_t cols, uint8_t* packed, cudaStream_t st) {
+  const int64_t n_bytes = rows * (int64_t)(cols / 2);
+  pack_int4_kernel<<<(unsigned)((n_bytes + 255) / 256), 256, 0, st>>>(codes, n_bytes, packed);
+  QWT_LAUNCH_CHECK();
+  return QWT_OK;
+}
+
+}  // namespace qwt

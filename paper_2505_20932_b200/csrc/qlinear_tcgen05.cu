@@ -1,0 +1,554 @@
+// CWAC-fused quantized linear layer (Section 3.4, Eq. 6-11 with zero-points 0) for sm_100a.
+//
+// One persistent, warp-specialised kernel:
+//   warp 0      TMA producer: non-multicast cp.async.bulk.tensor loads of the X tile [128 x 128 B] and the
+//               W tile [BN x 128 B] into a ring of 128-byte-swizzled shared-memory stages
+//   warp 1      MMA issuer: one thread issues tcgen05.mma kind::i8 (128 x BN x 32 per instruction) into a
+//               TMEM accumulator; tcgen05.commit releases the stage / publishes the accumulator
+//   warps 2-5   epilogue: tcgen05.ld of the INT32 accumulators, z = fma(float(acc) * x_scale[m], fscale[n],
+//               fbias[n]) (the folded M' and offset of Eq. 10-11), then the output stage.  TMEM holds
+//               512 / BN accumulator buffers so the next tile's mainloop overlaps this epilogue.
+//
+// Per-token INT8 output needs max_n |z[m, n]| over the whole row, but a CTA owns only BN columns of it.
+// Tiles are numbered strip-major (all column tiles of rows 0-127, then of rows 128-255, ...) and CTA c
+// takes tiles c, c + G, c + 2G, ...  After its mainloop a tile publishes its per-row maxima with
+// atomicMax on the float bit pattern (non-negative floats order like unsigned integers) and increments
+// its strip's arrival counter; it then waits until the counter shows every column tile of the strip,
+// re-reads its accumulator from TMEM (still resident) and emits the codes with the final row scale.
+// Progress: the lowest-numbered unpublished tile t can always run, because the tile that holds its
+// TMEM buffer (t - NACC*G) belongs to a strip whose tiles all have smaller numbers than t whenever
+// tiles_n <= G, so that strip is complete and its buffer is released.  The grid is launched
+// cooperatively so all G CTAs are resident.  Every wait is bounded; a wait that gives up records a code
+// in the workspace status word and the CTA tears down normally.
+#include <cuda.h>
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+#include <stdlib.h>
+
+#include <mutex>
+
+#include "ptx_sm100.cuh"
+#include "qwt2_internal.h"
+
+namespace qwt {
+
+namespace {
+
+constexpr int kBM = 128;           // rows of a CTA tile (= TMEM lanes)
+constexpr int kBK = 128;           // bytes of K per stage: one 128-byte swizzle row
+constexpr int kUmmaK = 32;         // K of one kind::i8 instruction
+constexpr int kTmemCols = 512;
+constexpr int kNumEpilogueWarps = 4;
+constexpr int kThreads = 32 * (2 + kNumEpilogueWarps);
+constexpr int kABytes = kBM * kBK;
+
+// status word codes (0 = clean)
+enum : uint32_t {
+  kStWaitEmpty = 1, kStWaitFull = 2, kStWaitTmemEmpty = 3, kStWaitTmemFull = 4, kStWaitStrip = 5,
+};
+
+struct QlParams {
+  const float* x_scale;
+  const float* fscale;
+  const float* fbias;
+  void* Y;
+  float* y_scale;
+  int M, N, K;
+  int tiles_n, num_tiles, num_kb;
+  uint32_t* status;
+  uint32_t* rowmax;     // [M] bit patterns of non-negative floats
+  uint32_t* counters;   // [tiles_m] arrivals of epilogue warps
+  uint32_t counter_target;
+  unsigned long long timeout_ns;
+};
+
+template <int BN>
+struct SmemLayout {
+  static constexpr int kBBytes = BN * kBK;
+  static constexpr int kStages = (BN == 256) ? 4 : 6;
+  static constexpr int kAcc = kTmemCols / BN;
+  static constexpr int kOffA = 0;
+  static constexpr int kOffB = kOffA + kStages * kABytes;
+  static constexpr int kOffFS = kOffB + kStages * kBBytes;         // float [epilogue warp][BN], private per warp
+  static constexpr int kOffFB = kOffFS + kNumEpilogueWarps * BN * 4;
+  static constexpr int kOffBars = kOffFB + kNumEpilogueWarps * BN * 4;   // full, empty, tfull, tempty, drain
+  static constexpr int kNumBars = 2 * kStages + 2 * kAcc + 1;
+  static constexpr int kOffMisc = kOffBars + kNumBars * 8;         // tmem base, abort word
+  static constexpr int kTotal = kOffMisc + 16;
+  static constexpr int kDynamic = kTotal + 1024;                   // slack to align the base to 1024
+};
+
+__device__ __forceinline__ float epilogue_z(uint32_t acc_bits, float xs, float fs, float fb) {
+  // Eq. 9 after the fold: (S_x acc) * (alpha S_W) + (alpha bias + beta)
+  return fmaf(__fmul_rn(__int2float_rn((int)acc_bits), xs), fs, fb);
+}
+
+__device__ __forceinline__ void st_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+  *reinterpret_cast<uint4*>(p) = make_uint4(a, b, c, d);
+}
+
+__device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
+  __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
+  return *reinterpret_cast<uint32_t*>(&v);
+}
+
+__device__ __forceinline__ uint32_t quant_code(float z, float ys) {
+  int q = __float2int_rn(__fdiv_rn(z, ys));
+  q = max(-127, min(127, q));
+  return (uint32_t)q & 0xFFu;
+}
+
+template <int BN, int OUT>
+__global__ void __launch_bounds__(kThreads, 1)
+qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const QlParams p) {
+  using L = SmemLayout<BN>;
+  extern __shared__ uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
+  uint8_t* sA = smem + L::kOffA;
+  uint8_t* sB = smem + L::kOffB;
+  float* sFS = reinterpret_cast<float*>(smem + L::kOffFS);
+  float* sFB = reinterpret_cast<float*>(smem + L::kOffFB);
+  uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kOffBars);
+  uint64_t* empty = full + L::kStages;
+  uint64_t* tfull = empty + L::kStages;
+  uint64_t* tempty = tfull + L::kAcc;
+  uint64_t* drain = tempty + L::kAcc;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kOffMisc);
+  volatile int* cta_abort = reinterpret_cast<volatile int*>(smem + L::kOffMisc + 4);
+
+  const int warp = threadIdx.x >> 5;
+  const int lane = threadIdx.x & 31;
+  const uint64_t tmo = p.timeout_ns;
+
+  if (threadIdx.x == 0) {
+    for (int i = 0; i < L::kStages; ++i) {
+      ptx::mbar_init(&full[i], 1);
+      ptx::mbar_init(&empty[i], 1);
+    }
+    for (int i = 0; i < L::kAcc; ++i) {
+      ptx::mbar_init(&tfull[i], 1);
+      ptx::mbar_init(&tempty[i], kNumEpilogueWarps);
+    }
+    ptx::mbar_init(drain, 1);
+    *cta_abort = 0;
+    ptx::fence_mbar_init();
+    ptx::prefetch_tensormap(&tmA);
+    ptx::prefetch_tensormap(&tmB);
+  }
+  if (warp == 1) {
+    ptx::tmem_alloc(tmem_slot, kTmemCols);
+    ptx::tmem_relinquish();
+  }
+  ptx::tc_fence_before();
+  __syncthreads();
+  ptx::tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  auto give_up = [&](uint32_t code) {
+    *cta_abort = 1;
+    atomicCAS(p.status, 0u, code);
+  };
+
+  if (warp == 0) {
+    // ------------------------------------------------------------------ TMA producer
+    if (lane == 0) {
+      uint32_t kbi = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+        const int m0 = (tile / p.tiles_n) * kBM;
+        const int n0 = (tile % p.tiles_n) * BN;
+        for (int kb = 0; kb < p.num_kb; ++kb, ++kbi) {
+          const uint32_t s = kbi % L::kStages;
+          if (!ptx::mbar_wait_bounded(&empty[s], ((kbi / L::kStages) & 1u) ^ 1u, cta_abort, tmo)) {
+            give_up(kStWaitEmpty);
+            ok = false;
+            break;
+          }
+          ptx::mbar_arrive_expect_tx(&full[s], kABytes + L::kBBytes);
+          ptx::tma_load_2d(sA + s * kABytes, &tmA, kb * kBK, m0, &full[s]);
+          ptx::tma_load_2d(sB + s * L::kBBytes, &tmB, kb * kBK, n0, &full[s]);
+        }
+      }
+      if (*cta_abort != 0) {
+        // let copies still in flight land before the CTA's shared memory is released
+        const uint32_t first = kbi > (uint32_t)L::kStages ? kbi - L::kStages : 0u;
+        for (uint32_t j = first; j < kbi; ++j) {
+          uint32_t polls = 0;
+          while (!ptx::mbar_try_wait(&full[j % L::kStages], (j / L::kStages) & 1u) && ++polls < (1u << 16)) {
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------------------------------------------ MMA issuer
+    if (lane == 0) {
+      constexpr uint32_t idesc = ptx::make_idesc_i8(kBM, BN);
+      const uint32_t a_base = ptx::smem_u32(sA), b_base = ptx::smem_u32(sB);
+      uint32_t kbi = 0, it = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x, ++it) {
+        const uint32_t buf = it % L::kAcc;
+        if (!ptx::mbar_wait_bounded(&tempty[buf], ((it / L::kAcc) & 1u) ^ 1u, cta_abort, tmo)) {
+          give_up(kStWaitTmemEmpty);
+          break;
+        }
+        ptx::tc_fence_after();
+        const uint32_t d_tmem = tmem_base + buf * BN;
+        for (int kb = 0; kb < p.num_kb; ++kb, ++kbi) {
+          const uint32_t s = kbi % L::kStages;
+          if (!ptx::mbar_wait_bounded(&full[s], (kbi / L::kStages) & 1u, cta_abort, tmo)) {
+            give_up(kStWaitFull);
+            ok = false;
+            break;
+          }
+          ptx::tc_fence_after();
+          const uint64_t a_desc = ptx::make_kmajor_sw128_desc(a_base + s * kABytes);
+          const uint64_t b_desc = ptx::make_kmajor_sw128_desc(b_base + s * L::kBBytes);
+#pragma unroll
+          for (int k = 0; k < kBK / kUmmaK; ++k) {
+            // next 32 bytes of K inside the swizzled 128-byte row: start address + 32 B (>> 4 = 2)
+            ptx::mma_i8_ss(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+          }
+          ptx::tc_commit(&empty[s]);
+        }
+        if (ok) ptx::tc_commit(&tfull[buf]);
+      }
+      if (*cta_abort != 0) {
+        // make sure no MMA is still running when TMEM is released
+        ptx::tc_commit(drain);
+        uint32_t polls = 0;
+        while (!ptx::mbar_try_wait(drain, 0) && ++polls < (1u << 16)) {
+        }
+      }
+    }
+  } else {
+    // ------------------------------------------------------------------ epilogue warps
+    const int qd = warp & 3;                       // TMEM lane quadrant this warp may read
+    // each warp stages the tile's fscale / fbias in its own slice (no cross-warp barrier to get stuck on)
+    float* fs = sFS + (warp - 2) * BN;
+    float* fb = sFB + (warp - 2) * BN;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x, ++it) {
+      const uint32_t buf = it % L::kAcc;
+      const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
+      const int m0 = tm * kBM, n0 = tn * BN;
+      __syncwarp();   // every lane is done with the previous tile's slice
+      if (OUT != QWT_OUT_INT32_ACC) {
+        for (int i = lane; i < BN; i += 32) {
+          const int c = n0 + i;
+          fs[i] = c < p.N ? __ldg(p.fscale + c) : 0.f;
+          fb[i] = c < p.N ? __ldg(p.fbias + c) : 0.f;
+        }
+      }
+      __syncwarp();
+      const int row = m0 + qd * 32 + lane;
+      const bool row_ok = row < p.M;
+      float xs = 0.f;
+      if (OUT != QWT_OUT_INT32_ACC && row_ok) xs = __ldg(p.x_scale + row);
+
+      if (!ptx::mbar_wait_bounded(&tfull[buf], (it / L::kAcc) & 1u, cta_abort, tmo)) {
+        give_up(kStWaitTmemFull);
+        break;
+      }
+      ptx::tc_fence_after();
+      const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + buf * BN;
+
+      if (OUT == QWT_OUT_INT8_PER_TOKEN) {
+        // pass 1: row maxima of |z| over this tile's columns
+        float amax = 0.f;
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          uint32_t r[32];
+          ptx::tmem_ld_32x32b_x32(taddr + ch * 32, r);
+          ptx::tmem_ld_wait();
+#pragma unroll
+          for (int j = 0; j < 32; ++j) {
+            const int c = ch * 32 + j;
+            amax = fmaxf(amax, fabsf(epilogue_z(r[j], xs, fs[c], fb[c])));   // columns >= N give |0*..+0| = 0
+          }
+        }
+        if (row_ok) atomicMax(p.rowmax + row, __float_as_uint(amax));
+        __threadfence();
+        __syncwarp();
+        if (lane == 0) {
+          ptx::red_release_gpu_add(p.counters + tm, 1u);
+          // wait for every column tile of this strip
+          uint32_t polls = 0;
+          uint64_t t0 = 0;
+          while (ptx::ld_acquire_gpu(p.counters + tm) < p.counter_target) {
+            if ((++polls & 63u) == 0u) {
+              const uint64_t now = ptx::globaltimer_ns();
+              if (t0 == 0) t0 = now;
+              if (*cta_abort != 0 || now - t0 > tmo || ptx::ld_acquire_gpu(p.status) != 0u) {
+                give_up(kStWaitStrip);
+                break;
+              }
+            }
+          }
+        }
+        __syncwarp();
+        if (*cta_abort != 0) {
+          ok = false;
+          break;
+        }
+        __threadfence();
+        float ys = 0.f;
+        if (row_ok) {
+          const float fin = __uint_as_float(__ldcg(p.rowmax + row));
+          ys = __fdiv_rn(fin, 127.f);
+          if (tn == 0) p.y_scale[row] = ys;
+        }
+        // pass 2: codes with the final scale
+        int8_t* yrow = static_cast<int8_t*>(p.Y) + (size_t)row * p.N + n0;
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          uint32_t r[32];
+          ptx::tmem_ld_32x32b_x32(taddr + ch * 32, r);
+          ptx::tmem_ld_wait();
+          uint32_t w[8];
+#pragma unroll
+          for (int g = 0; g < 8; ++g) {
+            uint32_t word = 0;
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const int c = ch * 32 + g * 4 + j;
+              const float z = epilogue_z(r[g * 4 + j], xs, fs[c], fb[c]);
+              const uint32_t code = ys > 0.f ? quant_code(z, ys) : 0u;
+              word |= code << (8 * j);
+            }
+            w[g] = word;
+          }
+          if (row_ok) {
+            const int c0 = n0 + ch * 32;
+            if (c0 + 16 <= p.N) st_v4(yrow + ch * 32, w[0], w[1], w[2], w[3]);
+            if (c0 + 32 <= p.N) st_v4(yrow + ch * 32 + 16, w[4], w[5], w[6], w[7]);
+          }
+        }
+      } else {
+        for (int ch = 0; ch < BN / 32; ++ch) {
+          uint32_t r[32];
+          ptx::tmem_ld_32x32b_x32(taddr + ch * 32, r);
+          ptx::tmem_ld_wait();
+          const int c0 = n0 + ch * 32;
+          if (OUT == QWT_OUT_INT32_ACC) {
+            if (row_ok) {
+              int32_t* yrow = static_cast<int32_t*>(p.Y) + (size_t)row * p.N + c0;
+#pragma unroll
+              for (int g = 0; g < 8; ++g)
+                if (c0 + g * 4 + 4 <= p.N) st_v4(yrow + g * 4, r[g * 4], r[g * 4 + 1], r[g * 4 + 2], r[g * 4 + 3]);
+            }
+          } else {
+            float z[32];
+#pragma unroll
+            for (int j = 0; j < 32; ++j) z[j] = epilogue_z(r[j], xs, fs[ch * 32 + j], fb[ch * 32 + j]);
+            if (OUT == QWT_OUT_FP32) {
+              if (row_ok) {
+                float* yrow = static_cast<float*>(p.Y) + (size_t)row * p.N + c0;
+#pragma unroll
+                for (int g = 0; g < 8; ++g)
+                  if (c0 + g * 4 + 4 <= p.N)
+                    st_v4(yrow + g * 4, __float_as_uint(z[g * 4]), __float_as_uint(z[g * 4 + 1]),
+                          __float_as_uint(z[g * 4 + 2]), __float_as_uint(z[g * 4 + 3]));
+              }
+            } else {  // BF16
+              if (row_ok) {
+                __nv_bfloat16* yrow = static_cast<__nv_bfloat16*>(p.Y) + (size_t)row * p.N + c0;
+#pragma unroll
+                for (int g = 0; g < 4; ++g)
+                  if (c0 + g * 8 + 8 <= p.N)
+                    st_v4(yrow + g * 8, pack_bf16x2(z[g * 8], z[g * 8 + 1]), pack_bf16x2(z[g * 8 + 2], z[g * 8 + 3]),
+                          pack_bf16x2(z[g * 8 + 4], z[g * 8 + 5]), pack_bf16x2(z[g * 8 + 6], z[g * 8 + 7]));
+              }
+            }
+          }
+        }
+      }
+      // accumulator buffer is free again
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) ptx::mbar_arrive(&tempty[buf]);
+    }
+  }
+
+  // ------------------------------------------------------------------ teardown
+  __syncwarp();
+  ptx::tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    ptx::tc_fence_after();
+    ptx::tmem_dealloc(tmem_base, kTmemCols);
+  }
+}
+
+// ------------------------------------------------------------------------------------------------ host side
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* sym = nullptr;
+    cudaDriverEntryPointQueryResult qres;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &sym, cudaEnableDefault, &qres) == cudaSuccess &&
+        qres == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(sym);
+  });
+  return fn;
+}
+
+// Row-major byte matrix [rows, row_bytes] -> map with a box of {box_bytes, box_rows}.
+bool make_byte_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t row_bytes, uint32_t box_bytes,
+                   uint32_t box_rows, CUtensorMapSwizzle swz) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[2] = {row_bytes, rows};
+  cuuint64_t strides[1] = {row_bytes};
+  cuuint32_t box[2] = {box_bytes, box_rows};
+  cuuint32_t estr[2] = {1, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+unsigned long long timeout_ns_from_env() {
+  static unsigned long long v = [] {
+    const char* e = getenv("QWT_TIMEOUT_MS");
+    unsigned long long ms = 2000;
+    if (e != nullptr) {
+      const long long x = atoll(e);
+      if (x > 0) ms = (unsigned long long)x;
+    }
+    return ms * 1000000ull;
+  }();
+  return v;
+}
+
+template <int BN, int OUT>
+qwt_status launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
+                       bool cooperative, cudaStream_t st) {
+  using L = SmemLayout<BN>;
+  auto kern = qlinear_cwac_kernel<BN, OUT>;
+  // per device and cheap, so it is simply set on every launch
+  QWT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic));
+  if (cooperative) {
+    void* args[] = {(void*)&tmA, (void*)&tmB, (void*)&prm};
+    QWT_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, L::kDynamic, st));
+    count_launch();
+  } else {
+    kern<<<grid, kThreads, L::kDynamic, st>>>(tmA, tmB, prm);
+    QWT_LAUNCH_CHECK();
+  }
+  return QWT_OK;
+}
+
+template <int BN>
+qwt_status launch_bn(int out_mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
+                     cudaStream_t st) {
+  switch (out_mode) {
+    case QWT_OUT_INT8_PER_TOKEN:
+      return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN>(tmA, tmB, prm, grid, true, st);
+    case QWT_OUT_BF16:
+      return launch_inst<BN, QWT_OUT_BF16>(tmA, tmB, prm, grid, false, st);
+    case QWT_OUT_FP32:
+      return launch_inst<BN, QWT_OUT_FP32>(tmA, tmB, prm, grid, false, st);
+    case QWT_OUT_INT32_ACC:
+      return launch_inst<BN, QWT_OUT_INT32_ACC>(tmA, tmB, prm, grid, false, st);
+  }
+  return QWT_ERR_UNSUPPORTED;
+}
+
+}  // namespace
+
+qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
+                        QlinearPlan* plan) {
+  (void)K;
+  (void)wfmt;
+  QlinearPlan pl{};
+  pl.tiles_m = (M + kBM - 1) / kBM;
+  // 256-wide tiles keep the tensor pipe ahead of shared-memory bandwidth; 128-wide ones are used when
+  // the wider tile would leave many SMs without work.
+  const int sms = dev.sm_count > 0 ? dev.sm_count : 148;
+  const long t256 = (long)pl.tiles_m * ((N + 255) / 256);
+  const long t128 = (long)pl.tiles_m * ((N + 127) / 128);
+  auto waves_eff = [&](long tiles) {
+    const long waves = (tiles + sms - 1) / sms;
+    return (double)tiles / (double)(waves * sms);
+  };
+  pl.bn = (N > 128 && waves_eff(t256) + 0.10 >= waves_eff(t128)) ? 256 : 128;
+  const char* force = getenv("QWT_FORCE_BN");
+  if (force != nullptr) {
+    const int f = atoi(force);
+    if (f == 128 || f == 256) pl.bn = f;
+  }
+  pl.tiles_n = (N + pl.bn - 1) / pl.bn;
+  const long tiles = (long)pl.tiles_m * pl.tiles_n;
+  pl.grid = (int)(tiles < sms ? tiles : sms);
+  pl.smem_bytes = pl.bn == 256 ? SmemLayout<256>::kDynamic : SmemLayout<128>::kDynamic;
+  pl.fused_requant = (out_mode == QWT_OUT_INT8_PER_TOKEN) && (pl.tiles_n <= pl.grid);
+  size_t off = 0;
+  pl.ws_status_off = off;
+  off += 256;
+  pl.ws_rowmax_off = off;
+  off += ((size_t)M * 4 + 255) / 256 * 256;
+  pl.ws_counter_off = off;
+  off += ((size_t)pl.tiles_m * 4 + 255) / 256 * 256;
+  pl.ws_z_off = off;
+  if (out_mode == QWT_OUT_INT8_PER_TOKEN && !pl.fused_requant) off += (size_t)M * N * 4;
+  pl.ws_total = off;
+  *plan = pl;
+  return QWT_OK;
+}
+
+qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, int32_t wfmt, const float* fscale,
+                          const float* fbias, int32_t M, int32_t N, int32_t K, int32_t out_mode, void* Y,
+                          float* y_scale, void* workspace, const QlinearPlan& plan, cudaStream_t st) {
+  if (wfmt != QWT_W_INT8) return QWT_ERR_UNSUPPORTED;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  CUtensorMap tmA, tmB;
+  if (!make_byte_map(&tmA, X, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
+      !make_byte_map(&tmB, W, (uint64_t)N, (uint64_t)K, kBK, (uint32_t)plan.bn, CU_TENSOR_MAP_SWIZZLE_128B)) {
+    set_cuda_error((int)cudaErrorInvalidValue);
+    return QWT_ERR_CUDA;
+  }
+  // status word, row maxima and strip counters start at zero
+  QWT_CUDA_TRY(cudaMemsetAsync(ws, 0, plan.ws_z_off, st));
+
+  QlParams prm{};
+  prm.x_scale = x_scale;
+  prm.fscale = fscale;
+  prm.fbias = fbias;
+  prm.Y = Y;
+  prm.y_scale = y_scale;
+  prm.M = M;
+  prm.N = N;
+  prm.K = K;
+  prm.tiles_n = plan.tiles_n;
+  prm.num_tiles = plan.tiles_m * plan.tiles_n;
+  prm.num_kb = (K + kBK - 1) / kBK;
+  prm.status = reinterpret_cast<uint32_t*>(ws + plan.ws_status_off);
+  prm.rowmax = reinterpret_cast<uint32_t*>(ws + plan.ws_rowmax_off);
+  prm.counters = reinterpret_cast<uint32_t*>(ws + plan.ws_counter_off);
+  prm.counter_target = (uint32_t)plan.tiles_n * kNumEpilogueWarps;
+  prm.timeout_ns = timeout_ns_from_env();
+
+  int mode = out_mode;
+  if (out_mode == QWT_OUT_INT8_PER_TOKEN && !plan.fused_requant) {
+    // very wide layers (more column tiles than CTAs): z goes through FP32 scratch and a row quantizer
+    mode = QWT_OUT_FP32;
+    prm.Y = ws + plan.ws_z_off;
+  }
+  qwt_status s = plan.bn == 256 ? launch_bn<256>(mode, tmA, tmB, prm, plan.grid, st)
+                                : launch_bn<128>(mode, tmA, tmB, prm, plan.grid, st);
+  if (s != QWT_OK) return s;
+  if (mode != out_mode)
+    return launch_quantize_rows(reinterpret_cast<const float*>(ws + plan.ws_z_off), M, N, N, 127,
+                                static_cast<int8_t*>(Y), y_scale, st);
+  return QWT_OK;
+}
+
+}  // namespace qwt

@@ -1,0 +1,81 @@
+// Internal declarations shared by the translation units of libqwt2 (not part of the C ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "qwt2.h"
+
+namespace qwt {
+
+// thread-local record of the last CUDA failure and of the number of kernels launched
+void set_cuda_error(int err);
+void count_launch(int n = 1);
+
+#define QWT_CUDA_TRY(expr)                                   \
+  do {                                                       \
+    cudaError_t _e = (expr);                                 \
+    if (_e != cudaSuccess) {                                 \
+      ::qwt::set_cuda_error((int)_e);                        \
+      return QWT_ERR_CUDA;                                   \
+    }                                                        \
+  } while (0)
+
+// after a kernel launch
+#define QWT_LAUNCH_CHECK()                                   \
+  do {                                                       \
+    cudaError_t _e = cudaGetLastError();                     \
+    if (_e != cudaSuccess) {                                 \
+      ::qwt::set_cuda_error((int)_e);                        \
+      return QWT_ERR_CUDA;                                   \
+    }                                                        \
+    ::qwt::count_launch();                                   \
+  } while (0)
+
+struct DeviceInfo {
+  int device;
+  int sm_count;
+  int cc_major;
+  int cc_minor;
+  int max_smem_optin;
+};
+// Properties of the current device (cached per device). Returns QWT_ERR_ARCH when it is not CC 10.x.
+qwt_status current_device(DeviceInfo* out);
+
+inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
+
+// ---- calibration (cwac_kernels.cu)
+struct CwacPlan {
+  int slabs;        // column slabs of 128 channels
+  int chunks;       // row chunks
+  int64_t chunk_rows;
+  size_t partial_bytes;  // double[chunks][4][channels_padded]
+  int cpad;         // channels rounded up to 128
+};
+CwacPlan cwac_plan(int64_t rows, int32_t channels, int sm_count);
+qwt_status launch_cwac_stats(const float* fp_out, const float* q_out, int64_t rows, int32_t channels, int64_t ld,
+                             double* stats, void* workspace, const CwacPlan& plan, cudaStream_t st);
+qwt_status launch_cwac_solve(const double* stats, int32_t channels, float* a, float* b, int32_t* n_degenerate,
+                             cudaStream_t st);
+qwt_status launch_cwac_fold(const float* w_scale, const float* bias, const float* a, const float* b, int32_t n,
+                            float* fscale, float* fbias, cudaStream_t st);
+qwt_status launch_quantize_rows(const float* X, int64_t rows, int32_t cols, int64_t ld, int32_t qmax, int8_t* Xq,
+                                float* scale, cudaStream_t st);
+qwt_status launch_pack_int4(const int8_t* codes, int64_t rows, int32_t cols, uint8_t* packed, cudaStream_t st);
+
+// ---- forward (qlinear_tcgen05.cu)
+struct QlinearPlan {
+  int bn;            // CTA tile width (128 or 256)
+  int tiles_m, tiles_n;
+  int grid;
+  size_t smem_bytes;
+  bool fused_requant;    // cross-CTA row-max protocol inside the GEMM kernel
+  size_t ws_status_off, ws_rowmax_off, ws_counter_off, ws_z_off, ws_total;
+};
+qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
+                        QlinearPlan* plan);
+qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, int32_t wfmt, const float* fscale,
+                          const float* fbias, int32_t M, int32_t N, int32_t K, int32_t out_mode, void* Y,
+                          float* y_scale, void* workspace, const QlinearPlan& plan, cudaStream_t st);
+
+}  // namespace qwt

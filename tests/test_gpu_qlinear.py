@@ -1,0 +1,168 @@
+"""GPU parity: the CWAC-fused quantized linear layer against the CPU oracle (through the C ABI)."""
+import numpy as np
+import pytest
+
+from oracle import qwt_oracle as O
+from paper_2505_20932_b200 import workload as WL
+from tolerances import assert_codes_close, assert_fp32_close
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def H():
+    import gpu_harness
+    return gpu_harness
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2505_20932_b200 import binding
+    return binding
+
+
+def random_layer(M, N, K, seed, planted=True):
+    rng = np.random.default_rng(seed)
+    Xq = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    Wq = rng.integers(-127, 128, (N, K)).astype(np.int8)
+    xs = rng.uniform(0.01, 0.05, M).astype(np.float32)
+    ws = rng.uniform(1e-4, 3e-4, N).astype(np.float32)
+    bias = (0.01 * rng.standard_normal(N)).astype(np.float32)
+    a = (1 + 0.05 * rng.standard_normal(N)).astype(np.float32)
+    b = (0.02 * rng.standard_normal(N)).astype(np.float32)
+    fs64, fb64 = O.cwac_fold(ws, bias, a, b)
+    return Xq, Wq, xs, fs64.astype(np.float32), fb64.astype(np.float32)
+
+
+SHAPES = [
+    (128, 128, 128),     # exactly one tile, one k-block
+    (128, 256, 256),
+    (1, 16, 16),         # smallest legal problem
+    (130, 272, 400),     # ragged in M, N and K (K tail of 16 bytes)
+    (788, 1536, 384),    # config 1
+    (300, 528, 1040),    # several k-blocks with a tail, N tail of 16
+    (257, 4096, 512),    # many column tiles per strip
+    (2000, 384, 1536),   # more tiles than SMs: second round of the persistent loop
+]
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+def test_int32_accumulators_bit_exact(H, B, M, N, K):
+    Xq, Wq, *_ = random_layer(M, N, K, seed=M + N + K)
+    acc, _ = H.gpu_forward(Xq, None, Wq, None, None, B.QWT_OUT_INT32_ACC)
+    assert np.array_equal(acc.astype(np.int64), O.int_matmul(Xq, Wq))
+
+
+def test_int32_extreme_codes(H, B):
+    M, N, K = 130, 144, 4096
+    Xq = np.full((M, K), 127, np.int8)
+    Xq[::2] = -127
+    Wq = np.full((N, K), -127, np.int8)
+    Wq[::3] = 127
+    acc, _ = H.gpu_forward(Xq, None, Wq, None, None, B.QWT_OUT_INT32_ACC)
+    assert np.array_equal(acc.astype(np.int64), O.int_matmul(Xq, Wq))
+    assert abs(int(acc[0, 0])) == 127 * 127 * K
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+def test_fp32_output_within_tolerance(H, B, M, N, K):
+    Xq, Wq, xs, fs, fb = random_layer(M, N, K, seed=M + N + K + 1)
+    z, _ = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_FP32)
+    z_ref = O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb)
+    assert_fp32_close(z, z_ref)
+
+
+@pytest.mark.parametrize("M,N,K", SHAPES)
+def test_int8_per_token_output(H, B, M, N, K):
+    Xq, Wq, xs, fs, fb = random_layer(M, N, K, seed=M + N + K + 2)
+    codes, ys = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_INT8_PER_TOKEN)
+    z_ref = O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb)
+    c_ref, ys_ref = O.requant_per_token(z_ref)
+    assert np.allclose(ys, ys_ref, rtol=1e-5, atol=0)
+    assert_codes_close(codes, c_ref)
+    # the codes reproduce z to half a step of the row's own scale
+    err = np.abs(z_ref - ys[:, None].astype(np.float64) * codes)
+    assert np.all(err <= 0.5 * ys[:, None] * (1 + 1e-4) + 1e-6)
+    assert codes.min() >= -127
+
+
+@pytest.mark.parametrize("M,N,K", [(130, 272, 400), (788, 1536, 384), (257, 4096, 512)])
+def test_bf16_output(H, B, M, N, K):
+    Xq, Wq, xs, fs, fb = random_layer(M, N, K, seed=M + N + K + 3)
+    bits, _ = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_BF16)
+    z_ref = O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb)
+    ref_bits = O.to_bf16_bits(z_ref)
+    d = np.abs(bits.astype(np.int32) - ref_bits.astype(np.int32))
+    assert d.max() <= 1                                   # at most one bfloat16 ulp ...
+    assert np.count_nonzero(d) <= max(1, int(1e-4 * d.size))     # ... on at most 0.01 % of the elements
+
+
+def test_zero_rows_and_zero_scale(H, B):
+    M, N, K = 140, 160, 128
+    Xq, Wq, xs, fs, fb = random_layer(M, N, K, seed=77)
+    Xq[5] = 0
+    xs[9] = 0.0
+    fb[:] = 0.0
+    codes, ys = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_INT8_PER_TOKEN)
+    assert ys[5] == 0 and ys[9] == 0 and not codes[5].any() and not codes[9].any()
+    c_ref, ys_ref = O.requant_per_token(O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb))
+    assert_codes_close(codes, c_ref)
+
+
+def test_config1_layer_end_to_end(H, B):
+    """Config 1: quantize -> calibrate CWAC on 32 images -> fold -> fused forward, every stage against the oracle."""
+    spec = WL.config_layers(1)[0]
+    d = WL.host_layer_inputs(spec, seed=0)
+    Xq, xs = O.quantize_rows_sym(d["X"], 127)
+    Wq, ws = O.quantize_rows_sym(d["W"], 127)
+    gXq, gxs = H.gpu_quantize_rows(d["X"], 127)
+    gWq, gws = H.gpu_quantize_rows(d["W"], 127)
+    assert np.array_equal(gXq, Xq) and np.array_equal(gxs, xs) and np.array_equal(gWq, Wq) and np.array_equal(gws, ws)
+
+    # calibration pair on the 6304 calibration tokens (Section 3.3): Y_full and Y_quant of the same X_in
+    Xcq, xcs = O.quantize_rows_sym(d["Xc"], 127)
+    q_out = O.dequant(O.int_matmul(Xcq, Wq), xcs, ws, d["bias"])
+    fp_out = O.linear_fp(d["Xc"], d["W"], d["bias"])
+    gq, _ = H.gpu_forward(Xcq, xcs, Wq, ws, d["bias"], B.QWT_OUT_FP32)     # no CWAC yet: fscale = S_W, fbias = bias
+    assert_fp32_close(gq, q_out, "q_out")
+    fp32, q32 = fp_out.astype(np.float32), q_out.astype(np.float32)
+    a_ref, b_ref, _ = O.cwac_fit(fp32, q32)
+    ga, gb, nd = H.gpu_calibrate(fp32, q32)
+    from tolerances import assert_ab_close
+    assert nd == 0
+    assert_ab_close(ga, gb, a_ref, b_ref, np.maximum(np.abs(fp_out.mean(0)), fp_out.std(0)))
+    assert 0.99 < a_ref.mean() < 1.01                     # W8A8: the compensation is close to identity
+
+    a32, b32 = a_ref.astype(np.float32), b_ref.astype(np.float32)
+    fs_ref, fb_ref = O.cwac_fold(ws, d["bias"], a32, b32)
+    gfs, gfb = H.gpu_fold(ws, d["bias"], a32, b32)
+    assert np.allclose(gfs, fs_ref, rtol=1e-6) and np.allclose(gfb, fb_ref, rtol=1e-6, atol=1e-9)
+
+    # forward with the folded parameters == unfolded reference (dequant, then CWAC)
+    z_unfolded = O.qlinear_cwac_reference(Xq, xs, Wq, ws, d["bias"], a32, b32)
+    fs32, fb32 = fs_ref.astype(np.float32), fb_ref.astype(np.float32)
+    gz, _ = H.gpu_forward(Xq, xs, Wq, fs32, fb32, B.QWT_OUT_FP32)
+    assert_fp32_close(gz, z_unfolded, "z (folded GPU vs unfolded oracle)")
+    codes, ys = H.gpu_forward(Xq, xs, Wq, fs32, fb32, B.QWT_OUT_INT8_PER_TOKEN)
+    c_ref, ys_ref = O.requant_per_token(O.forward_folded(O.int_matmul(Xq, Wq), xs, fs32, fb32))
+    assert np.allclose(ys, ys_ref, rtol=1e-5)
+    assert_codes_close(codes, c_ref)
+    # CWAC lowers the error against the full-precision layer (what Eq. 3 minimises on the calibration set)
+    y_fp = O.linear_fp(d["X"], d["W"], d["bias"])
+    y_q = O.dequant(O.int_matmul(Xq, Wq), xs, ws, d["bias"])
+    assert np.sum((gz - y_fp) ** 2) <= np.sum((y_q - y_fp) ** 2) * 1.001
+
+
+def test_forward_from_host_memory(H, B):
+    import torch
+    M, N, K = 300, 528, 1040
+    Xq, Wq, xs, fs, fb = random_layer(M, N, K, seed=5)
+    dW, dfs, dfb = H.dev(Wq), H.dev(fs), H.dev(fb)
+    Y = np.zeros((M, N), np.int8)
+    ys = np.zeros(M, np.float32)
+    sb = B.qwt_qlinear_host_staging_bytes(M, N, K, B.QWT_W_INT8, B.QWT_OUT_INT8_PER_TOKEN)
+    st = H.empty_bytes(sb)
+    B.qwt_qlinear_cwac_forward_host(Xq, xs, dW, B.QWT_W_INT8, dfs, dfb, M, N, K, B.QWT_OUT_INT8_PER_TOKEN, Y, ys, st, sb)
+    c_ref, ys_ref = O.requant_per_token(O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb))
+    assert np.allclose(ys, ys_ref, rtol=1e-5)
+    assert_codes_close(Y, c_ref)

@@ -1,0 +1,35 @@
+"""Tolerances of the parity tests (stated by the task's target; see the design doc for the arithmetic)."""
+import numpy as np
+
+FP32_REL = 1e-5      # dequantized + compensated outputs: |d| <= 1e-5 |ref| + 1e-6
+FP32_ABS = 1e-6
+CODE_MAX_LSB = 1     # requantized INT8 codes: at most 1 LSB ...
+CODE_MAX_FRAC = 1e-4  # ... on at most 0.01 % of the elements
+AB_REL = 1e-5        # CWAC a, b
+
+
+def assert_fp32_close(got, ref, what="z"):
+    ref = np.asarray(ref, dtype=np.float64)
+    d = np.abs(np.asarray(got, dtype=np.float64) - ref)
+    lim = FP32_REL * np.abs(ref) + FP32_ABS
+    bad = d > lim
+    assert not bad.any(), f"{what}: {bad.sum()} of {bad.size} outside tolerance, worst excess {np.max(d - lim):.3e}"
+
+
+def assert_codes_close(got, ref, what="codes"):
+    d = np.abs(got.astype(np.int32) - ref.astype(np.int32))
+    assert d.max(initial=0) <= CODE_MAX_LSB, f"{what}: a code differs by {d.max()} LSB"
+    frac = np.count_nonzero(d) / max(d.size, 1)
+    # tiny outputs: allow a single element
+    assert frac <= CODE_MAX_FRAC or np.count_nonzero(d) <= 1, f"{what}: {frac:.3e} of the codes differ"
+
+
+def assert_ab_close(a, b, a_ref, b_ref, scale_b):
+    """a: plain relative.  b: relative with an absolute floor of 1e-6 x the channel's natural scale."""
+    a_ref = np.asarray(a_ref, dtype=np.float64)
+    b_ref = np.asarray(b_ref, dtype=np.float64)
+    da = np.abs(a - a_ref)
+    assert np.all(da <= AB_REL * np.abs(a_ref) + 1e-7), f"a: worst rel {np.max(da / np.maximum(np.abs(a_ref), 1e-30)):.3e}"
+    db = np.abs(b - b_ref)
+    lim = AB_REL * np.abs(b_ref) + 1e-6 * np.asarray(scale_b) + 1e-7
+    assert np.all(db <= lim), f"b: worst excess {np.max(db - lim):.3e}"
