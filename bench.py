@@ -1,0 +1,520 @@
+#!/usr/bin/env python
+"""Benchmark of the CWAC hot path on B200.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--workload cfg2|cfg1|cfg3|cfg4|cfg5] [--impl ours|reference]
+
+A *step* is one pass of the whole hot path over one batch of synthetic input:
+  phase A  for every layer of the workload: CWAC statistics + closed-form solve on the layer's calibration
+           pair (qwt_cwac_calibrate) and the fold (qwt_cwac_fold);
+  phase B  for every layer: the CWAC-fused quantized linear forward (qwt_qlinear_cwac_forward).
+`value` is the GEMM throughput of phase B (2*M*N*K operations per layer / phase-B device time, TOPS);
+the calibration half of the metric (8 bytes per row and channel / phase-A device time, GB/s) is in
+`calibration`.  `ms_per_step` covers both phases.  All inputs are resident in HBM before the timed
+region; `e2e` repeats phase B through the host-buffer entry point with the copies inside the timing.
+Prints ONE JSON line on rank 0.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+METRIC = "CWAC-fused W8A8 GEMM TOPS & % INT8 peak; calibration GB/s & % HBM peak"
+UNIT = "TOPS"
+
+# Fallback peaks of this B200 pool when MEASURED_PEAKS.json is absent.
+FALLBACK_HBM_GBS = 6650.0
+FALLBACK_BF16_TFLOPS = 1590.0
+INT8_OVER_BF16 = 2.0      # nominal dense ratio (4.5 POPS int8 : 2.25 PFLOPS bf16)
+
+# DRAM bytes per algorithmic byte of cwac_stats_kernel, from the ncu capture summarised in
+# profiles/cwac_stats_kernel_cfg5_small.md (None until a capture exists).
+STATS_TRAFFIC_RATIO = None
+# same for the forward kernel on a LLaMA-shaped layer, profiles/qlinear_cwac_kernel_*.md
+QLINEAR_TRAFFIC_RATIO = None
+
+
+def load_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])), "source": "measured"}
+    return {"hbm_gbs": FALLBACK_HBM_GBS, "bf16_tflops": FALLBACK_BF16_TFLOPS,
+            "bf16_tflops_sustained": 1400.0, "source": "fallback"}
+
+
+# --------------------------------------------------------------------------------------------- clocks
+
+class ClockSampler(threading.Thread):
+    """Samples SM clock and throttle reasons of one GPU through NVML while the timed region runs."""
+
+    def __init__(self, index: int, period_s: float = 0.02):
+        super().__init__(daemon=True)
+        self.index, self.period = index, period_s
+        self.samples, self.reasons, self.max_mhz = [], set(), None
+        self._stop_evt = threading.Event()
+        self.ok = False
+        try:
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            self.h = pynvml.nvmlDeviceGetHandleByIndex(index)
+            self.max_mhz = pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM)
+            self.ok = True
+        except Exception:
+            self.ok = False
+
+    def run(self):
+        if not self.ok:
+            return
+        nv = self.nv
+        names = {
+            getattr(nv, "nvmlClocksEventReasonHwSlowdown", 0x8): "hw_slowdown",
+            getattr(nv, "nvmlClocksEventReasonHwThermalSlowdown", 0x40): "hw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwThermalSlowdown", 0x20): "sw_thermal_slowdown",
+            getattr(nv, "nvmlClocksEventReasonSwPowerCap", 0x4): "sw_power_cap",
+            getattr(nv, "nvmlClocksEventReasonHwPowerBrakeSlowdown", 0x80): "hw_power_brake_slowdown",
+        }
+        while not self._stop_evt.is_set():
+            try:
+                self.samples.append(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM))
+                try:
+                    mask = nv.nvmlDeviceGetCurrentClocksEventReasons(self.h)
+                except Exception:
+                    mask = nv.nvmlDeviceGetCurrentClocksThrottleReasons(self.h)
+                for bit, name in names.items():
+                    if mask & bit:
+                        self.reasons.add(name)
+            except Exception:
+                pass
+            self._stop_evt.wait(self.period)
+
+    def stop(self):
+        self._stop_evt.set()
+        if self.is_alive():
+            self.join(timeout=2)
+        return {"sm_mhz": (statistics.median(self.samples) if self.samples else None),
+                "sm_max_mhz": self.max_mhz, "reasons": sorted(self.reasons), "samples": len(self.samples)}
+
+
+# --------------------------------------------------------------------------------------------- workload on the device
+
+class Layer:
+    """Device-resident state of one quantized linear layer (inputs, parameters, outputs, scratch)."""
+    pass
+
+
+def _quant_rows(B, torch, X, qmax):
+    r, c = X.shape
+    q = torch.empty((r, c), dtype=torch.int8, device=X.device)
+    s = torch.empty(r, dtype=torch.float32, device=X.device)
+    B.qwt_quantize_rows_i8(X, r, c, c, qmax, q, s)
+    return q, s
+
+
+def build_layer(B, torch, WL, spec, seed, device, calib_rows=None):
+    L = Layer()
+    L.spec = spec
+    M, K, N = spec.M, spec.K, spec.N
+    R = spec.calib_rows if calib_rows is None else calib_rows
+    L.R = R
+    L.wfmt = B.QWT_W_INT8 if spec.w_bits == 8 else B.QWT_W_INT4_PACKED
+    L.out_mode = B.QWT_OUT_INT8_PER_TOKEN if spec.out == "int8" else B.QWT_OUT_BF16
+    X = WL.device_activations(spec.act, M, K, seed, spec.name + "|infer", device)
+    L.Xq, L.xs = _quant_rows(B, torch, X, 127)
+    del X
+    W = WL.device_weights(N, K, seed, spec.name, device=device)
+    qmax = 127 if spec.w_bits == 8 else 7
+    Wq, L.ws = _quant_rows(B, torch, W, qmax)
+    if spec.w_bits == 4:
+        L.W = torch.empty((N, K // 2), dtype=torch.uint8, device=device)
+        B.qwt_pack_int4(Wq, N, K, L.W)
+    else:
+        L.W = Wq
+    g = torch.Generator(device=device)
+    g.manual_seed(seed * 7919 + 13)
+    L.bias = torch.randn(N, generator=g, device=device) * 0.01
+    # calibration pair (Section 3.3): Y_full and Y_quant of the same calibration tokens
+    Xc = WL.device_activations(spec.act, R, K, seed, spec.name + "|calib", device)
+    Xcq, xcs = _quant_rows(B, torch, Xc, 127)
+    L.q_out = torch.empty((R, N), dtype=torch.float32, device=device)
+    wsb = B.qwt_qlinear_workspace_bytes(R, N, K, L.wfmt, B.QWT_OUT_FP32)
+    ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device=device)
+    B.qwt_qlinear_cwac_forward(Xcq, xcs, L.W, L.wfmt, L.ws, L.bias, R, N, K, B.QWT_OUT_FP32, L.q_out, None, ws, wsb)
+    B.qwt_qlinear_check_status(ws)
+    if spec.planted:
+        a_star, b_star = WL.host_planted_cwac(N, seed, spec.name)
+        a_s, b_s = torch.from_numpy(a_star).to(device), torch.from_numpy(b_star).to(device)
+        L.fp_out = L.q_out * a_s[None, :] + b_s[None, :]
+        sd = L.q_out[: min(R, 4096)].std(dim=0)
+        L.fp_out += torch.randn((R, N), generator=g, device=device) * (0.01 * sd)[None, :]
+    else:
+        L.fp_out = torch.addmm(L.bias, Xc, W.t())
+    del Xc, Xcq, xcs, W
+    L.a = torch.empty(N, dtype=torch.float32, device=device)
+    L.b = torch.empty(N, dtype=torch.float32, device=device)
+    L.fs = torch.empty(N, dtype=torch.float32, device=device)
+    L.fb = torch.empty(N, dtype=torch.float32, device=device)
+    L.cws_bytes = B.qwt_cwac_workspace_bytes(R, N)
+    L.cws = torch.empty(max(L.cws_bytes, 256), dtype=torch.uint8, device=device)
+    ydt = torch.int8 if spec.out == "int8" else torch.bfloat16
+    L.Y = torch.empty((M, N), dtype=ydt, device=device)
+    L.ys = torch.empty(M, dtype=torch.float32, device=device) if spec.out == "int8" else None
+    L.fws_bytes = B.qwt_qlinear_workspace_bytes(M, N, K, L.wfmt, L.out_mode)
+    L.fws = torch.empty(max(L.fws_bytes, 256), dtype=torch.uint8, device=device)
+    L.calib_bytes = 8 * R * N
+    out_b = 1 if spec.out == "int8" else 2
+    wb = K if spec.w_bits == 8 else K // 2
+    L.fwd_bytes = M * K + N * wb + M * N * out_b + 4 * M + 8 * N + (4 * M if spec.out == "int8" else 0)
+    return L
+
+
+def phase_a(B, layers, stream):
+    for L in layers:
+        s = L.spec
+        B.qwt_cwac_calibrate(L.fp_out, L.q_out, L.R, s.N, s.N, L.a, L.b, None, L.cws, L.cws_bytes, stream)
+        B.qwt_cwac_fold(L.ws, L.bias, L.a, L.b, s.N, L.fs, L.fb, stream)
+
+
+def phase_b(B, layers, stream):
+    for L in layers:
+        s = L.spec
+        B.qwt_qlinear_cwac_forward(L.Xq, L.xs, L.W, L.wfmt, L.fs, L.fb, s.M, s.N, s.K, L.out_mode, L.Y, L.ys,
+                                   L.fws, L.fws_bytes, stream)
+
+
+def workload_layers(WL, name):
+    if name == "cfg1":
+        return WL.config_layers(1), "config 1: single W8A8 layer 788x384->1536, CWAC fit on 32 images"
+    if name == "cfg2":
+        return WL.config_layers(2), "config 2: DeiT-S W8A8 stack, 12 blocks x (qkv, proj, fc1, fc2), batch 64x197 tokens, CWAC fit per layer on 512 images"
+    if name == "cfg3":
+        return WL.config_layers(3), "config 3: ViT-B W4A8 stack, 12 blocks, batch 128x197 tokens, BF16 out, CWAC fit on 1024 images"
+    if name == "cfg4":
+        return WL.config_layers(4), "config 4: LLaMA-7B shaped W8A8 layers at M=2048 and 8192, CWAC planted and refit from 128x2048 tokens"
+    raise ValueError(name)
+
+
+# --------------------------------------------------------------------------------------------- CPU oracle timing
+
+def oracle_block_time(layers_host, calib_rows_cap):
+    """Times the oracle (as it stands) on host copies of a few layers.  Returns (fwd_ops, fwd_s, cal_bytes, cal_s)."""
+    from oracle import qwt_oracle as O
+    fwd_ops = cal_bytes = 0
+    fwd_s = cal_s = 0.0
+    for h in layers_host:
+        t0 = time.perf_counter()
+        a, b, _ = O.cwac_fit(h["fp_out"], h["q_out"])
+        fs, fb = O.cwac_fold(h["ws"], h["bias"], a, b)
+        t1 = time.perf_counter()
+        acc = O.int_matmul(h["Xq"], h["Wq"])
+        z = O.forward_folded(acc, h["xs"], fs, fb)
+        if h["out"] == "int8":
+            O.requant_per_token(z)
+        else:
+            O.to_bf16_bits(z)
+        t2 = time.perf_counter()
+        cal_s += t1 - t0
+        fwd_s += t2 - t1
+        cal_bytes += 8 * h["fp_out"].shape[0] * h["fp_out"].shape[1]
+        fwd_ops += 2 * h["Xq"].shape[0] * h["Wq"].shape[0] * h["Xq"].shape[1]
+    return fwd_ops, fwd_s, cal_bytes, cal_s
+
+
+def host_copy_of_layer(L, rows_cap, calib_cap, O=None):
+    from oracle import qwt_oracle as Or
+    s = L.spec
+    m = min(s.M, rows_cap)
+    r = min(L.R, calib_cap)
+    W = L.W.cpu().numpy()
+    if s.w_bits == 4:
+        W = Or.unpack_int4(W)
+    return {"Xq": L.Xq[:m].cpu().numpy(), "xs": L.xs[:m].cpu().numpy(), "Wq": W, "ws": L.ws.cpu().numpy(),
+            "bias": L.bias.cpu().numpy(), "fp_out": L.fp_out[:r].cpu().numpy(), "q_out": L.q_out[:r].cpu().numpy(),
+            "out": s.out}
+
+
+def blas_threads():
+    try:
+        from threadpoolctl import threadpool_info
+        n = [p.get("num_threads", 1) for p in threadpool_info() if p.get("user_api") == "blas"]
+        return max(n) if n else 1
+    except Exception:
+        return os.cpu_count() or 1
+
+
+# --------------------------------------------------------------------------------------------- reference arm
+
+def run_reference(args):
+    """Times the CPU oracle on the host cores: each step = a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    from oracle import qwt_oracle as O
+    from paper_2505_20932_b200 import workload as WL
+    specs, desc = workload_layers(WL, args.workload)
+    specs = specs[:4]
+    rows_cap, calib_cap = 1024, 8192
+    hosts = []
+    for sp in specs:
+        m, r = min(sp.M, rows_cap), min(sp.calib_rows, calib_cap)
+        d = WL.host_layer_inputs(sp, seed=args.seed, rows=m, calib_rows=r)
+        qmax = 127 if sp.w_bits == 8 else 7
+        Xq, xs = O.quantize_rows_sym(d["X"], 127)
+        Wq, ws = O.quantize_rows_sym(d["W"], qmax)
+        Xcq, xcs = O.quantize_rows_sym(d["Xc"], 127)
+        q_out = O.dequant(O.int_matmul(Xcq, Wq), xcs, ws, d["bias"]).astype(np.float32)
+        if sp.planted:
+            fp_out = (q_out * d["a_star"] + d["b_star"]).astype(np.float32)
+        else:
+            fp_out = O.linear_fp(d["Xc"], d["W"], d["bias"]).astype(np.float32)
+        hosts.append({"Xq": Xq, "xs": xs, "Wq": Wq, "ws": ws, "bias": d["bias"], "fp_out": fp_out, "q_out": q_out,
+                      "out": sp.out})
+    for _ in range(args.warmup):
+        oracle_block_time(hosts, calib_cap)
+    t_f = t_c = 0.0
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        ops, fs_, cb, cs_ = oracle_block_time(hosts, calib_cap)
+        t_f += fs_
+        t_c += cs_
+    total = time.perf_counter() - t0
+    value = ops * args.steps / t_f / 1e12
+    sample = (f"first {len(specs)} layers of the workload, first {rows_cap} tokens (forward) and first {calib_cap} "
+              f"calibration rows (fit) of each, per step")
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": total / args.steps * 1e3, "higher_is_better": True, "scaling": "weak",
+        "vs_baseline": None, "dtype": "int8", "data": "synthetic",
+        "config": {"workload": desc, "l2": "n/a (CPU)"},
+        "calibration": {"value": cb * args.steps / t_c / 1e9, "unit": "GB/s"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": blas_threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# --------------------------------------------------------------------------------------------- our arm
+
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2505_20932_b200 import binding as B     # raises if libqwt2.so is missing: no fallback
+    from paper_2505_20932_b200 import workload as WL
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device(f"cuda:{local}"))
+    torch.cuda.set_device(local)
+    device = f"cuda:{local}"
+    torch.backends.cuda.matmul.allow_tf32 = False
+    peaks = load_peaks()
+
+    specs, desc = workload_layers(WL, args.workload)
+    specs = specs[args.first_layer:]
+    if args.layers:
+        specs = specs[: args.layers]
+    # every rank owns a full copy of the workload with its own seed (row shards of a larger batch): weak scaling
+    if args.out:
+        import dataclasses
+        specs = [dataclasses.replace(sp, out=args.out) for sp in specs]
+    layers = [build_layer(B, torch, WL, sp, args.seed + 1000 * rank + i, device,
+                          calib_rows=(min(sp.calib_rows, args.calib_rows) if args.calib_rows else None))
+              for i, sp in enumerate(specs)]
+    torch.cuda.synchronize()
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(args.warmup):
+        phase_a(B, layers, stream)
+        phase_b(B, layers, stream)
+    for L in layers:
+        if L.fws_bytes:
+            B.qwt_qlinear_check_status(L.fws)
+    barrier()
+
+    sampler = ClockSampler(local)
+    sampler.start()
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    B.qwt_launch_count_reset()
+    for k in range(args.steps):
+        ev[k][0].record(stream)
+        phase_a(B, layers, stream)
+        ev[k][1].record(stream)
+        phase_b(B, layers, stream)
+        ev[k][2].record(stream)
+    barrier()
+    launches = B.qwt_launch_count()
+    clocks = sampler.stop()
+    t_a = sum(e[0].elapsed_time(e[1]) for e in ev) * 1e-3
+    t_b = sum(e[1].elapsed_time(e[2]) for e in ev) * 1e-3
+    t_all = ev[0][0].elapsed_time(ev[-1][2]) * 1e-3
+    for L in layers:
+        B.qwt_qlinear_check_status(L.fws)
+
+    times = torch.tensor([t_a, t_b, t_all], dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(times, op=dist.ReduceOp.MAX)
+    t_a, t_b, t_all = [float(x) for x in times.cpu()]
+
+    fwd_ops = sum(L.spec.ops for L in layers)
+    cal_bytes = sum(L.calib_bytes for L in layers)
+    fwd_bytes = sum(L.fwd_bytes for L in layers)
+    tops = world * fwd_ops * args.steps / t_b / 1e12
+    cal_gbs = world * cal_bytes * args.steps / t_a / 1e9
+
+    # ---- e2e: phase B through the host-buffer entry point (pinned host activations in, host outputs back)
+    e2e = None
+    if not args.no_e2e:
+        host = []
+        for L in layers:
+            s = L.spec
+            hx = torch.empty((s.M, s.K), dtype=torch.int8).pin_memory()
+            hx.copy_(L.Xq)
+            hxs = L.xs.cpu().pin_memory()
+            hy = torch.empty(L.Y.shape, dtype=L.Y.dtype).pin_memory()
+            hys = torch.empty(s.M, dtype=torch.float32).pin_memory() if L.ys is not None else None
+            sb = B.qwt_qlinear_host_staging_bytes(s.M, s.N, s.K, L.wfmt, L.out_mode)
+            host.append((hx, hxs, hy, hys, sb))
+        sb_max = max(h[4] for h in host)
+        staging = torch.empty(sb_max, dtype=torch.uint8, device=device)
+
+        def e2e_pass():
+            for L, (hx, hxs, hy, hys, sb) in zip(layers, host):
+                s = L.spec
+                B.qwt_qlinear_cwac_forward_host(hx.data_ptr(), hxs.data_ptr(), L.W, L.wfmt, L.fs, L.fb, s.M, s.N, s.K,
+                                                L.out_mode, hy.data_ptr(), None if hys is None else hys.data_ptr(),
+                                                staging, sb_max, stream)
+        e2e_pass()
+        barrier()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        n_e2e = max(1, min(args.steps, 5))
+        e0.record(stream)
+        for _ in range(n_e2e):
+            e2e_pass()
+        e1.record(stream)
+        barrier()
+        t_e = torch.tensor([e0.elapsed_time(e1) * 1e-3], dtype=torch.float64, device=device)
+        if world > 1:
+            dist.all_reduce(t_e, op=dist.ReduceOp.MAX)
+        h2d = sum(h[0].numel() + h[1].numel() * 4 for h in host)
+        d2h = sum(h[2].numel() * h[2].element_size() + (h[3].numel() * 4 if h[3] is not None else 0) for h in host)
+        e2e = {"value": world * fwd_ops * n_e2e / float(t_e.item()) / 1e12, "unit": UNIT,
+               "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h, "steps": n_e2e,
+               "what": "phase B through qwt_qlinear_cwac_forward_host: pinned host X/x_scale in, host Y/y_scale out, per layer"}
+        del staging, host
+
+    # ---- rooflines
+    int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
+    int8_peak_sus = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
+    n_cal_launch = len(layers) * args.steps
+    cal_ach = cal_bytes * args.steps / t_a / 1e9           # per GPU
+    roof_cal = {"kernel": "cwac_stats_kernel", "bound": "hbm", "achieved": cal_ach, "peak": peaks["hbm_gbs"],
+                "unit": "GB/s", "frac": cal_ach / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
+                "traffic": (None if STATS_TRAFFIC_RATIO is None else STATS_TRAFFIC_RATIO * cal_bytes / len(layers)),
+                "algorithmic_bytes_per_launch": cal_bytes / len(layers), "launches": n_cal_launch,
+                "avg_launch_ms": t_a / n_cal_launch * 1e3,
+                "note": "duration = phase A (stats + reduce/solve + fold kernels of every layer) / launches"}
+    fwd_tops_gpu = fwd_ops * args.steps / t_b / 1e12
+    t_min_compute = fwd_ops / (int8_peak * 1e12)
+    t_min_hbm = fwd_bytes / (peaks["hbm_gbs"] * 1e9)
+    fwd_bound = "tensor" if t_min_compute >= t_min_hbm else "hbm"
+    if fwd_bound == "tensor":
+        roof_fwd = {"kernel": "qlinear_cwac_kernel", "bound": "tensor", "achieved": fwd_tops_gpu, "peak": int8_peak,
+                    "unit": "TOP/s", "frac": fwd_tops_gpu / int8_peak,
+                    "peak_source": f"2 x bf16 burst, of {peaks['source']}", "frac_of_sustained": fwd_tops_gpu / int8_peak_sus}
+    else:
+        ach = fwd_bytes * args.steps / t_b / 1e9
+        roof_fwd = {"kernel": "qlinear_cwac_kernel", "bound": "hbm", "achieved": ach, "peak": peaks["hbm_gbs"],
+                    "unit": "GB/s", "frac": ach / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
+                    "tensor_frac": fwd_tops_gpu / int8_peak}
+    roof_fwd.update({"traffic": None if QLINEAR_TRAFFIC_RATIO is None else QLINEAR_TRAFFIC_RATIO * fwd_bytes / len(layers),
+                     "algorithmic_bytes_per_launch": fwd_bytes / len(layers), "launches": len(layers) * args.steps,
+                     "avg_launch_ms": t_b / (len(layers) * args.steps) * 1e3})
+    dominant = roof_cal if t_a >= t_b else roof_fwd
+
+    line = None
+    if rank == 0:
+        cpu = None
+        if world == 1 and not args.no_cpu:
+            rows_cap, calib_cap = args.cpu_rows, args.cpu_calib_rows
+            hl = [host_copy_of_layer(L, rows_cap, calib_cap) for L in layers[:4]]
+            ops, fs_, cb, cs_ = oracle_block_time(hl, calib_cap)
+            cpu = {"value": ops / fs_ / 1e12, "unit": UNIT, "cores": blas_threads(), "kind": "oracle",
+                   "sample": (f"first {len(hl)} layers, first {rows_cap} tokens (forward: integer product, dequant+CWAC, "
+                              f"requant) and first {calib_cap} calibration rows (fit) of each; {fs_ + cs_:.1f} s of CPU work; "
+                              "BLAS matmul threaded, elementwise numpy single-threaded"),
+                   "calibration_gbs": cb / cs_ / 1e9, "host_cpus": os.cpu_count()}
+        line = {
+            "metric": METRIC, "value": tops, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": t_all / args.steps * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "int8", "data": "synthetic",
+            "config": {"workload": desc, "layers": len(layers), "first_layer": args.first_layer,
+                       "calib_rows_cap": args.calib_rows or None, "out_override": args.out or None, "l2": "inputs larger than L2: every step streams "
+                       f"{cal_bytes / 1e9:.1f} GB of calibration pairs and cycles {len(layers)} distinct layer buffer sets "
+                       f"({fwd_bytes / 1e6:.0f} MB)", "parallelism": f"row shards x{world}, no collective"},
+            "calibration": {"value": cal_gbs, "unit": "GB/s", "ms_per_step": t_a / args.steps * 1e3,
+                            "frac_hbm_peak": cal_gbs / world / peaks["hbm_gbs"]},
+            "forward": {"ms_per_step": t_b / args.steps * 1e3, "frac_int8_peak_burst": fwd_tops_gpu / int8_peak,
+                        "frac_int8_peak_sustained": fwd_tops_gpu / int8_peak_sus,
+                        "frac_int8_datasheet_4500": fwd_tops_gpu / 4500.0,
+                        "min_time_ms": max(t_min_compute, t_min_hbm) * 1e3,
+                        "frac_of_roofline": max(t_min_compute, t_min_hbm) / (t_b / args.steps)},
+            "roofline": dominant, "rooflines": [roof_cal, roof_fwd],
+            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+        }
+        print(json.dumps(line))
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--layers", type=int, default=0, help="only the first L layers of the workload (0 = all)")
+    ap.add_argument("--first-layer", type=int, default=0, help="skip this many layers of the workload")
+    ap.add_argument("--calib-rows", type=int, default=0, help="cap the calibration rows per layer (0 = the config's)")
+    ap.add_argument("--out", default="", choices=["", "int8", "bf16"], help="override the output stage")
+    ap.add_argument("--seed", type=int, default=0)
+    ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-cpu", action="store_true")
+    ap.add_argument("--cpu-rows", type=int, default=4096)
+    ap.add_argument("--cpu-calib-rows", type=int, default=32768)
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

@@ -155,19 +155,37 @@ __device__ __forceinline__ void cwac_solve_channel(double n, double Sq, double S
   *b = (float)(mf - alpha * mq);
 }
 
-// Adds the partials in chunk order.  stats_io (may be NULL): running statistics to update.
-// a, b (may be NULL): solve after the reduction (one-shot calibration).
-__global__ void __launch_bounds__(128)
+// Adds the partials of all row chunks.  A block owns 32 channels; its 8 row lanes each add every 8th
+// chunk, then the lanes are combined in a fixed order, so the result does not depend on scheduling.
+// stats_io (may be NULL): running statistics to update.  a, b (may be NULL): solve after the reduction.
+constexpr int kRedTX = 32;
+constexpr int kRedTY = 8;
+__global__ void __launch_bounds__(kRedTX * kRedTY)
 cwac_reduce_kernel(const double* __restrict__ partial, int chunks, int cpad, int channels, double n_rows,
                    double* __restrict__ stats_io, float* __restrict__ a, float* __restrict__ b,
                    int* __restrict__ n_degenerate) {
-  const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  if (c >= channels) return;
+  const int tx = threadIdx.x & (kRedTX - 1);
+  const int ty = threadIdx.x / kRedTX;
+  const int c = blockIdx.x * kRedTX + tx;       // < cpad by construction of the grid
   double s[4] = {0.0, 0.0, 0.0, 0.0};
-  for (int k = 0; k < chunks; ++k) {
-    const double* p = partial + (size_t)k * 4 * cpad + c;
+  if (c < channels) {
+    for (int k = ty; k < chunks; k += kRedTY) {
+      const double* p = partial + (size_t)k * 4 * cpad + c;
 #pragma unroll
-    for (int i = 0; i < 4; ++i) s[i] += p[(size_t)i * cpad];
+      for (int i = 0; i < 4; ++i) s[i] += p[(size_t)i * cpad];
+    }
+  }
+  __shared__ double red[kRedTY][4][kRedTX];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) red[ty][i][tx] = s[i];
+  __syncthreads();
+  if (ty != 0 || c >= channels) return;
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    double t = 0.0;
+#pragma unroll
+    for (int y = 0; y < kRedTY; ++y) t += red[y][i][tx];
+    s[i] = t;
   }
   double n = n_rows;
   if (stats_io != nullptr) {
@@ -247,17 +265,29 @@ pack_int4_kernel(const int8_t* __restrict__ codes, int64_t n_bytes, uint8_t* __r
 
 CwacPlan cwac_plan(int64_t rows, int32_t channels, int /*sm_count*/) {
   // The plan is a function of the shape only, so that the workspace size and the summation order
-  // (hence the bits of the result) do not depend on the device.  1184 = 148 SMs x 8 resident blocks.
+  // (hence the bits of the result) do not depend on the device.  The statistics kernel keeps two
+  // blocks resident per SM (148 x 2 = 296); the number of row chunks is chosen so that the grid fills
+  // whole waves of 296 blocks as well as possible with as few chunks as possible.
   CwacPlan p;
   p.slabs = (channels + kSlabChannels - 1) / kSlabChannels;
   p.cpad = p.slabs * kSlabChannels;
-  const int64_t target_blocks = 1184;
-  int64_t chunks = (target_blocks + p.slabs - 1) / p.slabs;
+  const int64_t resident = 296;
   const int64_t min_chunk = (int64_t)kStatsTY * kFlushRows;     // at least one full flush per thread
-  int64_t max_chunks = (rows + min_chunk - 1) / min_chunk;
-  if (chunks > max_chunks) chunks = max_chunks;
-  if (chunks < 1) chunks = 1;
-  int64_t chunk_rows = (rows + chunks - 1) / chunks;
+  const int64_t max_chunks = (rows + min_chunk - 1) / min_chunk;
+  int64_t best_chunks = 1;
+  double best_eff = -1.0;
+  for (int waves = 1; waves <= 8; ++waves) {
+    int64_t chunks = waves * resident / p.slabs;
+    if (chunks < 1) chunks = 1;
+    if (chunks > max_chunks) chunks = max_chunks;
+    const int64_t blocks = chunks * p.slabs;
+    const double eff = (double)blocks / (double)(((blocks + resident - 1) / resident) * resident);
+    if (eff > best_eff + 0.02) {
+      best_eff = eff;
+      best_chunks = chunks;
+    }
+  }
+  int64_t chunk_rows = (rows + best_chunks - 1) / best_chunks;
   chunk_rows = (chunk_rows + kStatsTY - 1) / kStatsTY * kStatsTY;
   p.chunk_rows = chunk_rows;
   p.chunks = (int)((rows + chunk_rows - 1) / chunk_rows);
@@ -277,7 +307,7 @@ qwt_status launch_cwac_stats(const float* fp_out, const float* q_out, int64_t ro
 qwt_status launch_cwac_reduce(const void* workspace, const CwacPlan& plan, int32_t channels, int64_t rows,
                               double* stats_io, float* a, float* b, int32_t* n_degenerate, cudaStream_t st) {
   if (a != nullptr && n_degenerate != nullptr) QWT_CUDA_TRY(cudaMemsetAsync(n_degenerate, 0, sizeof(int32_t), st));
-  cwac_reduce_kernel<<<(channels + 127) / 128, 128, 0, st>>>(static_cast<const double*>(workspace), plan.chunks,
+  cwac_reduce_kernel<<<(channels + kRedTX - 1) / kRedTX, kRedTX * kRedTY, 0, st>>>(static_cast<const double*>(workspace), plan.chunks,
                                                              plan.cpad, channels, (double)rows, stats_io, a, b,
                                                              n_degenerate);
   QWT_LAUNCH_CHECK();

@@ -1,4 +1,4 @@
-// Thin inline-PTX helpers for sm_100a: mbarrier, TMA (cp.async.bulk.tensor, never multicast),
+// Thin inline-PTX helpers for sm_100a: mbarrier, TMA (cp.async.bulk.tensor, each CTA loads for itself only),
 // tcgen05 (TMEM allocation, MMA, commit, load) and bounded waits.
 #pragma once
 
@@ -156,6 +156,9 @@ __device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p) {
   uint32_t v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
+}
+__device__ __forceinline__ void st_release_gpu(uint32_t* p, uint32_t v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
 __device__ __forceinline__ void red_release_gpu_add(uint32_t* p, uint32_t v) {
   asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");

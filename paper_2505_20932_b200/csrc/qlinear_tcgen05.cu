@@ -1,25 +1,27 @@
 // CWAC-fused quantized linear layer (Section 3.4, Eq. 6-11 with zero-points 0) for sm_100a.
 //
 // One persistent, warp-specialised kernel:
-//   warp 0      TMA producer: non-multicast cp.async.bulk.tensor loads of the X tile [128 x 128 B] and the
+//   warp 0      TMA producer: per-CTA cp.async.bulk.tensor loads of the X tile [128 x 128 B] and the
 //               W tile [BN x 128 B] into a ring of 128-byte-swizzled shared-memory stages
 //   warp 1      MMA issuer: one thread issues tcgen05.mma kind::i8 (128 x BN x 32 per instruction) into a
 //               TMEM accumulator; tcgen05.commit releases the stage / publishes the accumulator
-//   warps 2-5   epilogue: tcgen05.ld of the INT32 accumulators, z = fma(float(acc) * x_scale[m], fscale[n],
+//   warp 18     strip coordinator (per-token INT8 output only), see below
+//   warps 2-17  epilogue: tcgen05.ld of the INT32 accumulators, z = fma(float(acc) * x_scale[m], fscale[n],
 //               fbias[n]) (the folded M' and offset of Eq. 10-11), then the output stage.  TMEM holds
 //               512 / BN accumulator buffers so the next tile's mainloop overlaps this epilogue.
 //
 // Per-token INT8 output needs max_n |z[m, n]| over the whole row, but a CTA owns only BN columns of it.
 // Tiles are numbered strip-major (all column tiles of rows 0-127, then of rows 128-255, ...) and CTA c
-// takes tiles c, c + G, c + 2G, ...  After its mainloop a tile publishes its per-row maxima with
-// atomicMax on the float bit pattern (non-negative floats order like unsigned integers) and increments
-// its strip's arrival counter; it then waits until the counter shows every column tile of the strip,
-// re-reads its accumulator from TMEM (still resident) and emits the codes with the final row scale.
-// Progress: the lowest-numbered unpublished tile t can always run, because the tile that holds its
-// TMEM buffer (t - NACC*G) belongs to a strip whose tiles all have smaller numbers than t whenever
-// tiles_n <= G, so that strip is complete and its buffer is released.  The grid is launched
-// cooperatively so all G CTAs are resident.  Every wait is bounded; a wait that gives up records a code
-// in the workspace status word and the CTA tears down normally.
+// takes tiles c, c + G, c + 2G, ...  An epilogue warp computes z for its 32 x (BN/4) slice, keeps it in
+// registers, releases the TMEM buffer, publishes its per-row maxima with atomicMax on the float bit
+// pattern (non-negative floats order like unsigned integers) and increments its strip's arrival counter;
+// it then waits until the counter shows every slice of the strip and emits the codes with the final row
+// scale.  Progress: take the lowest-numbered tile t that has not published.  Its CTA's epilogue can only
+// be waiting on an earlier tile t - kG, whose strip ends before t whenever tiles_n <= G, so every tile of
+// that strip has published and the wait ends; the mainloop of t needs nothing but TMEM buffers that
+// lower-numbered tiles free without waiting.  The grid is launched cooperatively so all G CTAs are
+// resident.  Every wait is bounded; a wait that gives up records a code in the workspace status word and
+// the CTA tears down normally.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -39,8 +41,9 @@ constexpr int kBM = 128;           // rows of a CTA tile (= TMEM lanes)
 constexpr int kBK = 128;           // bytes of K per stage: one 128-byte swizzle row
 constexpr int kUmmaK = 32;         // K of one kind::i8 instruction
 constexpr int kTmemCols = 512;
-constexpr int kNumEpilogueWarps = 4;
-constexpr int kThreads = 32 * (2 + kNumEpilogueWarps);
+constexpr int kNumEpilogueWarps = 16;
+constexpr int kCoordWarp = 2 + kNumEpilogueWarps;      // warp that talks to the other CTAs of a row strip
+constexpr int kThreads = 32 * (3 + kNumEpilogueWarps);
 constexpr int kABytes = kBM * kBK;
 
 // status word codes (0 = clean)
@@ -58,7 +61,8 @@ struct QlParams {
   int tiles_n, num_tiles, num_kb;
   uint32_t* status;
   uint32_t* rowmax;     // [M] bit patterns of non-negative floats
-  uint32_t* counters;   // [tiles_m] arrivals of epilogue warps
+  uint32_t* counters;   // [tiles_m] tiles of the strip that have published their row maxima
+  uint32_t* flags;      // [tiles_m] set by the last tile of the strip
   uint32_t counter_target;
   unsigned long long timeout_ns;
 };
@@ -70,10 +74,10 @@ struct SmemLayout {
   static constexpr int kAcc = kTmemCols / BN;
   static constexpr int kOffA = 0;
   static constexpr int kOffB = kOffA + kStages * kABytes;
-  static constexpr int kOffFS = kOffB + kStages * kBBytes;         // float [epilogue warp][BN], private per warp
-  static constexpr int kOffFB = kOffFS + kNumEpilogueWarps * BN * 4;
-  static constexpr int kOffBars = kOffFB + kNumEpilogueWarps * BN * 4;   // full, empty, tfull, tempty, drain
-  static constexpr int kNumBars = 2 * kStages + 2 * kAcc + 1;
+  static constexpr int kOffFS = kOffB + kStages * kBBytes;         // float [epilogue warp][BN / 4], private per warp
+  static constexpr int kOffFB = kOffFS + kNumEpilogueWarps * (BN / 4) * 4;
+  static constexpr int kOffBars = kOffFB + kNumEpilogueWarps * (BN / 4) * 4;   // full, empty, tfull, tempty, drain
+  static constexpr int kNumBars = 2 * kStages + 2 * kAcc + 3;     // + drain, published, strip ready
   static constexpr int kOffMisc = kOffBars + kNumBars * 8;         // tmem base, abort word
   static constexpr int kTotal = kOffMisc + 16;
   static constexpr int kDynamic = kTotal + 1024;                   // slack to align the base to 1024
@@ -93,13 +97,7 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-__device__ __forceinline__ uint32_t quant_code(float z, float ys) {
-  int q = __float2int_rn(__fdiv_rn(z, ys));
-  q = max(-127, min(127, q));
-  return (uint32_t)q & 0xFFu;
-}
-
-template <int BN, int OUT>
+template <int BN, int OUT, bool RCP>
 __global__ void __launch_bounds__(kThreads, 1)
 qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const QlParams p) {
@@ -115,6 +113,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   uint64_t* tfull = empty + L::kStages;
   uint64_t* tempty = tfull + L::kAcc;
   uint64_t* drain = tempty + L::kAcc;
+  uint64_t* pub_bar = drain + 1;     // 16 arrivals: every epilogue warp has issued its atomicMax
+  uint64_t* ready_bar = drain + 2;   // 1 arrival: the strip's row maxima are final
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kOffMisc);
   volatile int* cta_abort = reinterpret_cast<volatile int*>(smem + L::kOffMisc + 4);
 
@@ -132,6 +132,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       ptx::mbar_init(&tempty[i], kNumEpilogueWarps);
     }
     ptx::mbar_init(drain, 1);
+    ptx::mbar_init(pub_bar, kNumEpilogueWarps);
+    ptx::mbar_init(ready_bar, 1);
     *cta_abort = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmA);
@@ -223,21 +225,68 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       }
     }
+  } else if (warp == kCoordWarp) {
+    // ------------------------------------------------------------------ strip coordinator (INT8 output only)
+    // One thread per CTA speaks for the tile: once the 16 epilogue warps have issued their row maxima it
+    // counts the tile as published; the last tile of a strip raises the strip's flag, the others poll the
+    // flag (a different word than the counter, with a back-off, so that arrivals are not queued behind
+    // polls) and then release the epilogue warps.
+    if (OUT == QWT_OUT_INT8_PER_TOKEN && lane == 0) {
+      uint32_t it = 0;
+      for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++it) {
+        const int tm = tile / p.tiles_n;
+        if (!ptx::mbar_wait_bounded(pub_bar, it & 1u, cta_abort, tmo)) {
+          give_up(kStWaitStrip);
+          break;
+        }
+        __threadfence();     // the warps' atomicMax (seen through the barrier) before the count
+        const uint32_t old = atomicAdd(p.counters + tm, 1u);
+        if (old + 1u == p.counter_target) {
+          __threadfence();
+          ptx::st_release_gpu(p.flags + tm, 1u);
+        } else {
+          uint32_t polls = 0;
+          uint64_t t0 = 0;
+          bool failed = false;
+          while (ptx::ld_acquire_gpu(p.flags + tm) == 0u) {
+            __nanosleep(64);
+            if ((++polls & 63u) == 0u) {
+              const uint64_t now = ptx::globaltimer_ns();
+              if (t0 == 0) t0 = now;
+              if (*cta_abort != 0 || now - t0 > tmo || ptx::ld_acquire_gpu(p.status) != 0u) {
+                failed = true;
+                break;
+              }
+            }
+          }
+          if (failed) {
+            give_up(kStWaitStrip);
+            break;
+          }
+        }
+        __threadfence();
+        ptx::mbar_arrive(ready_bar);
+      }
+    }
   } else {
     // ------------------------------------------------------------------ epilogue warps
-    const int qd = warp & 3;                       // TMEM lane quadrant this warp may read
-    // each warp stages the tile's fscale / fbias in its own slice (no cross-warp barrier to get stuck on)
-    float* fs = sFS + (warp - 2) * BN;
-    float* fb = sFB + (warp - 2) * BN;
+    // 16 warps: TMEM lane quadrant = warp % 4 (hardware rule), column group = (warp - 2) / 4.
+    // A warp owns 32 rows x CW columns of the tile; a thread owns one row of that.
+    constexpr int CW = BN / (kNumEpilogueWarps / 4);
+    const int qd = warp & 3;
+    const int cg = (warp - 2) >> 2;
+    // each warp stages its slice of fscale / fbias privately (no cross-warp barrier to get stuck on)
+    float* fs = sFS + (warp - 2) * CW;
+    float* fb = sFB + (warp - 2) * CW;
     uint32_t it = 0;
-    bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x, ++it) {
+    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++it) {
       const uint32_t buf = it % L::kAcc;
       const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
-      const int m0 = tm * kBM, n0 = tn * BN;
+      const int m0 = tm * kBM;
+      const int n0 = tn * BN + cg * CW;          // first column of this warp's slice
       __syncwarp();   // every lane is done with the previous tile's slice
       if (OUT != QWT_OUT_INT32_ACC) {
-        for (int i = lane; i < BN; i += 32) {
+        for (int i = lane; i < CW; i += 32) {
           const int c = n0 + i;
           fs[i] = c < p.N ? __ldg(p.fscale + c) : 0.f;
           fb[i] = c < p.N ? __ldg(p.fbias + c) : 0.f;
@@ -254,83 +303,73 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         break;
       }
       ptx::tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + buf * BN;
+      const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + buf * BN + cg * CW;
 
       if (OUT == QWT_OUT_INT8_PER_TOKEN) {
-        // pass 1: row maxima of |z| over this tile's columns
+        // z of the whole slice stays in registers; the accumulator buffer is released before the wait
+        float z[CW];
         float amax = 0.f;
-        for (int ch = 0; ch < BN / 32; ++ch) {
+#pragma unroll
+        for (int h = 0; h < CW / 32; ++h) {
           uint32_t r[32];
-          ptx::tmem_ld_32x32b_x32(taddr + ch * 32, r);
+          ptx::tmem_ld_32x32b_x32(taddr + h * 32, r);
           ptx::tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 32; ++j) {
-            const int c = ch * 32 + j;
-            amax = fmaxf(amax, fabsf(epilogue_z(r[j], xs, fs[c], fb[c])));   // columns >= N give |0*..+0| = 0
+          for (int j = 0; j < 32; j += 4) {
+            const float4 f4 = *reinterpret_cast<const float4*>(fs + h * 32 + j);
+            const float4 b4 = *reinterpret_cast<const float4*>(fb + h * 32 + j);
+            z[h * 32 + j + 0] = epilogue_z(r[j + 0], xs, f4.x, b4.x);   // columns >= N give 0 * 0 + 0
+            z[h * 32 + j + 1] = epilogue_z(r[j + 1], xs, f4.y, b4.y);
+            z[h * 32 + j + 2] = epilogue_z(r[j + 2], xs, f4.z, b4.z);
+            z[h * 32 + j + 3] = epilogue_z(r[j + 3], xs, f4.w, b4.w);
+            amax = fmaxf(fmaxf(amax, fmaxf(fabsf(z[h * 32 + j]), fabsf(z[h * 32 + j + 1]))),
+                         fmaxf(fabsf(z[h * 32 + j + 2]), fabsf(z[h * 32 + j + 3])));
           }
         }
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&tempty[buf]);
+
         if (row_ok) atomicMax(p.rowmax + row, __float_as_uint(amax));
-        __threadfence();
         __syncwarp();
-        if (lane == 0) {
-          ptx::red_release_gpu_add(p.counters + tm, 1u);
-          // wait for every column tile of this strip
-          uint32_t polls = 0;
-          uint64_t t0 = 0;
-          while (ptx::ld_acquire_gpu(p.counters + tm) < p.counter_target) {
-            if ((++polls & 63u) == 0u) {
-              const uint64_t now = ptx::globaltimer_ns();
-              if (t0 == 0) t0 = now;
-              if (*cta_abort != 0 || now - t0 > tmo || ptx::ld_acquire_gpu(p.status) != 0u) {
-                give_up(kStWaitStrip);
-                break;
-              }
-            }
-          }
-        }
-        __syncwarp();
-        if (*cta_abort != 0) {
-          ok = false;
+        if (lane == 0) ptx::mbar_arrive(pub_bar);
+        // the coordinator warp publishes the tile and waits for the rest of the strip
+        if (!ptx::mbar_wait_bounded(ready_bar, it & 1u, cta_abort, tmo)) {
+          give_up(kStWaitStrip);
           break;
         }
-        __threadfence();
         float ys = 0.f;
         if (row_ok) {
-          const float fin = __uint_as_float(__ldcg(p.rowmax + row));
-          ys = __fdiv_rn(fin, 127.f);
-          if (tn == 0) p.y_scale[row] = ys;
+          ys = __fdiv_rn(__uint_as_float(__ldcg(p.rowmax + row)), 127.f);
+          if (tn == 0 && cg == 0) p.y_scale[row] = ys;
         }
-        // pass 2: codes with the final scale
+        const float den = ys > 0.f ? ys : 1.f;       // a zero row has z == 0 everywhere: codes 0
+        const float inv = __fdiv_rn(1.f, den);
         int8_t* yrow = static_cast<int8_t*>(p.Y) + (size_t)row * p.N + n0;
-        for (int ch = 0; ch < BN / 32; ++ch) {
-          uint32_t r[32];
-          ptx::tmem_ld_32x32b_x32(taddr + ch * 32, r);
-          ptx::tmem_ld_wait();
-          uint32_t w[8];
 #pragma unroll
-          for (int g = 0; g < 8; ++g) {
-            uint32_t word = 0;
+        for (int g = 0; g < CW / 16; ++g) {
+          uint32_t w[4];
+#pragma unroll
+          for (int t = 0; t < 4; ++t) {
+            int q[4];
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
-              const int c = ch * 32 + g * 4 + j;
-              const float z = epilogue_z(r[g * 4 + j], xs, fs[c], fb[c]);
-              const uint32_t code = ys > 0.f ? quant_code(z, ys) : 0u;
-              word |= code << (8 * j);
+              const float zz = z[g * 16 + t * 4 + j];
+              q[j] = __float2int_rn(RCP ? __fmul_rn(zz, inv) : __fdiv_rn(zz, den));   // |q| <= 127 by construction
             }
-            w[g] = word;
+            const uint32_t lo = __byte_perm((uint32_t)q[0], (uint32_t)q[1], 0x0040);
+            const uint32_t hi = __byte_perm((uint32_t)q[2], (uint32_t)q[3], 0x0040);
+            w[t] = __byte_perm(lo, hi, 0x5410);
           }
-          if (row_ok) {
-            const int c0 = n0 + ch * 32;
-            if (c0 + 16 <= p.N) st_v4(yrow + ch * 32, w[0], w[1], w[2], w[3]);
-            if (c0 + 32 <= p.N) st_v4(yrow + ch * 32 + 16, w[4], w[5], w[6], w[7]);
-          }
+          if (row_ok && n0 + g * 16 + 16 <= p.N) st_v4(yrow + g * 16, w[0], w[1], w[2], w[3]);
         }
       } else {
-        for (int ch = 0; ch < BN / 32; ++ch) {
+#pragma unroll
+        for (int h = 0; h < CW / 32; ++h) {
           uint32_t r[32];
-          ptx::tmem_ld_32x32b_x32(taddr + ch * 32, r);
+          ptx::tmem_ld_32x32b_x32(taddr + h * 32, r);
           ptx::tmem_ld_wait();
-          const int c0 = n0 + ch * 32;
+          const int c0 = n0 + h * 32;
           if (OUT == QWT_OUT_INT32_ACC) {
             if (row_ok) {
               int32_t* yrow = static_cast<int32_t*>(p.Y) + (size_t)row * p.N + c0;
@@ -341,7 +380,14 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           } else {
             float z[32];
 #pragma unroll
-            for (int j = 0; j < 32; ++j) z[j] = epilogue_z(r[j], xs, fs[ch * 32 + j], fb[ch * 32 + j]);
+            for (int j = 0; j < 32; j += 4) {
+              const float4 f4 = *reinterpret_cast<const float4*>(fs + h * 32 + j);
+              const float4 b4 = *reinterpret_cast<const float4*>(fb + h * 32 + j);
+              z[j + 0] = epilogue_z(r[j + 0], xs, f4.x, b4.x);
+              z[j + 1] = epilogue_z(r[j + 1], xs, f4.y, b4.y);
+              z[j + 2] = epilogue_z(r[j + 2], xs, f4.z, b4.z);
+              z[j + 3] = epilogue_z(r[j + 3], xs, f4.w, b4.w);
+            }
             if (OUT == QWT_OUT_FP32) {
               if (row_ok) {
                 float* yrow = static_cast<float*>(p.Y) + (size_t)row * p.N + c0;
@@ -363,11 +409,11 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
           }
         }
+        // accumulator buffer is free again
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&tempty[buf]);
       }
-      // accumulator buffer is free again
-      ptx::tc_fence_before();
-      __syncwarp();
-      if (lane == 0) ptx::mbar_arrive(&tempty[buf]);
     }
   }
 
@@ -428,11 +474,21 @@ unsigned long long timeout_ns_from_env() {
   return v;
 }
 
-template <int BN, int OUT>
+// QWT_REQUANT_RECIPROCAL=1 replaces the division z / y_scale by a multiplication with 1 / y_scale
+// (codes may then differ from the division by one step on a few elements per million).
+bool requant_by_reciprocal() {
+  static const bool v = [] {
+    const char* e = getenv("QWT_REQUANT_RECIPROCAL");
+    return e != nullptr && e[0] == '1';
+  }();
+  return v;
+}
+
+template <int BN, int OUT, bool RCP>
 qwt_status launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
                        bool cooperative, cudaStream_t st) {
   using L = SmemLayout<BN>;
-  auto kern = qlinear_cwac_kernel<BN, OUT>;
+  auto kern = qlinear_cwac_kernel<BN, OUT, RCP>;
   // per device and cheap, so it is simply set on every launch
   QWT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic));
   if (cooperative) {
@@ -451,13 +507,14 @@ qwt_status launch_bn(int out_mode, const CUtensorMap& tmA, const CUtensorMap& tm
                      cudaStream_t st) {
   switch (out_mode) {
     case QWT_OUT_INT8_PER_TOKEN:
-      return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN>(tmA, tmB, prm, grid, true, st);
+      if (requant_by_reciprocal()) return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN, true>(tmA, tmB, prm, grid, true, st);
+      return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN, false>(tmA, tmB, prm, grid, true, st);
     case QWT_OUT_BF16:
-      return launch_inst<BN, QWT_OUT_BF16>(tmA, tmB, prm, grid, false, st);
+      return launch_inst<BN, QWT_OUT_BF16, false>(tmA, tmB, prm, grid, false, st);
     case QWT_OUT_FP32:
-      return launch_inst<BN, QWT_OUT_FP32>(tmA, tmB, prm, grid, false, st);
+      return launch_inst<BN, QWT_OUT_FP32, false>(tmA, tmB, prm, grid, false, st);
     case QWT_OUT_INT32_ACC:
-      return launch_inst<BN, QWT_OUT_INT32_ACC>(tmA, tmB, prm, grid, false, st);
+      return launch_inst<BN, QWT_OUT_INT32_ACC, false>(tmA, tmB, prm, grid, false, st);
   }
   return QWT_ERR_UNSUPPORTED;
 }
@@ -473,13 +530,15 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   // 256-wide tiles keep the tensor pipe ahead of shared-memory bandwidth; 128-wide ones are used when
   // the wider tile would leave many SMs without work.
   const int sms = dev.sm_count > 0 ? dev.sm_count : 148;
-  const long t256 = (long)pl.tiles_m * ((N + 255) / 256);
-  const long t128 = (long)pl.tiles_m * ((N + 127) / 128);
-  auto waves_eff = [&](long tiles) {
+  auto score = [&](int bn) {
+    const long tn = (N + bn - 1) / bn;
+    const long tiles = (long)pl.tiles_m * tn;
     const long waves = (tiles + sms - 1) / sms;
-    return (double)tiles / (double)(waves * sms);
+    const double wave_eff = (double)tiles / (double)(waves * sms);   // SMs busy in the last round
+    const double pad_eff = (double)N / (double)(tn * bn);            // useful columns of the tiles
+    return wave_eff * pad_eff;
   };
-  pl.bn = (N > 128 && waves_eff(t256) + 0.10 >= waves_eff(t128)) ? 256 : 128;
+  pl.bn = (N > 128 && score(256) + 0.05 >= score(128)) ? 256 : 128;
   const char* force = getenv("QWT_FORCE_BN");
   if (force != nullptr) {
     const int f = atoi(force);
@@ -496,6 +555,8 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   pl.ws_rowmax_off = off;
   off += ((size_t)M * 4 + 255) / 256 * 256;
   pl.ws_counter_off = off;
+  off += ((size_t)pl.tiles_m * 4 + 255) / 256 * 256;
+  pl.ws_flag_off = off;
   off += ((size_t)pl.tiles_m * 4 + 255) / 256 * 256;
   pl.ws_z_off = off;
   if (out_mode == QWT_OUT_INT8_PER_TOKEN && !pl.fused_requant) off += (size_t)M * N * 4;
@@ -533,7 +594,8 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   prm.status = reinterpret_cast<uint32_t*>(ws + plan.ws_status_off);
   prm.rowmax = reinterpret_cast<uint32_t*>(ws + plan.ws_rowmax_off);
   prm.counters = reinterpret_cast<uint32_t*>(ws + plan.ws_counter_off);
-  prm.counter_target = (uint32_t)plan.tiles_n * kNumEpilogueWarps;
+  prm.flags = reinterpret_cast<uint32_t*>(ws + plan.ws_flag_off);
+  prm.counter_target = (uint32_t)plan.tiles_n;
   prm.timeout_ns = timeout_ns_from_env();
 
   int mode = out_mode;

@@ -70,7 +70,7 @@ struct QlinearPlan {
   int grid;
   size_t smem_bytes;
   bool fused_requant;    // cross-CTA row-max protocol inside the GEMM kernel
-  size_t ws_status_off, ws_rowmax_off, ws_counter_off, ws_z_off, ws_total;
+  size_t ws_status_off, ws_rowmax_off, ws_counter_off, ws_flag_off, ws_z_off, ws_total;
 };
 qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
                         QlinearPlan* plan);
