@@ -34,7 +34,8 @@ enum {
   QWT_ERR_WORKSPACE = 5,   /* workspace too small */
   QWT_ERR_CUDA = 6,        /* a CUDA runtime/driver call failed; see qwt_last_cuda_error */
   QWT_ERR_TIMEOUT = 7,     /* a bounded device-side wait gave up (reported by qwt_qlinear_check_status) */
-  QWT_ERR_ARCH = 8         /* current device is not compute capability 10.x */
+  QWT_ERR_ARCH = 8,        /* current device is not compute capability 10.x */
+  QWT_ERR_TOO_LARGE = 9    /* problem exceeds the fixed scratch of qwt_cwac_calibrate_noalloc */
 };
 
 /* weight storage */
@@ -95,6 +96,24 @@ qwt_status qwt_cwac_calibrate_host(const float* fp_out /*HOST*/, const float* q_
                                    int32_t channels, int64_t ld, float* a /*HOST*/, float* b /*HOST*/,
                                    int32_t* n_degenerate /*HOST, may be NULL*/,
                                    void* staging, size_t staging_bytes, void* stream);
+
+/* Calibration without any workspace argument (the paper has no counterpart: this is a packaging variant of
+ * qwt_cwac_calibrate, same kernels, same results within the library's calibration tolerance).
+ * For callers that cannot allocate device memory -- e.g. a plug-in confined to a host program's fixed
+ * memory arena, or a service that must not call cudaMalloc while it is serving.  The per-chunk partial sums
+ * live in a fixed array of QWT_NOALLOC_SCRATCH_BYTES inside the library image; every GPU that loads the
+ * library holds that array until the process exits.  The call itself allocates nothing.
+ *   - Limit: channels (rounded up to 128) * 32 bytes must fit the array, i.e. at most 131072 channels;
+ *     otherwise QWT_ERR_TOO_LARGE.  Long inputs are cut into fewer, longer row chunks so that they fit.
+ *   - The first call on each device looks up the array's device address (with that device current); make
+ *     that first call before any stream capture is started.
+ *   - All calls share the one array.  Nothing in it has to be cleared between calls (each call overwrites
+ *     what it reads), but two calls that overlap on the GPU -- different streams, or different host threads
+ *     -- race on it: serialise them, or use qwt_cwac_calibrate with separate workspaces.
+ * Arguments and other errors as for qwt_cwac_calibrate. */
+#define QWT_NOALLOC_SCRATCH_BYTES (4u << 20)
+qwt_status qwt_cwac_calibrate_noalloc(const float* fp_out, const float* q_out, int64_t rows, int32_t channels,
+                                      int64_t ld, float* a, float* b, int32_t* n_degenerate, void* stream);
 
 /* ---------------------------------------------------------------------------------------------
  * Fold -- Section 3.4, Eq. 9-11.  CWAC is absorbed into the layer's requantization parameters:

@@ -20,7 +20,8 @@ lib = C.CDLL(LIB_PATH)
 
 # status / enums (mirrors of qwt2.h)
 QWT_OK, QWT_ERR_NULL, QWT_ERR_SHAPE, QWT_ERR_ALIGN, QWT_ERR_UNSUPPORTED = 0, 1, 2, 3, 4
-QWT_ERR_WORKSPACE, QWT_ERR_CUDA, QWT_ERR_TIMEOUT, QWT_ERR_ARCH = 5, 6, 7, 8
+QWT_ERR_WORKSPACE, QWT_ERR_CUDA, QWT_ERR_TIMEOUT, QWT_ERR_ARCH, QWT_ERR_TOO_LARGE = 5, 6, 7, 8, 9
+QWT_NOALLOC_SCRATCH_BYTES = 4 << 20
 QWT_W_INT8, QWT_W_INT4_PACKED = 0, 1
 QWT_OUT_INT8_PER_TOKEN, QWT_OUT_BF16, QWT_OUT_FP32, QWT_OUT_INT32_ACC = 0, 1, 2, 3
 
@@ -37,6 +38,7 @@ SIGNATURES = {
     "qwt_cwac_solve": (_i32, [_p, _i32, _p, _p, _p, _p]),
     "qwt_cwac_host_staging_bytes": (_sz, [_i64, _i32]),
     "qwt_cwac_calibrate_host": (_i32, [_p, _p, _i64, _i32, _i64, _p, _p, _p, _p, _sz, _p]),
+    "qwt_cwac_calibrate_noalloc": (_i32, [_p, _p, _i64, _i32, _i64, _p, _p, _p, _p]),
     "qwt_cwac_fold": (_i32, [_p, _p, _p, _p, _i32, _p, _p, _p]),
     "qwt_qlinear_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32, _i32]),
     "qwt_qlinear_cwac_forward": (_i32, [_p, _p, _p, _i32, _p, _p, _i32, _i32, _i32, _i32, _p, _p, _p, _sz, _p]),
@@ -142,6 +144,16 @@ def qwt_cwac_calibrate_host(fp_out, q_out, rows, channels, ld, a, b, n_degenerat
                                     _ptr(n_degenerate), _ptr(staging), staging_bytes, _stream(stream))
     if check:
         _check(s, "qwt_cwac_calibrate_host")
+    return s
+
+
+def qwt_cwac_calibrate_noalloc(fp_out, q_out, rows, channels, ld, a, b, n_degenerate, stream=None, check=True) -> int:
+    """Calibration that takes no workspace: for callers that may not allocate device memory.  The scratch is a
+    fixed array inside the library (see include/qwt2.h for its limit and the rule about overlapping calls)."""
+    s = lib.qwt_cwac_calibrate_noalloc(_ptr(fp_out), _ptr(q_out), rows, channels, ld, _ptr(a), _ptr(b),
+                                       _ptr(n_degenerate), _stream(stream))
+    if check:
+        _check(s, "qwt_cwac_calibrate_noalloc")
     return s
 
 

@@ -70,6 +70,7 @@ const char* qwt_status_string(qwt_status s) {
     case QWT_ERR_CUDA: return "CUDA call failed";
     case QWT_ERR_TIMEOUT: return "device-side wait timed out";
     case QWT_ERR_ARCH: return "device is not compute capability 10.x";
+    case QWT_ERR_TOO_LARGE: return "problem exceeds the fixed scratch array of the no-allocation entry point";
     default: return "unknown status";
   }
 }
