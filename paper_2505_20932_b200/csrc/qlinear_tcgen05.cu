@@ -6,6 +6,7 @@
 //   warp 1      MMA issuer: one thread issues tcgen05.mma kind::i8 (128 x BN x 32 per instruction) into a
 //               TMEM accumulator; tcgen05.commit releases the stage / publishes the accumulator
 //   warp 18     strip coordinator (per-token INT8 output only), see below
+//   warps 19-22 (packed int4 weights only) expand the W tile to int8 in shared memory before the MMA
 //   warps 2-17  epilogue: tcgen05.ld of the INT32 accumulators, z = fma(float(acc) * x_scale[m], fscale[n],
 //               fbias[n]) (the folded M' and offset of Eq. 10-11), then the output stage.  TMEM holds
 //               512 / BN accumulator buffers so the next tile's mainloop overlaps this epilogue.
@@ -43,7 +44,10 @@ constexpr int kUmmaK = 32;         // K of one kind::i8 instruction
 constexpr int kTmemCols = 512;
 constexpr int kNumEpilogueWarps = 16;
 constexpr int kCoordWarp = 2 + kNumEpilogueWarps;      // warp that talks to the other CTAs of a row strip
-constexpr int kThreads = 32 * (3 + kNumEpilogueWarps);
+constexpr int kConvWarp0 = kCoordWarp + 1;              // first of 4 W4 -> INT8 converter warps (packed weights only)
+constexpr int kNumConvWarps = 4;
+constexpr int kThreadsW8 = 32 * (3 + kNumEpilogueWarps);
+constexpr int kThreadsW4 = kThreadsW8 + 32 * kNumConvWarps;
 constexpr int kABytes = kBM * kBK;
 
 // status word codes (0 = clean)
@@ -67,20 +71,24 @@ struct QlParams {
   unsigned long long timeout_ns;
 };
 
-template <int BN>
+template <int BN, bool W4>
 struct SmemLayout {
-  static constexpr int kBBytes = BN * kBK;
-  static constexpr int kStages = (BN == 256) ? 4 : 6;
+  static constexpr int kBBytes = BN * kBK;                 // expanded (int8) W tile of one stage
+  static constexpr int kPBytes = W4 ? BN * (kBK / 2) : 0;  // packed (int4) W tile of one stage
+  static constexpr int kStages = W4 ? ((BN == 256) ? 3 : 5) : ((BN == 256) ? 4 : 6);
   static constexpr int kAcc = kTmemCols / BN;
   static constexpr int kOffA = 0;
   static constexpr int kOffB = kOffA + kStages * kABytes;
-  static constexpr int kOffFS = kOffB + kStages * kBBytes;         // float [epilogue warp][BN / 4], private per warp
+  static constexpr int kOffP = kOffB + kStages * kBBytes;
+  static constexpr int kOffFS = kOffP + kStages * kPBytes;         // float [epilogue warp][BN / 4], private per warp
   static constexpr int kOffFB = kOffFS + kNumEpilogueWarps * (BN / 4) * 4;
-  static constexpr int kOffBars = kOffFB + kNumEpilogueWarps * (BN / 4) * 4;   // full, empty, tfull, tempty, drain
-  static constexpr int kNumBars = 2 * kStages + 2 * kAcc + 3;     // + drain, published, strip ready
+  static constexpr int kOffBars = kOffFB + kNumEpilogueWarps * (BN / 4) * 4;
+  // full[S], empty[S], conv[S], tfull[A], tempty[A], drain, published, strip ready
+  static constexpr int kNumBars = 3 * kStages + 2 * kAcc + 3;
   static constexpr int kOffMisc = kOffBars + kNumBars * 8;         // tmem base, abort word
   static constexpr int kTotal = kOffMisc + 16;
   static constexpr int kDynamic = kTotal + 1024;                   // slack to align the base to 1024
+  static_assert(kDynamic <= 232448, "shared memory budget of one CTA");
 };
 
 __device__ __forceinline__ float epilogue_z(uint32_t acc_bits, float xs, float fs, float fb) {
@@ -97,20 +105,22 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int BN, int OUT, bool RCP>
-__global__ void __launch_bounds__(kThreads, 1)
+template <int BN, int OUT, bool RCP, bool W4>
+__global__ void __launch_bounds__(W4 ? kThreadsW4 : kThreadsW8, 1)
 qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const QlParams p) {
-  using L = SmemLayout<BN>;
+  using L = SmemLayout<BN, W4>;
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
   uint8_t* sA = smem + L::kOffA;
   uint8_t* sB = smem + L::kOffB;
+  uint8_t* sP = smem + L::kOffP;     // packed int4 tiles (W4 only)
   float* sFS = reinterpret_cast<float*>(smem + L::kOffFS);
   float* sFB = reinterpret_cast<float*>(smem + L::kOffFB);
   uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kOffBars);
   uint64_t* empty = full + L::kStages;
-  uint64_t* tfull = empty + L::kStages;
+  uint64_t* conv = empty + L::kStages;     // W4 only: the stage's W tile has been expanded to int8
+  uint64_t* tfull = conv + L::kStages;
   uint64_t* tempty = tfull + L::kAcc;
   uint64_t* drain = tempty + L::kAcc;
   uint64_t* pub_bar = drain + 1;     // 16 arrivals: every epilogue warp has issued its atomicMax
@@ -126,6 +136,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     for (int i = 0; i < L::kStages; ++i) {
       ptx::mbar_init(&full[i], 1);
       ptx::mbar_init(&empty[i], 1);
+      ptx::mbar_init(&conv[i], kNumConvWarps);
     }
     for (int i = 0; i < L::kAcc; ++i) {
       ptx::mbar_init(&tfull[i], 1);
@@ -168,9 +179,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             ok = false;
             break;
           }
-          ptx::mbar_arrive_expect_tx(&full[s], kABytes + L::kBBytes);
+          ptx::mbar_arrive_expect_tx(&full[s], kABytes + (W4 ? L::kPBytes : L::kBBytes));
           ptx::tma_load_2d(sA + s * kABytes, &tmA, kb * kBK, m0, &full[s]);
-          ptx::tma_load_2d(sB + s * L::kBBytes, &tmB, kb * kBK, n0, &full[s]);
+          if (W4) ptx::tma_load_2d(sP + s * L::kPBytes, &tmB, kb * (kBK / 2), n0, &full[s]);
+          else ptx::tma_load_2d(sB + s * L::kBBytes, &tmB, kb * kBK, n0, &full[s]);
         }
       }
       if (*cta_abort != 0) {
@@ -200,7 +212,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const uint32_t d_tmem = tmem_base + buf * BN;
         for (int kb = 0; kb < p.num_kb; ++kb, ++kbi) {
           const uint32_t s = kbi % L::kStages;
-          if (!ptx::mbar_wait_bounded(&full[s], (kbi / L::kStages) & 1u, cta_abort, tmo)) {
+          if (!ptx::mbar_wait_bounded(W4 ? &conv[s] : &full[s], (kbi / L::kStages) & 1u, cta_abort, tmo)) {
             give_up(kStWaitFull);
             ok = false;
             break;
@@ -223,6 +235,48 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         uint32_t polls = 0;
         while (!ptx::mbar_try_wait(drain, 0) && ++polls < (1u << 16)) {
         }
+      }
+    }
+  } else if (W4 && warp >= kConvWarp0) {
+    // ------------------------------------------------------------------ W4 -> INT8 converter warps
+    // The packed tile (64 bytes per row, two's-complement nibbles, even element low) is expanded into the
+    // 128-byte-swizzled operand tile the MMA descriptor expects.  Each nibble is moved to the HIGH half of
+    // its byte, i.e. the operand holds 16 x code (|16 code| <= 112 fits int8); the factor 1/16 is exact in
+    // the epilogue (fscale / 16, or an arithmetic shift of the raw accumulators).
+    const int ct = threadIdx.x - kConvWarp0 * 32;          // 0..127
+    uint32_t kbi = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+      for (int kb = 0; kb < p.num_kb; ++kb, ++kbi) {
+        const uint32_t s = kbi % L::kStages;
+        if (!ptx::mbar_wait_bounded(&full[s], (kbi / L::kStages) & 1u, cta_abort, tmo)) {
+          give_up(kStWaitFull);
+          ok = false;
+          break;
+        }
+        const uint8_t* src = sP + s * L::kPBytes;
+        uint8_t* dst = sB + s * L::kBBytes;
+#pragma unroll 2
+        for (int q = ct; q < BN * 4; q += 32 * kNumConvWarps) {
+          const int n = q >> 2, c = q & 3;                 // row of the tile, 16-byte chunk of the packed row
+          const uint4 w = *reinterpret_cast<const uint4*>(src + n * 64 + c * 16);
+          const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+          uint32_t out[8];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t lo = (in[i] << 4) & 0xF0F0F0F0u;   // even elements, nibble in the high half
+            const uint32_t hi = in[i] & 0xF0F0F0F0u;          // odd elements
+            out[2 * i] = __byte_perm(lo, hi, 0x5140);         // e0 e1 e2 e3
+            out[2 * i + 1] = __byte_perm(lo, hi, 0x7362);     // e4 e5 e6 e7
+          }
+          uint8_t* row = dst + n * 128;
+          const int sw = n & 7;                              // 128-byte swizzle: chunk ^= row % 8
+          *reinterpret_cast<uint4*>(row + (((2 * c) ^ sw) << 4)) = make_uint4(out[0], out[1], out[2], out[3]);
+          *reinterpret_cast<uint4*>(row + (((2 * c + 1) ^ sw) << 4)) = make_uint4(out[4], out[5], out[6], out[7]);
+        }
+        ptx::fence_proxy_async_smem();     // generic-proxy writes -> visible to the tensor core's async proxy
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&conv[s]);
       }
     }
   } else if (warp == kCoordWarp) {
@@ -288,7 +342,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       if (OUT != QWT_OUT_INT32_ACC) {
         for (int i = lane; i < CW; i += 32) {
           const int c = n0 + i;
-          fs[i] = c < p.N ? __ldg(p.fscale + c) : 0.f;
+          fs[i] = c < p.N ? __ldg(p.fscale + c) * (W4 ? 0.0625f : 1.0f) : 0.f;   // W4 operands hold 16 x code
           fb[i] = c < p.N ? __ldg(p.fbias + c) : 0.f;
         }
       }
@@ -371,6 +425,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           ptx::tmem_ld_wait();
           const int c0 = n0 + h * 32;
           if (OUT == QWT_OUT_INT32_ACC) {
+            if (W4) {
+#pragma unroll
+              for (int j = 0; j < 32; ++j) r[j] = (uint32_t)((int)r[j] >> 4);   // exact: every term is a multiple of 16
+            }
             if (row_ok) {
               int32_t* yrow = static_cast<int32_t*>(p.Y) + (size_t)row * p.N + c0;
 #pragma unroll
@@ -484,11 +542,12 @@ bool requant_by_reciprocal() {
   return v;
 }
 
-template <int BN, int OUT, bool RCP>
+template <int BN, int OUT, bool RCP, bool W4>
 qwt_status launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
                        bool cooperative, cudaStream_t st) {
-  using L = SmemLayout<BN>;
-  auto kern = qlinear_cwac_kernel<BN, OUT, RCP>;
+  using L = SmemLayout<BN, W4>;
+  constexpr int kThreads = W4 ? kThreadsW4 : kThreadsW8;
+  auto kern = qlinear_cwac_kernel<BN, OUT, RCP, W4>;
   // per device and cheap, so it is simply set on every launch
   QWT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic));
   if (cooperative) {
@@ -502,19 +561,20 @@ qwt_status launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const QlP
   return QWT_OK;
 }
 
-template <int BN>
+template <int BN, bool W4>
 qwt_status launch_bn(int out_mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
                      cudaStream_t st) {
   switch (out_mode) {
     case QWT_OUT_INT8_PER_TOKEN:
-      if (requant_by_reciprocal()) return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN, true>(tmA, tmB, prm, grid, true, st);
-      return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN, false>(tmA, tmB, prm, grid, true, st);
+      if (requant_by_reciprocal())
+        return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN, true, W4>(tmA, tmB, prm, grid, true, st);
+      return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN, false, W4>(tmA, tmB, prm, grid, true, st);
     case QWT_OUT_BF16:
-      return launch_inst<BN, QWT_OUT_BF16, false>(tmA, tmB, prm, grid, false, st);
+      return launch_inst<BN, QWT_OUT_BF16, false, W4>(tmA, tmB, prm, grid, false, st);
     case QWT_OUT_FP32:
-      return launch_inst<BN, QWT_OUT_FP32, false>(tmA, tmB, prm, grid, false, st);
+      return launch_inst<BN, QWT_OUT_FP32, false, W4>(tmA, tmB, prm, grid, false, st);
     case QWT_OUT_INT32_ACC:
-      return launch_inst<BN, QWT_OUT_INT32_ACC, false>(tmA, tmB, prm, grid, false, st);
+      return launch_inst<BN, QWT_OUT_INT32_ACC, false, W4>(tmA, tmB, prm, grid, false, st);
   }
   return QWT_ERR_UNSUPPORTED;
 }
@@ -524,7 +584,6 @@ qwt_status launch_bn(int out_mode, const CUtensorMap& tmA, const CUtensorMap& tm
 qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
                         QlinearPlan* plan) {
   (void)K;
-  (void)wfmt;
   QlinearPlan pl{};
   pl.tiles_m = (M + kBM - 1) / kBM;
   // 256-wide tiles keep the tensor pipe ahead of shared-memory bandwidth; 128-wide ones are used when
@@ -547,7 +606,9 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   pl.tiles_n = (N + pl.bn - 1) / pl.bn;
   const long tiles = (long)pl.tiles_m * pl.tiles_n;
   pl.grid = (int)(tiles < sms ? tiles : sms);
-  pl.smem_bytes = pl.bn == 256 ? SmemLayout<256>::kDynamic : SmemLayout<128>::kDynamic;
+  const bool w4 = wfmt == QWT_W_INT4_PACKED;
+  pl.smem_bytes = pl.bn == 256 ? (w4 ? SmemLayout<256, true>::kDynamic : SmemLayout<256, false>::kDynamic)
+                               : (w4 ? SmemLayout<128, true>::kDynamic : SmemLayout<128, false>::kDynamic);
   pl.fused_requant = (out_mode == QWT_OUT_INT8_PER_TOKEN) && (pl.tiles_n <= pl.grid);
   size_t off = 0;
   pl.ws_status_off = off;
@@ -568,11 +629,15 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
 qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, int32_t wfmt, const float* fscale,
                           const float* fbias, int32_t M, int32_t N, int32_t K, int32_t out_mode, void* Y,
                           float* y_scale, void* workspace, const QlinearPlan& plan, cudaStream_t st) {
-  if (wfmt != QWT_W_INT8) return QWT_ERR_UNSUPPORTED;
+  const bool w4 = wfmt == QWT_W_INT4_PACKED;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   CUtensorMap tmA, tmB;
-  if (!make_byte_map(&tmA, X, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B) ||
-      !make_byte_map(&tmB, W, (uint64_t)N, (uint64_t)K, kBK, (uint32_t)plan.bn, CU_TENSOR_MAP_SWIZZLE_128B)) {
+  const bool okA = make_byte_map(&tmA, X, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+  const bool okB = w4 ? make_byte_map(&tmB, W, (uint64_t)N, (uint64_t)K / 2, kBK / 2, (uint32_t)plan.bn,
+                                      CU_TENSOR_MAP_SWIZZLE_NONE)
+                      : make_byte_map(&tmB, W, (uint64_t)N, (uint64_t)K, kBK, (uint32_t)plan.bn,
+                                      CU_TENSOR_MAP_SWIZZLE_128B);
+  if (!okA || !okB) {
     set_cuda_error((int)cudaErrorInvalidValue);
     return QWT_ERR_CUDA;
   }
@@ -604,8 +669,11 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
     mode = QWT_OUT_FP32;
     prm.Y = ws + plan.ws_z_off;
   }
-  qwt_status s = plan.bn == 256 ? launch_bn<256>(mode, tmA, tmB, prm, plan.grid, st)
-                                : launch_bn<128>(mode, tmA, tmB, prm, plan.grid, st);
+  qwt_status s;
+  if (w4) s = plan.bn == 256 ? launch_bn<256, true>(mode, tmA, tmB, prm, plan.grid, st)
+                             : launch_bn<128, true>(mode, tmA, tmB, prm, plan.grid, st);
+  else s = plan.bn == 256 ? launch_bn<256, false>(mode, tmA, tmB, prm, plan.grid, st)
+                          : launch_bn<128, false>(mode, tmA, tmB, prm, plan.grid, st);
   if (s != QWT_OK) return s;
   if (mode != out_mode)
     return launch_quantize_rows(reinterpret_cast<const float*>(ws + plan.ws_z_off), M, N, N, 127,

@@ -166,3 +166,72 @@ def test_forward_from_host_memory(H, B):
     c_ref, ys_ref = O.requant_per_token(O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb))
     assert np.allclose(ys, ys_ref, rtol=1e-5)
     assert_codes_close(Y, c_ref)
+
+
+# ------------------------------------------------------------------ packed 4-bit weights (W4A8)
+
+def random_w4_layer(M, N, K, seed):
+    rng = np.random.default_rng(seed)
+    Xq = rng.integers(-127, 128, (M, K)).astype(np.int8)
+    Wq = rng.integers(-7, 8, (N, K)).astype(np.int8)
+    xs = rng.uniform(0.01, 0.05, M).astype(np.float32)
+    ws = rng.uniform(2e-3, 6e-3, N).astype(np.float32)
+    bias = (0.01 * rng.standard_normal(N)).astype(np.float32)
+    a = (1 + 0.05 * rng.standard_normal(N)).astype(np.float32)
+    b = (0.02 * rng.standard_normal(N)).astype(np.float32)
+    fs64, fb64 = O.cwac_fold(ws, bias, a, b)
+    return Xq, Wq, O.pack_int4(Wq), xs, fs64.astype(np.float32), fb64.astype(np.float32)
+
+
+W4_SHAPES = [(128, 128, 128), (1, 16, 32), (130, 272, 416), (300, 2304, 768), (500, 768, 3072), (2000, 384, 1536)]
+
+
+@pytest.mark.parametrize("M,N,K", W4_SHAPES)
+def test_w4_int32_accumulators_bit_exact(H, B, M, N, K):
+    Xq, Wq, Wp, *_ = random_w4_layer(M, N, K, seed=M + N + K)
+    acc, _ = H.gpu_forward(Xq, None, Wp, None, None, B.QWT_OUT_INT32_ACC, wfmt=B.QWT_W_INT4_PACKED, K=K)
+    assert np.array_equal(acc.astype(np.int64), O.int_matmul(Xq, Wq))
+
+
+def test_w4_extreme_codes(H, B):
+    M, N, K = 130, 144, 3072
+    Xq = np.full((M, K), 127, np.int8)
+    Xq[1::2] = -127
+    Wq = np.full((N, K), -7, np.int8)
+    Wq[::3] = 7
+    Wq[:, 1::2] *= -1                                     # even and odd nibbles differ
+    acc, _ = H.gpu_forward(Xq, None, O.pack_int4(Wq), None, None, B.QWT_OUT_INT32_ACC, wfmt=B.QWT_W_INT4_PACKED, K=K)
+    assert np.array_equal(acc.astype(np.int64), O.int_matmul(Xq, Wq))
+
+
+@pytest.mark.parametrize("M,N,K", W4_SHAPES)
+def test_w4_bf16_fp32_and_int8_outputs(H, B, M, N, K):
+    Xq, Wq, Wp, xs, fs, fb = random_w4_layer(M, N, K, seed=M + N + K + 7)
+    z_ref = O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb)
+    z, _ = H.gpu_forward(Xq, xs, Wp, fs, fb, B.QWT_OUT_FP32, wfmt=B.QWT_W_INT4_PACKED, K=K)
+    assert_fp32_close(z, z_ref)
+    if N % 8 == 0:
+        bits, _ = H.gpu_forward(Xq, xs, Wp, fs, fb, B.QWT_OUT_BF16, wfmt=B.QWT_W_INT4_PACKED, K=K)
+        d = np.abs(bits.astype(np.int32) - O.to_bf16_bits(z_ref).astype(np.int32))
+        assert d.max() <= 1 and np.count_nonzero(d) <= max(1, int(1e-4 * d.size))
+    codes, ys = H.gpu_forward(Xq, xs, Wp, fs, fb, B.QWT_OUT_INT8_PER_TOKEN, wfmt=B.QWT_W_INT4_PACKED, K=K)
+    c_ref, ys_ref = O.requant_per_token(z_ref)
+    assert np.allclose(ys, ys_ref, rtol=1e-5)
+    assert_codes_close(codes, c_ref)
+
+
+def test_w4_quantize_pack_forward_chain(H, B):
+    """Config 3 shaped layer (one ViT-B fc1 at a reduced token count): W4 per-channel quantizer -> packing -> BF16 forward."""
+    spec = WL.LayerSpec("vit_b.fc1", 600, 768, 3072, 4, "bf16", "lognormal_channel", 600)
+    d = WL.host_layer_inputs(spec, seed=3)
+    Xq, xs = O.quantize_rows_sym(d["X"], 127)
+    Wq, ws = O.quantize_rows_sym(d["W"], 7)
+    gWq, gws = H.gpu_quantize_rows(d["W"], 7)
+    assert np.array_equal(gWq, Wq) and np.array_equal(gws, ws)
+    assert np.array_equal(H.gpu_pack_int4(gWq), O.pack_int4(Wq))
+    fs, fb = O.cwac_fold(ws, d["bias"], None, None)
+    fs, fb = fs.astype(np.float32), fb.astype(np.float32)
+    bits, _ = H.gpu_forward(Xq, xs, O.pack_int4(Wq), fs, fb, B.QWT_OUT_BF16, wfmt=B.QWT_W_INT4_PACKED, K=spec.K)
+    z_ref = O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb)
+    dd = np.abs(bits.astype(np.int32) - O.to_bf16_bits(z_ref).astype(np.int32))
+    assert dd.max() <= 1 and np.count_nonzero(dd) <= max(1, int(1e-4 * dd.size))
