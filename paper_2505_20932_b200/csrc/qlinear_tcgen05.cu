@@ -1,28 +1,39 @@
 // CWAC-fused quantized linear layer (Section 3.4, Eq. 6-11 with zero-points 0) for sm_100a.
 //
-// One persistent, warp-specialised kernel:
+// One persistent, warp-specialised kernel; CTA c takes the 128 x BN output tiles c, c + G, c + 2G, ...
+// (tiles are numbered strip-major: all column tiles of rows 0-127, then of rows 128-255, ...):
 //   warp 0      TMA producer: per-CTA cp.async.bulk.tensor loads of the X tile [128 x 128 B] and the
-//               W tile [BN x 128 B] into a ring of 128-byte-swizzled shared-memory stages
-//   warp 1      MMA issuer: one thread issues tcgen05.mma kind::i8 (128 x BN x 32 per instruction) into a
-//               TMEM accumulator; tcgen05.commit releases the stage / publishes the accumulator
-//   warp 18     strip coordinator (per-token INT8 output only), see below
-//   warps 19-22 (packed int4 weights only) expand the W tile to int8 in shared memory before the MMA
-//   warps 2-17  epilogue: tcgen05.ld of the INT32 accumulators, z = fma(float(acc) * x_scale[m], fscale[n],
-//               fbias[n]) (the folded M' and offset of Eq. 10-11), then the output stage.  TMEM holds
-//               512 / BN accumulator buffers so the next tile's mainloop overlaps this epilogue.
+//               W tile [BN x 128 B] into a ring of 128-byte-swizzled shared-memory stages.  For short K
+//               the CTA's W tile is loaded once and stays resident; the ring then carries X only.
+//   warp 1      MMA issuer: one thread issues tcgen05.mma kind::i8 (128 x BN x 32 per instruction) into one of
+//               kAcc = 512 / BN TMEM accumulator buffers; tcgen05.commit releases the stage / publishes the buffer
+//   warps 2-17  epilogue: 4 groups of 4 warps.  The work item of a group is a unit = 128 columns of a tile;
+//               the CTA's units are dealt to the groups round-robin (the 512 TMEM columns hold 4 units).
+//               Inside a group the warp's TMEM lane quadrant is warp % 4, so a thread owns ONE ROW of the
+//               unit with its 128 columns.  It reads the INT32 accumulators with
+//               tcgen05.ld (32 columns at a time), forms z = fma(float(acc) * x_scale[m], fscale[n], fbias[n])
+//               (the folded M' and offset of Eq. 10-11, two elements per packed-FP32 instruction), converts,
+//               writes 32-row boxes into swizzled shared memory and hands them to the TMA store unit
+//               (row-contiguous, full-sector writes; rows >= M and columns >= N are clipped by the tensor
+//               map).  The groups run out of phase, so the fixed latencies of one group (waits, proxy fence,
+//               store hand-off) are covered by the arithmetic of the others.
+//   warps 18-21 (packed int4 weights only) expand the W tile to int8 in shared memory before the MMA
 //
 // Per-token INT8 output needs max_n |z[m, n]| over the whole row, but a CTA owns only BN columns of it.
-// Tiles are numbered strip-major (all column tiles of rows 0-127, then of rows 128-255, ...) and CTA c
-// takes tiles c, c + G, c + 2G, ...  An epilogue warp computes z for its 32 x (BN/4) slice, keeps it in
-// registers, releases the TMEM buffer, publishes its per-row maxima with atomicMax on the float bit
-// pattern (non-negative floats order like unsigned integers) and increments its strip's arrival counter;
-// it then waits until the counter shows every slice of the strip and emits the codes with the final row
-// scale.  Progress: take the lowest-numbered tile t that has not published.  Its CTA's epilogue can only
-// be waiting on an earlier tile t - kG, whose strip ends before t whenever tiles_n <= G, so every tile of
-// that strip has published and the wait ends; the mainloop of t needs nothing but TMEM buffers that
-// lower-numbered tiles free without waiting.  The grid is launched cooperatively so all G CTAs are
-// resident.  Every wait is bounded; a wait that gives up records a code in the workspace status word and
-// the CTA tears down normally.
+// The epilogue of a tile therefore has two phases and the accumulators stay in TMEM between them:
+//   phase 1  z from TMEM -> the thread's row maximum over the unit -> atomicMax on rowmax[m] (bit pattern of a
+//            non-negative float orders like an unsigned integer); the group's lead warp then counts the unit
+//            on its strip's counter, and the unit that completes the strip raises the strip's flag;
+//   phase 2  once the flag is up every thread reads its row's final maximum, derives the scale (column tile 0
+//            writes y_scale), re-reads the accumulators, recomputes z, divides, rounds and stores the codes;
+//            only then is the TMEM buffer released.
+// While a group waits for its strip the other groups work on the following tiles.  Progress: phase 1 of
+// tile t needs (a) its group, i.e. phase 2 of tile t - kAcc*G finished, and (b) its accumulator, whose
+// buffer is released by that same phase 2; phase 2 of a tile u needs phase 1 of the tiles of u's strip, all
+// numbered below u + tiles_n <= u + G.  Every dependency of phase 1 of t is thus a phase 1 of a lower-numbered
+// tile, so by induction every phase 1 and then every phase 2 completes, provided all G CTAs are resident:
+// the grid is launched cooperatively with G <= number of SMs and one CTA per SM.  Every wait is bounded; a
+// wait that gives up records a code in the workspace status word and the CTA tears down normally.
 #include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
@@ -42,17 +53,17 @@ constexpr int kBM = 128;           // rows of a CTA tile (= TMEM lanes)
 constexpr int kBK = 128;           // bytes of K per stage: one 128-byte swizzle row
 constexpr int kUmmaK = 32;         // K of one kind::i8 instruction
 constexpr int kTmemCols = 512;
-constexpr int kNumEpilogueWarps = 16;
-constexpr int kCoordWarp = 2 + kNumEpilogueWarps;      // warp that talks to the other CTAs of a row strip
-constexpr int kConvWarp0 = kCoordWarp + 1;              // first of 4 W4 -> INT8 converter warps (packed weights only)
-constexpr int kNumConvWarps = 4;
-constexpr int kThreadsW8 = 32 * (3 + kNumEpilogueWarps);
-constexpr int kThreadsW4 = kThreadsW8 + 32 * kNumConvWarps;
+constexpr int kGroupWarps = 4;        // warps of an epilogue group (one per TMEM lane quadrant)
+constexpr int kGroups = 4;            // epilogue groups; a group works on one 128-column unit of a tile at a time
+constexpr int kUnitN = 128;           // columns of an epilogue unit (512 TMEM columns = 4 units in flight)
+constexpr int kEpiWarps = kGroupWarps * kGroups;
+constexpr int kNumConvWarps = 4;      // W4 -> INT8 converter warps (packed weights only)
 constexpr int kABytes = kBM * kBK;
+constexpr int kSmemBudget = 232448 - 1024;            // opt-in maximum of one CTA minus the slack to align the base
 
 // status word codes (0 = clean)
 enum : uint32_t {
-  kStWaitEmpty = 1, kStWaitFull = 2, kStWaitTmemEmpty = 3, kStWaitTmemFull = 4, kStWaitStrip = 5,
+  kStWaitEmpty = 1, kStWaitFull = 2, kStWaitTmemEmpty = 3, kStWaitTmemFull = 4, kStWaitStrip = 5, kStWaitParam = 6,
 };
 
 struct QlParams {
@@ -63,40 +74,70 @@ struct QlParams {
   float* y_scale;
   int M, N, K;
   int tiles_n, num_tiles, num_kb;
+  int stages;           // depth of the operand ring in shared memory
+  int res_kb;           // > 0: the CTA's W tile (all res_kb k-blocks) stays resident, the ring holds X only
   uint32_t* status;
   uint32_t* rowmax;     // [M] bit patterns of non-negative floats
   uint32_t* counters;   // [tiles_m] tiles of the strip that have published their row maxima
-  uint32_t* flags;      // [tiles_m] set by the last tile of the strip
+  uint32_t* flags;      // [tiles_m] raised by the tile that completes the strip
   uint32_t counter_target;
   unsigned long long timeout_ns;
 };
 
-template <int BN, bool W4>
-struct SmemLayout {
-  static constexpr int kBBytes = BN * kBK;                 // expanded (int8) W tile of one stage
-  static constexpr int kPBytes = W4 ? BN * (kBK / 2) : 0;  // packed (int4) W tile of one stage
-  static constexpr int kStages = W4 ? ((BN == 256) ? 3 : 5) : ((BN == 256) ? 4 : 6);
-  static constexpr int kAcc = kTmemCols / BN;
-  static constexpr int kOffA = 0;
-  static constexpr int kOffB = kOffA + kStages * kABytes;
-  static constexpr int kOffP = kOffB + kStages * kBBytes;
-  static constexpr int kOffFS = kOffP + kStages * kPBytes;         // float [epilogue warp][BN / 4], private per warp
-  static constexpr int kOffFB = kOffFS + kNumEpilogueWarps * (BN / 4) * 4;
-  static constexpr int kOffBars = kOffFB + kNumEpilogueWarps * (BN / 4) * 4;
-  // full[S], empty[S], conv[S], tfull[A], tempty[A], drain, published, strip ready
-  static constexpr int kNumBars = 3 * kStages + 2 * kAcc + 3;
-  static constexpr int kOffMisc = kOffBars + kNumBars * 8;         // tmem base, abort word
-  static constexpr int kTotal = kOffMisc + 16;
-  static constexpr int kDynamic = kTotal + 1024;                   // slack to align the base to 1024
-  static_assert(kDynamic <= 232448, "shared memory budget of one CTA");
+// Compile-time geometry of one instantiation.
+template <int BN, int OUT, bool W4, bool WIDE>
+struct Cfg {
+  static constexpr bool kInt8Out = OUT == QWT_OUT_INT8_PER_TOKEN;
+  static constexpr bool kHasParams = OUT != QWT_OUT_INT32_ACC;       // x_scale / fscale / fbias are used
+  static constexpr int kEsz = kInt8Out ? 1 : (OUT == QWT_OUT_BF16 ? 2 : 4);
+  static constexpr int kAcc = kTmemCols / BN;                        // accumulator buffers (tiles) in TMEM
+  static constexpr int kUPT = BN / kUnitN;                           // epilogue units per tile
+  static constexpr int kConvWarp0 = 2 + kEpiWarps;                   // first converter warp (W4 only)
+  static constexpr int kThreads = 32 * (2 + kEpiWarps + (W4 ? kNumConvWarps : 0));
+  // output staging: one box of 32 rows per epilogue warp, through which a warp turns "thread = row" into
+  // row-contiguous global stores.  128-byte rows for 128-wide tiles; 256-wide tiles use 32-byte rows when the
+  // operand ring needs the room (long K: the epilogue hides behind the mainloop) and 64-byte rows otherwise
+  static constexpr int kBoxBytes = BN == 128 ? 128 : (WIDE ? 64 : 32);
+  static constexpr int kBC = kBoxBytes / kEsz;                       // columns per box
+  static constexpr int kSlotBytes = 32 * kBoxBytes;
+  static constexpr int kStagingBytes = kEpiWarps * kSlotBytes;
+  static constexpr int kBBytes = BN * kBK;                           // expanded (int8) W tile of one stage
+  static constexpr int kPBytes = W4 ? BN * (kBK / 2) : 0;            // packed (int4) W tile of one stage
+  static constexpr int kStageBytes = kABytes + kBBytes + kPBytes;
+  static constexpr int kParamBytes = kGroups * 2 * kUnitN * 4;       // fscale | fbias slice of each group's unit
+  static constexpr int kBarBytes = 512;
+  static constexpr int kFixedBytes = kStagingBytes + kParamBytes + kBarBytes;
+  static constexpr int kMaxStages = 12;
+  // full[S], empty[S], conv[S], tfull[A], tempty[A], pfull[4], pub[4], ready[4], gdone[4], drain, wfull
+  static constexpr int kNumBars = 3 * kMaxStages + 2 * kAcc + 4 * kGroups + 2;
+  static_assert(kNumBars * 8 + 16 <= kBarBytes, "barrier block");
+  // Shared memory, in this order (every block a multiple of 1024 bytes):
+  //   [resident W: res_kb x kBBytes] [X ring: stages x kABytes] [W ring: stages x kBBytes, streaming only]
+  //   [packed W ring, int4 only] [output staging] [fscale|fbias] [barriers]
+  // Streaming: every stage carries an X and a W k-block.  Resident: the CTA's W tile is loaded once.
+  __host__ __device__ static constexpr int stage_bytes(bool resident) { return resident ? kABytes : kStageBytes; }
+  __host__ __device__ static constexpr int stages_for(int res_kb) {
+    const int avail = kSmemBudget - kFixedBytes - res_kb * kBBytes;
+    if (avail <= 0) return 0;
+    const int n = avail / stage_bytes(res_kb > 0);
+    return n > kMaxStages ? kMaxStages : n;
+  }
+  __host__ __device__ static constexpr int ring_bytes(int stages, int res_kb) {
+    return res_kb * kBBytes + stages * stage_bytes(res_kb > 0);
+  }
+  __host__ __device__ static constexpr int dynamic_bytes(int stages, int res_kb) {
+    return ring_bytes(stages, res_kb) + kFixedBytes + 1024;         // slack to align the base to 1024
+  }
+  static_assert(stages_for(0) >= 3, "shared memory budget of one CTA");
 };
 
-__device__ __forceinline__ float epilogue_z(uint32_t acc_bits, float xs, float fs, float fb) {
-  // Eq. 9 after the fold: (S_x acc) * (alpha S_W) + (alpha bias + beta)
-  return fmaf(__fmul_rn(__int2float_rn((int)acc_bits), xs), fs, fb);
+// 16-byte chunk index XOR of the TMA shared-memory swizzle for a dense box whose rows are BOXB bytes long.
+template <int BOXB>
+__device__ __forceinline__ uint32_t swizzle_xor(int row) {
+  return BOXB == 32 ? ((row >> 2) & 1) : (BOXB == 64 ? ((row >> 1) & 3) : (row & 7));
 }
 
-__device__ __forceinline__ void st_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
+__device__ __forceinline__ void st_shared_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
   *reinterpret_cast<uint4*>(p) = make_uint4(a, b, c, d);
 }
 
@@ -105,46 +146,69 @@ __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
   return *reinterpret_cast<uint32_t*>(&v);
 }
 
-template <int BN, int OUT, bool RCP, bool W4>
-__global__ void __launch_bounds__(W4 ? kThreadsW4 : kThreadsW8, 1)
+// Eq. 9 after the fold for two neighbouring columns: (S_x acc) * (alpha S_W) + (alpha bias + beta)
+__device__ __forceinline__ float2 z_pair(uint32_t a0, uint32_t a1, float2 xs2, float f0, float f1, float b0,
+                                         float b1) {
+  const float2 a = make_float2(__int2float_rn((int)a0), __int2float_rn((int)a1));
+  return __ffma2_rn(__fmul2_rn(a, xs2), make_float2(f0, f1), make_float2(b0, b1));
+}
+
+template <int BN, int OUT, bool W4, bool WIDE>
+__global__ void __launch_bounds__((Cfg<BN, OUT, W4, WIDE>::kThreads), 1)
 qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const QlParams p) {
-  using L = SmemLayout<BN, W4>;
+  using C = Cfg<BN, OUT, W4, WIDE>;
+  constexpr int kAcc = C::kAcc;
+  constexpr int kMaxStages = C::kMaxStages;
+  const int stages = p.stages;
+  const bool resident = p.res_kb > 0;      // the CTA's W tile is loaded once; the ring carries X only
   extern __shared__ uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~uintptr_t(1023));
-  uint8_t* sA = smem + L::kOffA;
-  uint8_t* sB = smem + L::kOffB;
-  uint8_t* sP = smem + L::kOffP;     // packed int4 tiles (W4 only)
-  float* sFS = reinterpret_cast<float*>(smem + L::kOffFS);
-  float* sFB = reinterpret_cast<float*>(smem + L::kOffFB);
-  uint64_t* full = reinterpret_cast<uint64_t*>(smem + L::kOffBars);
-  uint64_t* empty = full + L::kStages;
-  uint64_t* conv = empty + L::kStages;     // W4 only: the stage's W tile has been expanded to int8
-  uint64_t* tfull = conv + L::kStages;
-  uint64_t* tempty = tfull + L::kAcc;
-  uint64_t* drain = tempty + L::kAcc;
-  uint64_t* pub_bar = drain + 1;     // 16 arrivals: every epilogue warp has issued its atomicMax
-  uint64_t* ready_bar = drain + 2;   // 1 arrival: the strip's row maxima are final
-  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::kOffMisc);
-  volatile int* cta_abort = reinterpret_cast<volatile int*>(smem + L::kOffMisc + 4);
+  uint8_t* sWres = smem;                                               // [res_kb][BN x 128 B]
+  uint8_t* sA = sWres + p.res_kb * C::kBBytes;                         // [stages][128 x 128 B]
+  uint8_t* sB = sA + stages * kABytes;                                 // [stages][BN x 128 B] (streaming)
+  uint8_t* sP = sB + (resident ? 0 : stages * C::kBBytes);             // [stages][BN x 64 B] packed int4 (W4 only)
+  uint8_t* sStage = smem + C::ring_bytes(stages, p.res_kb);
+  float* sParam = reinterpret_cast<float*>(sStage + C::kStagingBytes);      // [group][fscale 128 | fbias 128]
+  uint8_t* sBars = sStage + C::kStagingBytes + C::kParamBytes;
+  uint64_t* full = reinterpret_cast<uint64_t*>(sBars);
+  uint64_t* empty = full + kMaxStages;
+  uint64_t* conv = empty + kMaxStages;   // W4 only: the stage's W tile has been expanded to int8
+  uint64_t* tfull = conv + kMaxStages;   // accumulator buffer complete (MMA -> epilogue)
+  uint64_t* tempty = tfull + kAcc;       // accumulator buffer free (every warp that read it -> MMA)
+  uint64_t* pfull = tempty + kAcc;       // per group: fscale / fbias slice of its unit is in shared memory (lead warp)
+  uint64_t* pub = pfull + kGroups;       // per group: its 4 warps have issued the unit's row maxima
+  uint64_t* ready = pub + kGroups;       // per group: the strip's row maxima are final
+  uint64_t* gdone = ready + kGroups;     // per group: its 4 warps have finished the unit (parameter slice reusable)
+  uint64_t* drain = gdone + kGroups;
+  uint64_t* wfull = drain + 1;           // resident W tile has landed
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(sBars + C::kBarBytes - 16);
+  volatile int* cta_abort = reinterpret_cast<volatile int*>(sBars + C::kBarBytes - 12);
 
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint64_t tmo = p.timeout_ns;
+  const int G = (int)gridDim.x;
+  const int n_local = (p.num_tiles - (int)blockIdx.x + G - 1) / G;    // tiles of this CTA
 
   if (threadIdx.x == 0) {
-    for (int i = 0; i < L::kStages; ++i) {
+    for (int i = 0; i < stages; ++i) {
       ptx::mbar_init(&full[i], 1);
       ptx::mbar_init(&empty[i], 1);
       ptx::mbar_init(&conv[i], kNumConvWarps);
     }
-    for (int i = 0; i < L::kAcc; ++i) {
+    for (int i = 0; i < kAcc; ++i) {
       ptx::mbar_init(&tfull[i], 1);
-      ptx::mbar_init(&tempty[i], kNumEpilogueWarps);
+      ptx::mbar_init(&tempty[i], kGroupWarps * C::kUPT);
+    }
+    for (int i = 0; i < kGroups; ++i) {
+      ptx::mbar_init(&pfull[i], 1);
+      ptx::mbar_init(&pub[i], kGroupWarps);
+      ptx::mbar_init(&ready[i], 1);
+      ptx::mbar_init(&gdone[i], kGroupWarps);
     }
     ptx::mbar_init(drain, 1);
-    ptx::mbar_init(pub_bar, kNumEpilogueWarps);
-    ptx::mbar_init(ready_bar, 1);
+    ptx::mbar_init(wfull, 1);
     *cta_abort = 0;
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmA);
@@ -159,6 +223,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
+  // Without the INT8 exchange nothing else in the workspace is used: the first CTA clears the status word
+  // (a wait can only give up seconds later).
+  if (!C::kInt8Out && blockIdx.x == 0 && threadIdx.x == 0) *p.status = 0u;
+
   auto give_up = [&](uint32_t code) {
     *cta_abort = 1;
     atomicCAS(p.status, 0u, code);
@@ -167,30 +235,53 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
-      uint32_t kbi = 0;
+      if (resident) {
+        // With a grid that is a multiple of tiles_n every tile of this CTA has the same column tile: its W
+        // tile is loaded once and the ring below streams X only (half the bytes per tile through the SM's
+        // load port, which is what bounds short-K layers).
+        const int n0 = ((int)blockIdx.x % p.tiles_n) * BN;
+        ptx::mbar_arrive_expect_tx(wfull, (uint32_t)(p.res_kb * C::kBBytes));
+        for (int kb = 0; kb < p.res_kb; ++kb) ptx::tma_load_2d(sWres + kb * C::kBBytes, &tmB, kb * kBK, n0, wfull);
+      }
+      uint32_t issued = 0, s = 0, ph = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
+      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += G) {
         const int m0 = (tile / p.tiles_n) * kBM;
         const int n0 = (tile % p.tiles_n) * BN;
-        for (int kb = 0; kb < p.num_kb; ++kb, ++kbi) {
-          const uint32_t s = kbi % L::kStages;
-          if (!ptx::mbar_wait_bounded(&empty[s], ((kbi / L::kStages) & 1u) ^ 1u, cta_abort, tmo)) {
+        for (int kb = 0; kb < p.num_kb; ++kb, ++issued) {
+          if (!ptx::mbar_wait_bounded(&empty[s], ph ^ 1u, cta_abort, tmo)) {
             give_up(kStWaitEmpty);
             ok = false;
             break;
           }
-          ptx::mbar_arrive_expect_tx(&full[s], kABytes + (W4 ? L::kPBytes : L::kBBytes));
-          ptx::tma_load_2d(sA + s * kABytes, &tmA, kb * kBK, m0, &full[s]);
-          if (W4) ptx::tma_load_2d(sP + s * L::kPBytes, &tmB, kb * (kBK / 2), n0, &full[s]);
-          else ptx::tma_load_2d(sB + s * L::kBBytes, &tmB, kb * kBK, n0, &full[s]);
+          if (resident) {
+            ptx::mbar_arrive_expect_tx(&full[s], kABytes);
+            ptx::tma_load_2d(sA + s * kABytes, &tmA, kb * kBK, m0, &full[s]);
+          } else {
+            ptx::mbar_arrive_expect_tx(&full[s], kABytes + (W4 ? C::kPBytes : C::kBBytes));
+            ptx::tma_load_2d(sA + s * kABytes, &tmA, kb * kBK, m0, &full[s]);
+            if (W4) ptx::tma_load_2d(sP + s * C::kPBytes, &tmB, kb * (kBK / 2), n0, &full[s]);
+            else ptx::tma_load_2d(sB + s * C::kBBytes, &tmB, kb * kBK, n0, &full[s]);
+          }
+          if (++s == (uint32_t)stages) {
+            s = 0;
+            ph ^= 1u;
+          }
         }
       }
       if (*cta_abort != 0) {
         // let copies still in flight land before the CTA's shared memory is released
-        const uint32_t first = kbi > (uint32_t)L::kStages ? kbi - L::kStages : 0u;
-        for (uint32_t j = first; j < kbi; ++j) {
+        const uint32_t back = issued < (uint32_t)stages ? issued : (uint32_t)stages;
+        for (uint32_t j = 0; j < back; ++j) {
+          // walk back over the last `back` issues: stage and phase of issue number issued - 1 - j
+          const uint32_t n = issued - 1 - j;
           uint32_t polls = 0;
-          while (!ptx::mbar_try_wait(&full[j % L::kStages], (j / L::kStages) & 1u) && ++polls < (1u << 16)) {
+          while (!ptx::mbar_try_wait(&full[n % stages], (n / stages) & 1u) && ++polls < (1u << 16)) {
+          }
+        }
+        if (resident) {
+          uint32_t polls = 0;
+          while (!ptx::mbar_try_wait(wfull, 0) && ++polls < (1u << 16)) {
           }
         }
       }
@@ -199,33 +290,40 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
       constexpr uint32_t idesc = ptx::make_idesc_i8(kBM, BN);
-      const uint32_t a_base = ptx::smem_u32(sA), b_base = ptx::smem_u32(sB);
-      uint32_t kbi = 0, it = 0;
+      const uint32_t a_base = ptx::smem_u32(sA), b_base = ptx::smem_u32(sB), w_base = ptx::smem_u32(sWres);
+      uint32_t s = 0, ph = 0, it = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x, ++it) {
-        const uint32_t buf = it % L::kAcc;
-        if (!ptx::mbar_wait_bounded(&tempty[buf], ((it / L::kAcc) & 1u) ^ 1u, cta_abort, tmo)) {
+      if (resident && !ptx::mbar_wait_bounded(wfull, 0, cta_abort, tmo)) {
+        give_up(kStWaitFull);
+        ok = false;
+      }
+      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += G, ++it) {
+        const uint32_t buf = it % kAcc;
+        if (!ptx::mbar_wait_bounded(&tempty[buf], ((it / kAcc) & 1u) ^ 1u, cta_abort, tmo)) {
           give_up(kStWaitTmemEmpty);
           break;
         }
         ptx::tc_fence_after();
         const uint32_t d_tmem = tmem_base + buf * BN;
-        for (int kb = 0; kb < p.num_kb; ++kb, ++kbi) {
-          const uint32_t s = kbi % L::kStages;
-          if (!ptx::mbar_wait_bounded(W4 ? &conv[s] : &full[s], (kbi / L::kStages) & 1u, cta_abort, tmo)) {
+        for (int kb = 0; kb < p.num_kb; ++kb) {
+          if (!ptx::mbar_wait_bounded(W4 ? &conv[s] : &full[s], ph, cta_abort, tmo)) {
             give_up(kStWaitFull);
             ok = false;
             break;
           }
           ptx::tc_fence_after();
           const uint64_t a_desc = ptx::make_kmajor_sw128_desc(a_base + s * kABytes);
-          const uint64_t b_desc = ptx::make_kmajor_sw128_desc(b_base + s * L::kBBytes);
+          const uint64_t b_desc = ptx::make_kmajor_sw128_desc(resident ? w_base + kb * C::kBBytes : b_base + s * C::kBBytes);
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             // next 32 bytes of K inside the swizzled 128-byte row: start address + 32 B (>> 4 = 2)
             ptx::mma_i8_ss(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
           }
           ptx::tc_commit(&empty[s]);
+          if (++s == (uint32_t)stages) {
+            s = 0;
+            ph ^= 1u;
+          }
         }
         if (ok) ptx::tc_commit(&tfull[buf]);
       }
@@ -237,25 +335,24 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       }
     }
-  } else if (W4 && warp >= kConvWarp0) {
+  } else if (W4 && warp >= C::kConvWarp0) {
     // ------------------------------------------------------------------ W4 -> INT8 converter warps
     // The packed tile (64 bytes per row, two's-complement nibbles, even element low) is expanded into the
     // 128-byte-swizzled operand tile the MMA descriptor expects.  Each nibble is moved to the HIGH half of
     // its byte, i.e. the operand holds 16 x code (|16 code| <= 112 fits int8); the factor 1/16 is exact in
     // the epilogue (fscale / 16, or an arithmetic shift of the raw accumulators).
-    const int ct = threadIdx.x - kConvWarp0 * 32;          // 0..127
-    uint32_t kbi = 0;
+    const int ct = threadIdx.x - C::kConvWarp0 * 32;       // 0..127
+    uint32_t s = 0, ph = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += gridDim.x) {
-      for (int kb = 0; kb < p.num_kb; ++kb, ++kbi) {
-        const uint32_t s = kbi % L::kStages;
-        if (!ptx::mbar_wait_bounded(&full[s], (kbi / L::kStages) & 1u, cta_abort, tmo)) {
+    for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += G) {
+      for (int kb = 0; kb < p.num_kb; ++kb) {
+        if (!ptx::mbar_wait_bounded(&full[s], ph, cta_abort, tmo)) {
           give_up(kStWaitFull);
           ok = false;
           break;
         }
-        const uint8_t* src = sP + s * L::kPBytes;
-        uint8_t* dst = sB + s * L::kBBytes;
+        const uint8_t* src = sP + s * C::kPBytes;
+        uint8_t* dst = sB + s * C::kBBytes;
 #pragma unroll 2
         for (int q = ct; q < BN * 4; q += 32 * kNumConvWarps) {
           const int n = q >> 2, c = q & 3;                 // row of the tile, 16-byte chunk of the packed row
@@ -277,201 +374,266 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         ptx::fence_proxy_async_smem();     // generic-proxy writes -> visible to the tensor core's async proxy
         __syncwarp();
         if (lane == 0) ptx::mbar_arrive(&conv[s]);
-      }
-    }
-  } else if (warp == kCoordWarp) {
-    // ------------------------------------------------------------------ strip coordinator (INT8 output only)
-    // One thread per CTA speaks for the tile: once the 16 epilogue warps have issued their row maxima it
-    // counts the tile as published; the last tile of a strip raises the strip's flag, the others poll the
-    // flag (a different word than the counter, with a back-off, so that arrivals are not queued behind
-    // polls) and then release the epilogue warps.
-    if (OUT == QWT_OUT_INT8_PER_TOKEN && lane == 0) {
-      uint32_t it = 0;
-      for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++it) {
-        const int tm = tile / p.tiles_n;
-        if (!ptx::mbar_wait_bounded(pub_bar, it & 1u, cta_abort, tmo)) {
-          give_up(kStWaitStrip);
-          break;
+        if (++s == (uint32_t)stages) {
+          s = 0;
+          ph ^= 1u;
         }
-        __threadfence();     // the warps' atomicMax (seen through the barrier) before the count
-        const uint32_t old = atomicAdd(p.counters + tm, 1u);
-        if (old + 1u == p.counter_target) {
-          __threadfence();
-          ptx::st_release_gpu(p.flags + tm, 1u);
-        } else {
-          uint32_t polls = 0;
-          uint64_t t0 = 0;
-          bool failed = false;
-          while (ptx::ld_acquire_gpu(p.flags + tm) == 0u) {
-            __nanosleep(64);
-            if ((++polls & 63u) == 0u) {
-              const uint64_t now = ptx::globaltimer_ns();
-              if (t0 == 0) t0 = now;
-              if (*cta_abort != 0 || now - t0 > tmo || ptx::ld_acquire_gpu(p.status) != 0u) {
-                failed = true;
-                break;
-              }
-            }
-          }
-          if (failed) {
-            give_up(kStWaitStrip);
-            break;
-          }
-        }
-        __threadfence();
-        ptx::mbar_arrive(ready_bar);
       }
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps
-    // 16 warps: TMEM lane quadrant = warp % 4 (hardware rule), column group = (warp - 2) / 4.
-    // A warp owns 32 rows x CW columns of the tile; a thread owns one row of that.
-    constexpr int CW = BN / (kNumEpilogueWarps / 4);
-    const int qd = warp & 3;
-    const int cg = (warp - 2) >> 2;
-    // each warp stages its slice of fscale / fbias privately (no cross-warp barrier to get stuck on)
-    float* fs = sFS + (warp - 2) * CW;
-    float* fb = sFB + (warp - 2) * CW;
-    uint32_t it = 0;
-    for (int tile = blockIdx.x; tile < p.num_tiles; tile += gridDim.x, ++it) {
-      const uint32_t buf = it % L::kAcc;
-      const int tm = tile / p.tiles_n, tn = tile % p.tiles_n;
-      const int m0 = tm * kBM;
-      const int n0 = tn * BN + cg * CW;          // first column of this warp's slice
-      __syncwarp();   // every lane is done with the previous tile's slice
-      if (OUT != QWT_OUT_INT32_ACC) {
-        for (int i = lane; i < CW; i += 32) {
-          const int c = n0 + i;
-          fs[i] = c < p.N ? __ldg(p.fscale + c) * (W4 ? 0.0625f : 1.0f) : 0.f;   // W4 operands hold 16 x code
-          fb[i] = c < p.N ? __ldg(p.fbias + c) : 0.f;
+    // Work item = one unit: 128 columns of a tile.  The CTA's units are numbered u = j * kUPT + half
+    // (j = local tile); group g takes u = g, g + 4, ...  Unit u lives in TMEM columns (u % 4) * 128.
+    constexpr int UPT = C::kUPT;
+    constexpr int NC = 32;                  // columns per tcgen05.ld
+    constexpr int BOXB = C::kBoxBytes;
+    constexpr int BC = C::kBC;              // columns per staging box
+    constexpr int ESZ = C::kEsz;
+    const int ew = warp - 2;
+    const int g = ew / kGroupWarps;
+    const int qd = warp & 3;                // TMEM lane quadrant (hardware rule: warp % 4)
+    const bool lead = qd == 0;              // stages fscale / fbias and speaks for the group to the other CTAs
+    uint8_t* stg = sStage + ew * C::kSlotBytes;
+    const uint32_t swz = swizzle_xor<BOXB>(lane);
+    float* const ps_fs = sParam + g * 2 * kUnitN;   // this group's fscale slice, then its fbias slice
+    float* const ps_fb = ps_fs + kUnitN;
+    const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + g * kUnitN;
+    const int n_units = n_local * UPT;
+    float pre_fs[kUnitN / 32], pre_fb[kUnitN / 32];
+
+    auto unit_col0 = [&](int u) {           // first column of unit u in the output matrix
+      const int tile = (int)blockIdx.x + (u / UPT) * G;
+      return (tile % p.tiles_n) * BN + (u % UPT) * kUnitN;
+    };
+    auto prefetch_params = [&](int u) {
+      const int n0 = unit_col0(u);
+#pragma unroll
+      for (int i = 0; i < kUnitN / 32; ++i) {
+        const int c = n0 + i * 32 + lane;
+        pre_fs[i] = c < p.N ? __ldg(p.fscale + c) * (W4 ? 0.0625f : 1.0f) : 0.f;   // W4 operands hold 16 x code
+        pre_fb[i] = c < p.N ? __ldg(p.fbias + c) : 0.f;
+      }
+    };
+    if (C::kHasParams && lead && g < n_units) prefetch_params(g);
+
+    // Writes the warp's box (32 rows x BOXB bytes, swizzled in its staging slot) to global memory: lanes are
+    // re-dealt so that one store instruction covers whole box rows (BOXB contiguous bytes each).
+    // x_bytes / y = position of the box in the output matrix, in bytes / rows.
+    auto store_box = [&](int x_bytes, int y) {
+      constexpr int CPR = BOXB / 16;                 // 16-byte chunks per box row
+      constexpr int RPI = 32 / CPR;                  // rows per store instruction
+      __syncwarp();
+      const int chunk = lane % CPR;
+      const int xb = x_bytes + chunk * 16;
+      const bool col_ok = xb < p.N * ESZ;            // N * ESZ is a multiple of 16: a chunk is all in or all out
+      uint8_t* out = static_cast<uint8_t*>(p.Y) + xb;
+#pragma unroll
+      for (int i = 0; i < CPR; ++i) {
+        const int r = i * RPI + lane / CPR;
+        const uint4 v = *reinterpret_cast<const uint4*>(stg + r * BOXB + ((chunk ^ swizzle_xor<BOXB>(r)) << 4));
+        if (col_ok && y + r < p.M) *reinterpret_cast<uint4*>(out + (size_t)(y + r) * p.N * ESZ) = v;
+      }
+      __syncwarp();                                  // the slot may be rewritten
+    };
+
+    int use = 0;                            // units this group has handled
+    for (int u = g; u < n_units; u += kGroups, ++use) {
+      const int j = u / UPT;
+      const int tile = (int)blockIdx.x + j * G;
+      const int tm = tile / p.tiles_n;
+      const int n0 = unit_col0(u);
+      const uint32_t buf = j % kAcc, tpar = (j / kAcc) & 1u, upar = use & 1u;
+      const int row = tm * kBM + qd * 32 + lane;
+      const int y0 = tm * kBM + qd * 32;
+      float xs = 0.f;
+      if (C::kHasParams && row < p.M) xs = __ldg(p.x_scale + row);     // issued before the waits below
+      bool ok = true;
+      if (C::kHasParams) {
+        if (lead) {
+          // the slice is free once the group's 4 warps have finished the unit that used it before
+          if (!ptx::mbar_wait_bounded(&gdone[g], upar ^ 1u, cta_abort, tmo)) {
+            give_up(kStWaitParam);
+            break;
+          }
+#pragma unroll
+          for (int i = 0; i < kUnitN / 32; ++i) {
+            ps_fs[i * 32 + lane] = pre_fs[i];
+            ps_fb[i * 32 + lane] = pre_fb[i];
+          }
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&pfull[g]);
+          if (u + kGroups < n_units) prefetch_params(u + kGroups);
+        }
+        if (!ptx::mbar_wait_bounded(&pfull[g], upar, cta_abort, tmo)) {
+          give_up(kStWaitParam);
+          break;
         }
       }
-      __syncwarp();
-      const int row = m0 + qd * 32 + lane;
-      const bool row_ok = row < p.M;
-      float xs = 0.f;
-      if (OUT != QWT_OUT_INT32_ACC && row_ok) xs = __ldg(p.x_scale + row);
-
-      if (!ptx::mbar_wait_bounded(&tfull[buf], (it / L::kAcc) & 1u, cta_abort, tmo)) {
+      if (!ptx::mbar_wait_bounded(&tfull[buf], tpar, cta_abort, tmo)) {
         give_up(kStWaitTmemFull);
         break;
       }
       ptx::tc_fence_after();
-      const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + buf * BN + cg * CW;
+      const float2 xs2 = make_float2(xs, xs);
+      const bool in_range = n0 < p.N;        // a unit entirely right of the matrix has nothing to compute or store
 
-      if (OUT == QWT_OUT_INT8_PER_TOKEN) {
-        // z of the whole slice stays in registers; the accumulator buffer is released before the wait
-        float z[CW];
+      float den = 1.f, inv = 1.f;
+      bool slow = false;
+      if (C::kInt8Out && in_range) {
+        // ---------------------------------------------------------------- phase 1: row maxima of the unit
         float amax = 0.f;
-#pragma unroll
-        for (int h = 0; h < CW / 32; ++h) {
-          uint32_t r[32];
-          ptx::tmem_ld_32x32b_x32(taddr + h * 32, r);
+#pragma unroll 1
+        for (int h = 0; h < kUnitN / NC; ++h) {
+          uint32_t r[NC];
+          ptx::tmem_ld_32x32b_x32(taddr + h * NC, r);
           ptx::tmem_ld_wait();
 #pragma unroll
-          for (int j = 0; j < 32; j += 4) {
-            const float4 f4 = *reinterpret_cast<const float4*>(fs + h * 32 + j);
-            const float4 b4 = *reinterpret_cast<const float4*>(fb + h * 32 + j);
-            z[h * 32 + j + 0] = epilogue_z(r[j + 0], xs, f4.x, b4.x);   // columns >= N give 0 * 0 + 0
-            z[h * 32 + j + 1] = epilogue_z(r[j + 1], xs, f4.y, b4.y);
-            z[h * 32 + j + 2] = epilogue_z(r[j + 2], xs, f4.z, b4.z);
-            z[h * 32 + j + 3] = epilogue_z(r[j + 3], xs, f4.w, b4.w);
-            amax = fmaxf(fmaxf(amax, fmaxf(fabsf(z[h * 32 + j]), fabsf(z[h * 32 + j + 1]))),
-                         fmaxf(fabsf(z[h * 32 + j + 2]), fabsf(z[h * 32 + j + 3])));
+          for (int e = 0; e < NC; e += 4) {
+            const float4 f4 = *reinterpret_cast<const float4*>(ps_fs + h * NC + e);
+            const float4 b4 = *reinterpret_cast<const float4*>(ps_fb + h * NC + e);
+            const float2 z01 = z_pair(r[e], r[e + 1], xs2, f4.x, f4.y, b4.x, b4.y);   // columns >= N give 0 * 0 + 0
+            const float2 z23 = z_pair(r[e + 2], r[e + 3], xs2, f4.z, f4.w, b4.z, b4.w);
+            amax = fmaxf(fmaxf(amax, fmaxf(fabsf(z01.x), fabsf(z01.y))), fmaxf(fabsf(z23.x), fabsf(z23.y)));
           }
         }
-        ptx::tc_fence_before();
+        if (row < p.M) atomicMax(p.rowmax + row, __float_as_uint(amax));
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&tempty[buf]);
-
-        if (row_ok) atomicMax(p.rowmax + row, __float_as_uint(amax));
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(pub_bar);
-        // the coordinator warp publishes the tile and waits for the rest of the strip
-        if (!ptx::mbar_wait_bounded(ready_bar, it & 1u, cta_abort, tmo)) {
+        if (lane == 0) {
+          __threadfence();                  // this warp's maxima before the arrival below
+          ptx::mbar_arrive(&pub[g]);
+        }
+        if (lead) {
+          // the lead warp counts the unit once the whole group has published, then waits for the strip
+          if (lane == 0) {
+            int good = ptx::mbar_wait_bounded(&pub[g], upar, cta_abort, tmo) ? 1 : 0;
+            if (good) {
+              __threadfence();
+              const uint32_t old = atomicAdd(p.counters + tm, 1u);
+              if (old + 1u == p.counter_target) {
+                __threadfence();
+                ptx::st_release_gpu(p.flags + tm, 1u);
+              } else {
+                uint32_t polls = 0;
+                uint64_t t0 = 0;
+                while (ptx::ld_acquire_gpu(p.flags + tm) == 0u) {
+                  __nanosleep(32);
+                  if ((++polls & 63u) == 0u) {
+                    const uint64_t now = ptx::globaltimer_ns();
+                    if (t0 == 0) t0 = now;
+                    if (*cta_abort != 0 || now - t0 > tmo || ptx::ld_acquire_gpu(p.status) != 0u) {
+                      good = 0;
+                      break;
+                    }
+                  }
+                }
+              }
+              __threadfence();
+            }
+            if (good) ptx::mbar_arrive(&ready[g]);
+            else give_up(kStWaitStrip);
+          }
+          __syncwarp();     // the other lanes wait here, not in a spin loop beside lane 0
+        }
+        if (!ptx::mbar_wait_bounded(&ready[g], upar, cta_abort, tmo)) {
           give_up(kStWaitStrip);
           break;
         }
-        float ys = 0.f;
-        if (row_ok) {
-          ys = __fdiv_rn(__uint_as_float(__ldcg(p.rowmax + row)), 127.f);
-          if (tn == 0 && cg == 0) p.y_scale[row] = ys;
-        }
-        const float den = ys > 0.f ? ys : 1.f;       // a zero row has z == 0 everywhere: codes 0
-        const float inv = __fdiv_rn(1.f, den);
-        int8_t* yrow = static_cast<int8_t*>(p.Y) + (size_t)row * p.N + n0;
-#pragma unroll
-        for (int g = 0; g < CW / 16; ++g) {
-          uint32_t w[4];
-#pragma unroll
-          for (int t = 0; t < 4; ++t) {
-            int q[4];
-#pragma unroll
-            for (int j = 0; j < 4; ++j) {
-              const float zz = z[g * 16 + t * 4 + j];
-              q[j] = __float2int_rn(RCP ? __fmul_rn(zz, inv) : __fdiv_rn(zz, den));   // |q| <= 127 by construction
-            }
-            const uint32_t lo = __byte_perm((uint32_t)q[0], (uint32_t)q[1], 0x0040);
-            const uint32_t hi = __byte_perm((uint32_t)q[2], (uint32_t)q[3], 0x0040);
-            w[t] = __byte_perm(lo, hi, 0x5410);
-          }
-          if (row_ok && n0 + g * 16 + 16 <= p.N) st_v4(yrow + g * 16, w[0], w[1], w[2], w[3]);
-        }
-      } else {
-#pragma unroll
-        for (int h = 0; h < CW / 32; ++h) {
-          uint32_t r[32];
-          ptx::tmem_ld_32x32b_x32(taddr + h * 32, r);
-          ptx::tmem_ld_wait();
-          const int c0 = n0 + h * 32;
-          if (OUT == QWT_OUT_INT32_ACC) {
-            if (W4) {
-#pragma unroll
-              for (int j = 0; j < 32; ++j) r[j] = (uint32_t)((int)r[j] >> 4);   // exact: every term is a multiple of 16
-            }
-            if (row_ok) {
-              int32_t* yrow = static_cast<int32_t*>(p.Y) + (size_t)row * p.N + c0;
-#pragma unroll
-              for (int g = 0; g < 8; ++g)
-                if (c0 + g * 4 + 4 <= p.N) st_v4(yrow + g * 4, r[g * 4], r[g * 4 + 1], r[g * 4 + 2], r[g * 4 + 3]);
-            }
-          } else {
-            float z[32];
-#pragma unroll
-            for (int j = 0; j < 32; j += 4) {
-              const float4 f4 = *reinterpret_cast<const float4*>(fs + h * 32 + j);
-              const float4 b4 = *reinterpret_cast<const float4*>(fb + h * 32 + j);
-              z[j + 0] = epilogue_z(r[j + 0], xs, f4.x, b4.x);
-              z[j + 1] = epilogue_z(r[j + 1], xs, f4.y, b4.y);
-              z[j + 2] = epilogue_z(r[j + 2], xs, f4.z, b4.z);
-              z[j + 3] = epilogue_z(r[j + 3], xs, f4.w, b4.w);
-            }
-            if (OUT == QWT_OUT_FP32) {
-              if (row_ok) {
-                float* yrow = static_cast<float*>(p.Y) + (size_t)row * p.N + c0;
-#pragma unroll
-                for (int g = 0; g < 8; ++g)
-                  if (c0 + g * 4 + 4 <= p.N)
-                    st_v4(yrow + g * 4, __float_as_uint(z[g * 4]), __float_as_uint(z[g * 4 + 1]),
-                          __float_as_uint(z[g * 4 + 2]), __float_as_uint(z[g * 4 + 3]));
-              }
-            } else {  // BF16
-              if (row_ok) {
-                __nv_bfloat16* yrow = static_cast<__nv_bfloat16*>(p.Y) + (size_t)row * p.N + c0;
-#pragma unroll
-                for (int g = 0; g < 4; ++g)
-                  if (c0 + g * 8 + 8 <= p.N)
-                    st_v4(yrow + g * 8, pack_bf16x2(z[g * 8], z[g * 8 + 1]), pack_bf16x2(z[g * 8 + 2], z[g * 8 + 3]),
-                          pack_bf16x2(z[g * 8 + 4], z[g * 8 + 5]), pack_bf16x2(z[g * 8 + 6], z[g * 8 + 7]));
-              }
-            }
-          }
-        }
-        // accumulator buffer is free again
-        ptx::tc_fence_before();
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&tempty[buf]);
+        // ---------------------------------------------------------------- phase 2: scale, codes
+        const float amax_row = row < p.M ? __uint_as_float(__ldcg(p.rowmax + row)) : 0.f;
+        const float ys = __fdiv_rn(amax_row, 127.f);
+        if (n0 == 0 && row < p.M) p.y_scale[row] = ys;
+        den = ys > 0.f ? ys : 1.f;          // a zero row has z == 0 everywhere: codes 0
+        inv = __frcp_rn(den);
+        // a scale so small that its reciprocal overflows (never on real data): divide directly
+        slow = __any_sync(0xffffffffu, !(inv <= 3.0e38f));
       }
+
+      // ------------------------------------------------------------------ conversion and store, box by box
+      if (in_range) {
+        const float2 inv2 = make_float2(inv, inv);
+        const float2 nden2 = make_float2(-den, -den);
+        const float2 magic2 = make_float2(12582912.f, 12582912.f);
+        // z / den rounded to nearest: q0 = z * (1/den), then one residual correction with fused multiply-adds;
+        // adding 1.5 * 2^23 leaves rne(q) in the low mantissa bits (|q| <= 127 by construction)
+        auto quant = [&](float2 z) -> float2 {
+          float2 q;
+          if (slow) {
+            q = make_float2(__fdiv_rn(z.x, den), __fdiv_rn(z.y, den));
+          } else {
+            const float2 q0 = __fmul2_rn(z, inv2);
+            const float2 rem = __ffma2_rn(q0, nden2, z);
+            q = __ffma2_rn(rem, inv2, q0);
+          }
+          return __fadd2_rn(q, magic2);
+        };
+        constexpr int LDC = BC < NC ? BC : NC;       // columns per load inside a box
+#pragma unroll 1
+        for (int bx = 0; bx < kUnitN / BC; ++bx) {
+          if (n0 + bx * BC >= p.N) break;
+          uint8_t* dst = stg + lane * BOXB;
+#pragma unroll 1
+          for (int h = 0; h < BC / LDC; ++h) {
+            const int c0 = bx * BC + h * LDC;         // first column (inside the unit) of this load
+            uint32_t r[LDC];
+            ptx::tmem_ld_cols<LDC>(taddr + c0, r);
+            ptx::tmem_ld_wait();
+            constexpr int EPC = 16 / ESZ;            // elements per 16-byte chunk
+#pragma unroll
+            for (int c = 0; c < LDC / EPC; ++c) {
+              uint32_t w[4];
+              if (OUT == QWT_OUT_INT32_ACC) {
+#pragma unroll
+                for (int t = 0; t < 4; ++t)           // W4: every term is a multiple of 16, the shift is exact
+                  w[t] = W4 ? (uint32_t)((int)r[c * 4 + t] >> 4) : r[c * 4 + t];
+              } else if (OUT == QWT_OUT_FP32) {
+                const int e = c * 4;
+                const float4 f4 = *reinterpret_cast<const float4*>(ps_fs + c0 + e);
+                const float4 b4 = *reinterpret_cast<const float4*>(ps_fb + c0 + e);
+                const float2 z01 = z_pair(r[e], r[e + 1], xs2, f4.x, f4.y, b4.x, b4.y);
+                const float2 z23 = z_pair(r[e + 2], r[e + 3], xs2, f4.z, f4.w, b4.z, b4.w);
+                w[0] = __float_as_uint(z01.x);
+                w[1] = __float_as_uint(z01.y);
+                w[2] = __float_as_uint(z23.x);
+                w[3] = __float_as_uint(z23.y);
+              } else if (OUT == QWT_OUT_BF16) {
+#pragma unroll
+                for (int t = 0; t < 2; ++t) {
+                  const int e = c * 8 + t * 4;
+                  const float4 f4 = *reinterpret_cast<const float4*>(ps_fs + c0 + e);
+                  const float4 b4 = *reinterpret_cast<const float4*>(ps_fb + c0 + e);
+                  const float2 z01 = z_pair(r[e], r[e + 1], xs2, f4.x, f4.y, b4.x, b4.y);
+                  const float2 z23 = z_pair(r[e + 2], r[e + 3], xs2, f4.z, f4.w, b4.z, b4.w);
+                  w[2 * t] = pack_bf16x2(z01.x, z01.y);
+                  w[2 * t + 1] = pack_bf16x2(z23.x, z23.y);
+                }
+              } else {  // INT8 codes
+#pragma unroll
+                for (int t = 0; t < 4; ++t) {
+                  const int e = c * 16 + t * 4;
+                  const float4 f4 = *reinterpret_cast<const float4*>(ps_fs + c0 + e);
+                  const float4 b4 = *reinterpret_cast<const float4*>(ps_fb + c0 + e);
+                  const float2 m01 = quant(z_pair(r[e], r[e + 1], xs2, f4.x, f4.y, b4.x, b4.y));
+                  const float2 m23 = quant(z_pair(r[e + 2], r[e + 3], xs2, f4.z, f4.w, b4.z, b4.w));
+                  const uint32_t lo = __byte_perm(__float_as_uint(m01.x), __float_as_uint(m01.y), 0x0040);
+                  const uint32_t hi = __byte_perm(__float_as_uint(m23.x), __float_as_uint(m23.y), 0x0040);
+                  w[t] = __byte_perm(lo, hi, 0x5410);
+                }
+              }
+              const uint32_t chunk = (uint32_t)(h * (LDC / EPC) + c);     // 16-byte chunk inside the box row
+              st_shared_v4(dst + ((chunk ^ swz) << 4), w[0], w[1], w[2], w[3]);
+            }
+          }
+          store_box((n0 + bx * BC) * ESZ, y0);
+        }
+      }
+      // the accumulator buffer and the group's parameter slice are free again
+      ptx::tc_fence_before();
+      __syncwarp();
+      if (lane == 0) {
+        ptx::mbar_arrive(&tempty[buf]);
+        ptx::mbar_arrive(&gdone[g]);
+      }
+      (void)ok;
     }
   }
 
@@ -532,49 +694,61 @@ unsigned long long timeout_ns_from_env() {
   return v;
 }
 
-// QWT_REQUANT_RECIPROCAL=1 replaces the division z / y_scale by a multiplication with 1 / y_scale
-// (codes may then differ from the division by one step on a few elements per million).
-bool requant_by_reciprocal() {
-  static const bool v = [] {
-    const char* e = getenv("QWT_REQUANT_RECIPROCAL");
-    return e != nullptr && e[0] == '1';
-  }();
-  return v;
-}
-
-template <int BN, int OUT, bool RCP, bool W4>
-qwt_status launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
-                       bool cooperative, cudaStream_t st) {
-  using L = SmemLayout<BN, W4>;
-  constexpr int kThreads = W4 ? kThreadsW4 : kThreadsW8;
-  auto kern = qlinear_cwac_kernel<BN, OUT, RCP, W4>;
-  // per device and cheap, so it is simply set on every launch
-  QWT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::kDynamic));
-  if (cooperative) {
+template <int BN, int OUT, bool W4, bool WIDE>
+qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams prm, int grid, int res_kb,
+                      cudaStream_t st) {
+  using C = Cfg<BN, OUT, W4, WIDE>;
+  constexpr int kThreads = C::kThreads;
+  auto kern = qlinear_cwac_kernel<BN, OUT, W4, WIDE>;
+  prm.res_kb = res_kb;
+  prm.stages = C::stages_for(res_kb);
+  const int smem_bytes = C::dynamic_bytes(prm.stages, res_kb);
+  // the opt-in shared-memory size is a per-device attribute of the function: set once per device
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  QWT_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    QWT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  if (C::kInt8Out) {
+    // the row-maximum exchange needs every CTA of the grid resident
     void* args[] = {(void*)&tmA, (void*)&tmB, (void*)&prm};
-    QWT_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, L::kDynamic, st));
+    QWT_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, smem_bytes, st));
     count_launch();
   } else {
-    kern<<<grid, kThreads, L::kDynamic, st>>>(tmA, tmB, prm);
+    kern<<<grid, kThreads, smem_bytes, st>>>(tmA, tmB, prm);
     QWT_LAUNCH_CHECK();
   }
   return QWT_OK;
 }
 
+// Operand ring: the resident-W layout (with the wider output staging that short-K layers want) when the plan
+// asks for it and at least 4 X stages remain, else the streaming layout.
+template <int BN, int OUT, bool W4>
+qwt_status launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
+                       bool want_resident, cudaStream_t st) {
+  if (!W4) {
+    constexpr bool kWide = BN == 256;
+    using CW = Cfg<BN, OUT, false, kWide>;
+    if (want_resident && CW::stages_for(prm.num_kb) >= 4)
+      return launch_cfg<BN, OUT, false, kWide>(tmA, tmB, prm, grid, prm.num_kb, st);
+  }
+  return launch_cfg<BN, OUT, W4, false>(tmA, tmB, prm, grid, 0, st);
+}
+
 template <int BN, bool W4>
 qwt_status launch_bn(int out_mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
-                     cudaStream_t st) {
+                     bool want_resident, cudaStream_t st) {
   switch (out_mode) {
     case QWT_OUT_INT8_PER_TOKEN:
-      if (requant_by_reciprocal())
-        return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN, true, W4>(tmA, tmB, prm, grid, true, st);
-      return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN, false, W4>(tmA, tmB, prm, grid, true, st);
+      return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN, W4>(tmA, tmB, prm, grid, want_resident, st);
     case QWT_OUT_BF16:
-      return launch_inst<BN, QWT_OUT_BF16, false, W4>(tmA, tmB, prm, grid, false, st);
+      return launch_inst<BN, QWT_OUT_BF16, W4>(tmA, tmB, prm, grid, want_resident, st);
     case QWT_OUT_FP32:
-      return launch_inst<BN, QWT_OUT_FP32, false, W4>(tmA, tmB, prm, grid, false, st);
+      return launch_inst<BN, QWT_OUT_FP32, W4>(tmA, tmB, prm, grid, want_resident, st);
     case QWT_OUT_INT32_ACC:
-      return launch_inst<BN, QWT_OUT_INT32_ACC, false, W4>(tmA, tmB, prm, grid, false, st);
+      return launch_inst<BN, QWT_OUT_INT32_ACC, W4>(tmA, tmB, prm, grid, want_resident, st);
   }
   return QWT_ERR_UNSUPPORTED;
 }
@@ -583,11 +757,11 @@ qwt_status launch_bn(int out_mode, const CUtensorMap& tmA, const CUtensorMap& tm
 
 qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
                         QlinearPlan* plan) {
-  (void)K;
   QlinearPlan pl{};
   pl.tiles_m = (M + kBM - 1) / kBM;
-  // 256-wide tiles keep the tensor pipe ahead of shared-memory bandwidth; 128-wide ones are used when
-  // the wider tile would leave many SMs without work.
+  // 256-wide tiles keep the tensor pipe ahead of shared-memory bandwidth and are used when the mainloop
+  // dominates (long K); short-K layers are bound by the epilogue, which is organised around 128-wide tiles
+  // (four accumulator buffers, so the INT8 row-maximum exchange can trail by two tiles).
   const int sms = dev.sm_count > 0 ? dev.sm_count : 148;
   auto score = [&](int bn) {
     const long tn = (N + bn - 1) / bn;
@@ -597,7 +771,7 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
     const double pad_eff = (double)N / (double)(tn * bn);            // useful columns of the tiles
     return wave_eff * pad_eff;
   };
-  pl.bn = (N > 128 && score(256) + 0.05 >= score(128)) ? 256 : 128;
+  pl.bn = (N > 128 && score(256) + 0.15 >= score(128)) ? 256 : 128;
   const char* force = getenv("QWT_FORCE_BN");
   if (force != nullptr) {
     const int f = atoi(force);
@@ -606,9 +780,14 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   pl.tiles_n = (N + pl.bn - 1) / pl.bn;
   const long tiles = (long)pl.tiles_m * pl.tiles_n;
   pl.grid = (int)(tiles < sms ? tiles : sms);
+  // Short K: a CTA keeps its W tile (K x bn bytes, at most 96 KB) in shared memory for the whole call.  That
+  // needs every tile of a CTA in the same column tile, i.e. a grid that is a multiple of tiles_n.
   const bool w4 = wfmt == QWT_W_INT4_PACKED;
-  pl.smem_bytes = pl.bn == 256 ? (w4 ? SmemLayout<256, true>::kDynamic : SmemLayout<256, false>::kDynamic)
-                               : (w4 ? SmemLayout<128, true>::kDynamic : SmemLayout<128, false>::kDynamic);
+  const long w_tile_bytes = (long)((K + kBK - 1) / kBK) * kBK * pl.bn;
+  const char* nores = getenv("QWT_NO_RESIDENT_W");
+  pl.w_resident = !w4 && w_tile_bytes <= 96 * 1024 && pl.tiles_n <= sms && tiles > sms &&
+                  !(nores != nullptr && nores[0] == '1');
+  if (pl.w_resident) pl.grid = (sms / pl.tiles_n) * pl.tiles_n;
   pl.fused_requant = (out_mode == QWT_OUT_INT8_PER_TOKEN) && (pl.tiles_n <= pl.grid);
   size_t off = 0;
   pl.ws_status_off = off;
@@ -641,14 +820,14 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
     set_cuda_error((int)cudaErrorInvalidValue);
     return QWT_ERR_CUDA;
   }
-  // status word, row maxima and strip counters start at zero
-  QWT_CUDA_TRY(cudaMemsetAsync(ws, 0, plan.ws_z_off, st));
+  // per-token INT8 output: status word, row maxima, strip counters and flags start at zero.  The other output
+  // modes use only the status word, which their kernel clears itself (one launch less per call).
+  if (out_mode == QWT_OUT_INT8_PER_TOKEN && plan.fused_requant) QWT_CUDA_TRY(cudaMemsetAsync(ws, 0, plan.ws_z_off, st));
 
   QlParams prm{};
   prm.x_scale = x_scale;
   prm.fscale = fscale;
   prm.fbias = fbias;
-  prm.Y = Y;
   prm.y_scale = y_scale;
   prm.M = M;
   prm.N = N;
@@ -660,20 +839,21 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   prm.rowmax = reinterpret_cast<uint32_t*>(ws + plan.ws_rowmax_off);
   prm.counters = reinterpret_cast<uint32_t*>(ws + plan.ws_counter_off);
   prm.flags = reinterpret_cast<uint32_t*>(ws + plan.ws_flag_off);
-  prm.counter_target = (uint32_t)plan.tiles_n;
+  prm.counter_target = (uint32_t)((N + kUnitN - 1) / kUnitN);   // units of a row strip that lie inside the matrix
   prm.timeout_ns = timeout_ns_from_env();
 
   int mode = out_mode;
+  prm.Y = Y;
   if (out_mode == QWT_OUT_INT8_PER_TOKEN && !plan.fused_requant) {
     // very wide layers (more column tiles than CTAs): z goes through FP32 scratch and a row quantizer
     mode = QWT_OUT_FP32;
     prm.Y = ws + plan.ws_z_off;
   }
   qwt_status s;
-  if (w4) s = plan.bn == 256 ? launch_bn<256, true>(mode, tmA, tmB, prm, plan.grid, st)
-                             : launch_bn<128, true>(mode, tmA, tmB, prm, plan.grid, st);
-  else s = plan.bn == 256 ? launch_bn<256, false>(mode, tmA, tmB, prm, plan.grid, st)
-                          : launch_bn<128, false>(mode, tmA, tmB, prm, plan.grid, st);
+  if (w4) s = plan.bn == 256 ? launch_bn<256, true>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, st)
+                             : launch_bn<128, true>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, st);
+  else s = plan.bn == 256 ? launch_bn<256, false>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, st)
+                          : launch_bn<128, false>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, st);
   if (s != QWT_OK) return s;
   if (mode != out_mode)
     return launch_quantize_rows(reinterpret_cast<const float*>(ws + plan.ws_z_off), M, N, N, 127,

@@ -68,8 +68,8 @@ struct QlinearPlan {
   int bn;            // CTA tile width (128 or 256)
   int tiles_m, tiles_n;
   int grid;
-  size_t smem_bytes;
   bool fused_requant;    // cross-CTA row-max protocol inside the GEMM kernel
+  bool w_resident;       // grid is a multiple of tiles_n: a CTA's W tile can stay in shared memory
   size_t ws_status_off, ws_rowmax_off, ws_counter_off, ws_flag_off, ws_z_off, ws_total;
 };
 qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
