@@ -77,10 +77,12 @@ struct QlParams {
   int stages;           // depth of the operand ring in shared memory
   int res_kb;           // > 0: the CTA's W tile (all res_kb k-blocks) stays resident, the ring holds X only
   uint32_t* status;
-  uint32_t* rowmax;     // [M] bit patterns of non-negative floats
-  uint32_t* counters;   // [tiles_m] tiles of the strip that have published their row maxima
-  uint32_t* flags;      // [tiles_m] raised by the tile that completes the strip
-  uint32_t counter_target;
+  unsigned long long* partial;   // [tiles_m][units per strip][128]: (tag, row maximum of the unit), zero = not yet there
+  uint32_t counter_target;       // units of a row strip that lie inside the matrix
+  int gather_words;              // exchange words per row: one per unit, or 0 = counter protocol for wide layers
+  uint32_t* rowmax;              // counter protocol: [M] bit patterns of non-negative floats
+  uint32_t* counters;            // [tiles_m] units of the strip that have published their row maxima
+  uint32_t* flags;               // [tiles_m] raised by the unit that completes the strip
   unsigned long long timeout_ns;
 };
 
@@ -496,50 +498,88 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             amax = fmaxf(fmaxf(amax, fmaxf(fabsf(z01.x), fabsf(z01.y))), fmaxf(fabsf(z23.x), fabsf(z23.y)));
           }
         }
-        if (row < p.M) atomicMax(p.rowmax + row, __float_as_uint(amax));
-        __syncwarp();
-        if (lane == 0) {
-          __threadfence();                  // this warp's maxima before the arrival below
-          ptx::mbar_arrive(&pub[g]);
-        }
-        if (lead) {
-          // the lead warp counts the unit once the whole group has published, then waits for the strip
+        // Exchange of the row maxima between the CTAs of a row strip (all words start at zero):
+        //  - up to 16 units per strip: every unit stores (tag 1, its maximum) in an 8-byte word of its own per
+        //    row -- a single aligned 8-byte access is indivisible, so no fence is needed -- and a thread polls
+        //    the words of its row until all are tagged (one store, then loads that hit L2);
+        //  - wider layers (their long mainloop hides the extra round trips): atomicMax into rowmax[m] (a
+        //    non-negative float orders like its bit pattern), then the group's lead warp counts the unit on
+        //    the strip's counter; the unit that completes the strip raises the strip's flag, the others poll it.
+        const int strip_units = (int)p.counter_target;            // units of a row strip inside the matrix
+        const int words = p.gather_words;                         // words per row: strip_units, or 0
+        unsigned long long* slot = p.partial + ((size_t)tm * words) * kBM + qd * 32 + lane;
+        float amax_row = 0.f;
+        int good = 1;
+        if (words > 0) {
+          ptx::st_relaxed_gpu_u64(slot + (size_t)(n0 / kUnitN) * kBM,
+                                  (1ull << 32) | (unsigned long long)__float_as_uint(amax));
+          uint32_t polls = 0;
+          uint64_t t0 = 0;
+          int v = 0;
+          while (v < strip_units) {
+            const unsigned long long w = ptx::ld_relaxed_gpu_u64(slot + (size_t)v * kBM);
+            if ((w >> 32) != 0ull) {
+              amax_row = fmaxf(amax_row, __uint_as_float((uint32_t)w));
+              ++v;
+              continue;
+            }
+            __nanosleep(20);
+            if ((++polls & 127u) == 0u) {
+              const uint64_t now = ptx::globaltimer_ns();
+              if (t0 == 0) t0 = now;
+              if (*cta_abort != 0 || now - t0 > tmo) {
+                good = 0;
+                break;
+              }
+            }
+          }
+        } else {
+          if (row < p.M) atomicMax(p.rowmax + row, __float_as_uint(amax));
+          __syncwarp();
           if (lane == 0) {
-            int good = ptx::mbar_wait_bounded(&pub[g], upar, cta_abort, tmo) ? 1 : 0;
-            if (good) {
-              __threadfence();
-              const uint32_t old = atomicAdd(p.counters + tm, 1u);
-              if (old + 1u == p.counter_target) {
+            __threadfence();                  // this warp's maxima before the arrival below
+            ptx::mbar_arrive(&pub[g]);
+          }
+          if (lead) {
+            // the lead warp counts the unit once the whole group has published, then waits for the strip
+            if (lane == 0) {
+              int fine = ptx::mbar_wait_bounded(&pub[g], upar, cta_abort, tmo) ? 1 : 0;
+              if (fine) {
                 __threadfence();
-                ptx::st_release_gpu(p.flags + tm, 1u);
-              } else {
-                uint32_t polls = 0;
-                uint64_t t0 = 0;
-                while (ptx::ld_acquire_gpu(p.flags + tm) == 0u) {
-                  __nanosleep(32);
-                  if ((++polls & 63u) == 0u) {
-                    const uint64_t now = ptx::globaltimer_ns();
-                    if (t0 == 0) t0 = now;
-                    if (*cta_abort != 0 || now - t0 > tmo || ptx::ld_acquire_gpu(p.status) != 0u) {
-                      good = 0;
-                      break;
+                const uint32_t old = atomicAdd(p.counters + tm, 1u);
+                if (old + 1u == p.counter_target) {
+                  __threadfence();
+                  ptx::st_release_gpu(p.flags + tm, 1u);
+                } else {
+                  uint32_t polls = 0;
+                  uint64_t t0 = 0;
+                  while (ptx::ld_acquire_gpu(p.flags + tm) == 0u) {
+                    __nanosleep(32);
+                    if ((++polls & 63u) == 0u) {
+                      const uint64_t now = ptx::globaltimer_ns();
+                      if (t0 == 0) t0 = now;
+                      if (*cta_abort != 0 || now - t0 > tmo || ptx::ld_acquire_gpu(p.status) != 0u) {
+                        fine = 0;
+                        break;
+                      }
                     }
                   }
                 }
+                __threadfence();
               }
-              __threadfence();
+              if (fine) ptx::mbar_arrive(&ready[g]);
+              else give_up(kStWaitStrip);
             }
-            if (good) ptx::mbar_arrive(&ready[g]);
-            else give_up(kStWaitStrip);
+            __syncwarp();     // the other lanes wait here, not in a spin loop beside lane 0
           }
-          __syncwarp();     // the other lanes wait here, not in a spin loop beside lane 0
+          if (!ptx::mbar_wait_bounded(&ready[g], upar, cta_abort, tmo)) good = 0;
+          else amax_row = row < p.M ? __uint_as_float(__ldcg(p.rowmax + row)) : 0.f;
         }
-        if (!ptx::mbar_wait_bounded(&ready[g], upar, cta_abort, tmo)) {
-          give_up(kStWaitStrip);
+        if (!__all_sync(0xffffffffu, good)) {
+          if (lane == 0) give_up(kStWaitStrip);
           break;
         }
         // ---------------------------------------------------------------- phase 2: scale, codes
-        const float amax_row = row < p.M ? __uint_as_float(__ldcg(p.rowmax + row)) : 0.f;
         const float ys = __fdiv_rn(amax_row, 127.f);
         if (n0 == 0 && row < p.M) p.y_scale[row] = ys;
         den = ys > 0.f ? ys : 1.f;          // a zero row has z == 0 everywhere: codes 0
@@ -792,12 +832,16 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   size_t off = 0;
   pl.ws_status_off = off;
   off += 256;
-  pl.ws_rowmax_off = off;
-  off += ((size_t)M * 4 + 255) / 256 * 256;
-  pl.ws_counter_off = off;
-  off += ((size_t)pl.tiles_m * 4 + 255) / 256 * 256;
-  pl.ws_flag_off = off;
-  off += ((size_t)pl.tiles_m * 4 + 255) / 256 * 256;
+  pl.ws_partial_off = off;      // (tag, row maximum) per strip row and 128-column unit
+  const int strip_units = (N + kUnitN - 1) / kUnitN;
+  pl.gather_words = strip_units <= 16 ? strip_units : 0;
+  if (out_mode == QWT_OUT_INT8_PER_TOKEN) {
+    if (pl.gather_words > 0) {
+      off += (size_t)pl.tiles_m * kBM * pl.gather_words * sizeof(unsigned long long);
+    } else {     // rowmax[tiles_m * 128] | counters[tiles_m] | flags[tiles_m]
+      off += ((size_t)pl.tiles_m * kBM * 4 + 2 * (size_t)pl.tiles_m * 4 + 255) / 256 * 256;
+    }
+  }
   pl.ws_z_off = off;
   if (out_mode == QWT_OUT_INT8_PER_TOKEN && !pl.fused_requant) off += (size_t)M * N * 4;
   pl.ws_total = off;
@@ -820,7 +864,7 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
     set_cuda_error((int)cudaErrorInvalidValue);
     return QWT_ERR_CUDA;
   }
-  // per-token INT8 output: status word, row maxima, strip counters and flags start at zero.  The other output
+  // per-token INT8 output: the status word and the exchanged row maxima start at zero.  The other output
   // modes use only the status word, which their kernel clears itself (one launch less per call).
   if (out_mode == QWT_OUT_INT8_PER_TOKEN && plan.fused_requant) QWT_CUDA_TRY(cudaMemsetAsync(ws, 0, plan.ws_z_off, st));
 
@@ -836,10 +880,12 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   prm.num_tiles = plan.tiles_m * plan.tiles_n;
   prm.num_kb = (K + kBK - 1) / kBK;
   prm.status = reinterpret_cast<uint32_t*>(ws + plan.ws_status_off);
-  prm.rowmax = reinterpret_cast<uint32_t*>(ws + plan.ws_rowmax_off);
-  prm.counters = reinterpret_cast<uint32_t*>(ws + plan.ws_counter_off);
-  prm.flags = reinterpret_cast<uint32_t*>(ws + plan.ws_flag_off);
+  prm.partial = reinterpret_cast<unsigned long long*>(ws + plan.ws_partial_off);
   prm.counter_target = (uint32_t)((N + kUnitN - 1) / kUnitN);   // units of a row strip that lie inside the matrix
+  prm.gather_words = plan.gather_words;
+  prm.rowmax = reinterpret_cast<uint32_t*>(ws + plan.ws_partial_off);
+  prm.counters = prm.rowmax + (size_t)plan.tiles_m * kBM;
+  prm.flags = prm.counters + plan.tiles_m;
   prm.timeout_ns = timeout_ns_from_env();
 
   int mode = out_mode;

@@ -69,8 +69,9 @@ struct QlinearPlan {
   int tiles_m, tiles_n;
   int grid;
   bool fused_requant;    // cross-CTA row-max protocol inside the GEMM kernel
+  int gather_words;      // INT8 output: exchange words per row (one per 128-column unit; 0 = counter protocol)
   bool w_resident;       // grid is a multiple of tiles_n: a CTA's W tile can stay in shared memory
-  size_t ws_status_off, ws_rowmax_off, ws_counter_off, ws_flag_off, ws_z_off, ws_total;
+  size_t ws_status_off, ws_partial_off, ws_z_off, ws_total;
 };
 qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
                         QlinearPlan* plan);
