@@ -13,20 +13,20 @@
 //               unit with its 128 columns.  It reads the INT32 accumulators with
 //               tcgen05.ld (32 columns at a time), forms z = fma(float(acc) * x_scale[m], fscale[n], fbias[n])
 //               (the folded M' and offset of Eq. 10-11, two elements per packed-FP32 instruction), converts,
-//               writes 32-row boxes into swizzled shared memory and hands them to the TMA store unit
-//               (row-contiguous, full-sector writes; rows >= M and columns >= N are clipped by the tensor
-//               map).  The groups run out of phase, so the fixed latencies of one group (waits, proxy fence,
-//               store hand-off) are covered by the arithmetic of the others.
+//               writes 16-byte chunks into a swizzled 32-row box in shared memory; the warp then re-deals its
+//               lanes so that each global store instruction covers whole box rows (row-contiguous writes; rows
+//               >= M and chunks >= N are predicated off).  The groups run out of phase, so the fixed
+//               latencies of one group (waits, exchange) are covered by the arithmetic of the others.
 //   warps 18-21 (packed int4 weights only) expand the W tile to int8 in shared memory before the MMA
 //
 // Per-token INT8 output needs max_n |z[m, n]| over the whole row, but a CTA owns only BN columns of it.
 // The epilogue of a tile therefore has two phases and the accumulators stay in TMEM between them:
-//   phase 1  z from TMEM -> the thread's row maximum over the unit -> atomicMax on rowmax[m] (bit pattern of a
-//            non-negative float orders like an unsigned integer); the group's lead warp then counts the unit
-//            on its strip's counter, and the unit that completes the strip raises the strip's flag;
-//   phase 2  once the flag is up every thread reads its row's final maximum, derives the scale (column tile 0
-//            writes y_scale), re-reads the accumulators, recomputes z, divides, rounds and stores the codes;
-//            only then is the TMEM buffer released.
+//   phase 1  z from TMEM -> the thread's row maximum over the unit -> published to the other CTAs of the strip:
+//            as a tagged 8-byte word per row and unit (strips of at most 16 units), or by atomicMax on
+//            rowmax[m] plus a strip counter and flag (wider layers);
+//   phase 2  once the maxima of every unit of the strip are there, every thread derives its row's scale (the
+//            unit at column 0 writes y_scale), re-reads the accumulators, recomputes z, divides, rounds and
+//            stores the codes; only then is the TMEM buffer released.
 // While a group waits for its strip the other groups work on the following tiles.  Progress: phase 1 of
 // tile t needs (a) its group, i.e. phase 2 of tile t - kAcc*G finished, and (b) its accumulator, whose
 // buffer is released by that same phase 2; phase 2 of a tile u needs phase 1 of the tiles of u's strip, all
