@@ -513,15 +513,23 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (words > 0) {
           ptx::st_relaxed_gpu_u64(slot + (size_t)(n0 / kUnitN) * kBM,
                                   (1ull << 32) | (unsigned long long)__float_as_uint(amax));
+          // all words of the row are requested together (one L2 round trip when they are all there)
           uint32_t polls = 0;
           uint64_t t0 = 0;
-          int v = 0;
-          while (v < strip_units) {
-            const unsigned long long w = ptx::ld_relaxed_gpu_u64(slot + (size_t)v * kBM);
-            if ((w >> 32) != 0ull) {
-              amax_row = fmaxf(amax_row, __uint_as_float((uint32_t)w));
-              ++v;
-              continue;
+          while (true) {
+            unsigned long long w[16];
+#pragma unroll
+            for (int v = 0; v < 16; ++v) w[v] = v < strip_units ? ptx::ld_relaxed_gpu_u64(slot + (size_t)v * kBM) : (1ull << 32);
+            bool all = true;
+            float m = 0.f;
+#pragma unroll
+            for (int v = 0; v < 16; ++v) {
+              all = all && (w[v] >> 32) != 0ull;
+              m = fmaxf(m, __uint_as_float((uint32_t)w[v]));
+            }
+            if (all) {
+              amax_row = m;
+              break;
             }
             __nanosleep(20);
             if ((++polls & 127u) == 0u) {
