@@ -41,6 +41,7 @@
 #include <stdlib.h>
 
 #include <mutex>
+#include <type_traits>
 
 #include "ptx_sm100.cuh"
 #include "qwt2_internal.h"
@@ -603,9 +604,12 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const float2 magic2 = make_float2(12582912.f, 12582912.f);
         // z / den rounded to nearest: q0 = z * (1/den), then one residual correction with fused multiply-adds;
         // adding 1.5 * 2^23 leaves rne(q) in the low mantissa bits (|q| <= 127 by construction)
+        // (the whole box loop is instantiated twice so that the common case carries no branch per element)
+        auto convert_and_store = [&](auto slow_tag) {
+        constexpr bool SLOW = decltype(slow_tag)::value;
         auto quant = [&](float2 z) -> float2 {
           float2 q;
-          if (slow) {
+          if (SLOW) {
             q = make_float2(__fdiv_rn(z.x, den), __fdiv_rn(z.y, den));
           } else {
             const float2 q0 = __fmul2_rn(z, inv2);
@@ -673,6 +677,9 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
           store_box((n0 + bx * BC) * ESZ, y0);
         }
+        };
+        if (C::kInt8Out && slow) convert_and_store(std::true_type{});
+        else convert_and_store(std::false_type{});
       }
       // the accumulator buffer and the group's parameter slice are free again
       ptx::tc_fence_before();
