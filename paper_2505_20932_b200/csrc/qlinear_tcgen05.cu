@@ -388,7 +388,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // Work item = one unit: 128 columns of a tile.  The CTA's units are numbered u = j * kUPT + half
     // (j = local tile); group g takes u = g, g + 4, ...  Unit u lives in TMEM columns (u % 4) * 128.
     constexpr int UPT = C::kUPT;
-    constexpr int NC = 32;                  // columns per tcgen05.ld
+    constexpr int NC = 16;                  // columns per tcgen05.ld
     constexpr int BOXB = C::kBoxBytes;
     constexpr int BC = C::kBC;              // columns per staging box
     constexpr int ESZ = C::kEsz;
@@ -488,7 +488,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll 1
         for (int h = 0; h < kUnitN / NC; ++h) {
           uint32_t r[NC];
-          ptx::tmem_ld_32x32b_x32(taddr + h * NC, r);
+          ptx::tmem_ld_cols<NC>(taddr + h * NC, r);
           ptx::tmem_ld_wait();
 #pragma unroll
           for (int e = 0; e < NC; e += 4) {
