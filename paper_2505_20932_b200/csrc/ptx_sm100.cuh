@@ -159,6 +159,43 @@ __device__ __forceinline__ void tmem_ld_cols(uint32_t taddr, uint32_t (&r)[NC]) 
   else tmem_ld_32x32b_x8(taddr, r);
 }
 
+// 16 lanes x (8 * NB) columns of 32-bit, the layout of an m16n8 accumulator fragment repeated NB times along
+// the columns: with q = lane / 4 and c = lane % 4, registers 4i, 4i+1 hold lane (base + q), columns 8i + 2c and
+// 8i + 2c + 1; registers 4i+2, 4i+3 hold lane (base + q + 8), same columns.  A thread therefore sees only a
+// quarter of the columns, but four rows per pair of loads (base = first lane of the warp's quadrant, and + 16).
+__device__ __forceinline__ void tmem_ld_16x256b_x4(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x4.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+               : "r"(taddr)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld_16x256b_x2(uint32_t taddr, uint32_t (&r)[8]) {
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x2.b32 {%0, %1, %2, %3, %4, %5, %6, %7}, [%8];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7])
+               : "r"(taddr)
+               : "memory");
+}
+__device__ __forceinline__ void tmem_ld_16x256b_x1(uint32_t taddr, uint32_t (&r)[4]) {
+  asm volatile("tcgen05.ld.sync.aligned.16x256b.x1.b32 {%0, %1, %2, %3}, [%4];"
+               : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3])
+               : "r"(taddr)
+               : "memory");
+}
+template <int NB>
+__device__ __forceinline__ void tmem_ld_frag(uint32_t taddr, uint32_t (&r)[4 * NB]) {
+  static_assert(NB == 4 || NB == 2 || NB == 1, "8-column blocks per tcgen05.ld");
+  if constexpr (NB == 4) tmem_ld_16x256b_x4(taddr, r);
+  else if constexpr (NB == 2) tmem_ld_16x256b_x2(taddr, r);
+  else tmem_ld_16x256b_x1(taddr, r);
+}
+
+// Registers -> TMEM, same fragment layout as tmem_ld_16x256b_x4 (32 columns x 16 lanes).
+__device__ __forceinline__ void tmem_st_16x256b_x4(uint32_t taddr, const uint32_t (&r)[16]) {
+  asm volatile("tcgen05.st.sync.aligned.16x256b.x4.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
+               : "memory");
+}
+__device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
 // Shared-memory matrix descriptor of a K-major operand tile stored as rows of 128 bytes with the
 // 128-byte swizzle (the layout a TMA box {128 bytes, rows} with SWIZZLE_128B produces):
 //   bits  0-13 start address >> 4      bits 16-29 leading byte offset >> 4 (not used by this layout, 1)

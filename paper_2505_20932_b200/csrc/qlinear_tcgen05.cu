@@ -9,11 +9,13 @@
 //               kAcc = 512 / BN TMEM accumulator buffers; tcgen05.commit releases the stage / publishes the buffer
 //   warps 2-17  epilogue: 4 groups of 4 warps.  The work item of a group is a unit = 128 columns of a tile;
 //               the CTA's units are dealt to the groups round-robin (the 512 TMEM columns hold 4 units).
-//               Inside a group the warp's TMEM lane quadrant is warp % 4, so a thread owns ONE ROW of the
-//               unit with its 128 columns.  It reads the INT32 accumulators with
-//               tcgen05.ld (32 columns at a time), forms z = fma(float(acc) * x_scale[m], fscale[n], fbias[n])
+//               Inside a group the warp's TMEM lane quadrant is warp % 4.  The accumulators are read with
+//               tcgen05.ld.16x256b (the m16n8 fragment layout): a thread sees four rows and a quarter of the
+//               columns, so a per-column parameter is loaded once and used four times -- with one row per
+//               thread every lane needs every column's fscale/fbias and the shared-memory pipe bounds the
+//               epilogue.  It forms z = fma(float(acc) * x_scale[m], fscale[n], fbias[n])
 //               (the folded M' and offset of Eq. 10-11, two elements per packed-FP32 instruction), converts,
-//               writes 16-byte chunks into a swizzled 32-row box in shared memory; the warp then re-deals its
+//               writes its words into a swizzled 32-row box in shared memory; the warp then re-deals its
 //               lanes so that each global store instruction covers whole box rows (row-contiguous writes; rows
 //               >= M and chunks >= N are predicated off).  The groups run out of phase, so the fixed
 //               latencies of one group (waits, exchange) are covered by the arithmetic of the others.
@@ -21,12 +23,13 @@
 //
 // Per-token INT8 output needs max_n |z[m, n]| over the whole row, but a CTA owns only BN columns of it.
 // The epilogue of a tile therefore has two phases and the accumulators stay in TMEM between them:
-//   phase 1  z from TMEM -> the thread's row maximum over the unit -> published to the other CTAs of the strip:
+//   phase 1  z from the accumulators (written back to TMEM in their place) -> row maxima of the unit (combined
+//            over the four lanes that share a row) -> published to the other CTAs of the strip:
 //            as a tagged 8-byte word per row and unit (strips of at most 16 units), or by atomicMax on
 //            rowmax[m] plus a strip counter and flag (wider layers);
-//   phase 2  once the maxima of every unit of the strip are there, every thread derives its row's scale (the
-//            unit at column 0 writes y_scale), re-reads the accumulators, recomputes z, divides, rounds and
-//            stores the codes; only then is the TMEM buffer released.
+//   phase 2  once the maxima of every unit of the strip are there, the rows' scales follow (the unit at column
+//            0 writes y_scale); z is read back from TMEM, divided, rounded and stored as codes; only then is
+//            the TMEM buffer released.
 // While a group waits for its strip the other groups work on the following tiles.  Progress: phase 1 of
 // tile t needs (a) its group, i.e. phase 2 of tile t - kAcc*G finished, and (b) its accumulator, whose
 // buffer is released by that same phase 2; phase 2 of a tile u needs phase 1 of the tiles of u's strip, all
@@ -138,10 +141,6 @@ struct Cfg {
 template <int BOXB>
 __device__ __forceinline__ uint32_t swizzle_xor(int row) {
   return BOXB == 32 ? ((row >> 2) & 1) : (BOXB == 64 ? ((row >> 1) & 3) : (row & 7));
-}
-
-__device__ __forceinline__ void st_shared_v4(void* p, uint32_t a, uint32_t b, uint32_t c, uint32_t d) {
-  *reinterpret_cast<uint4*>(p) = make_uint4(a, b, c, d);
 }
 
 __device__ __forceinline__ uint32_t pack_bf16x2(float lo, float hi) {
@@ -388,7 +387,6 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // Work item = one unit: 128 columns of a tile.  The CTA's units are numbered u = j * kUPT + half
     // (j = local tile); group g takes u = g, g + 4, ...  Unit u lives in TMEM columns (u % 4) * 128.
     constexpr int UPT = C::kUPT;
-    constexpr int NC = 16;                  // columns per tcgen05.ld
     constexpr int BOXB = C::kBoxBytes;
     constexpr int BC = C::kBC;              // columns per staging box
     constexpr int ESZ = C::kEsz;
@@ -446,10 +444,15 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int tm = tile / p.tiles_n;
       const int n0 = unit_col0(u);
       const uint32_t buf = j % kAcc, tpar = (j / kAcc) & 1u, upar = use & 1u;
-      const int row = tm * kBM + qd * 32 + lane;
       const int y0 = tm * kBM + qd * 32;
-      float xs = 0.f;
-      if (C::kHasParams && row < p.M) xs = __ldg(p.x_scale + row);     // issued before the waits below
+      float xs4[4] = {0.f, 0.f, 0.f, 0.f};    // x_scale of the thread's four rows, requested before the waits below
+      if (C::kHasParams) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int r = y0 + (lane >> 2) + 8 * k;
+          if (r < p.M) xs4[k] = __ldg(p.x_scale + r);
+        }
+      }
       bool ok = true;
       if (C::kHasParams) {
         if (lead) {
@@ -477,28 +480,64 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         break;
       }
       ptx::tc_fence_after();
-      const float2 xs2 = make_float2(xs, xs);
+      // Fragment geometry of this thread (see tmem_ld_frag): it sees the unit's columns 8i + 2c, 8i + 2c + 1 and
+      // the four rows q + 8k (k = 0..3) of the warp's 32.  Per-column parameters are then loaded once per column
+      // pair and used for four rows, which is what keeps the shared-memory pipe from bounding the epilogue.
+      const int q = lane >> 2, c = lane & 3;
+      const float2 xs2[4] = {make_float2(xs4[0], xs4[0]), make_float2(xs4[1], xs4[1]), make_float2(xs4[2], xs4[2]),
+                             make_float2(xs4[3], xs4[3])};
       const bool in_range = n0 < p.N;        // a unit entirely right of the matrix has nothing to compute or store
+      // z of one 8-column block for the thread's four rows; a = registers of lanes q, q + 8 (half 0) and of
+      // lanes q + 16, q + 24 (half 1); col = first column of the block inside the unit
+      auto z_block = [&](const uint32_t* a0, const uint32_t* a1, int col, float2 (&z)[4]) {
+        const float2 f2 = *reinterpret_cast<const float2*>(ps_fs + col + 2 * c);
+        const float2 b2 = *reinterpret_cast<const float2*>(ps_fb + col + 2 * c);
+        z[0] = z_pair(a0[0], a0[1], xs2[0], f2.x, f2.y, b2.x, b2.y);     // columns >= N give 0 * 0 + 0
+        z[1] = z_pair(a0[2], a0[3], xs2[1], f2.x, f2.y, b2.x, b2.y);
+        z[2] = z_pair(a1[0], a1[1], xs2[2], f2.x, f2.y, b2.x, b2.y);
+        z[3] = z_pair(a1[2], a1[3], xs2[3], f2.x, f2.y, b2.x, b2.y);
+      };
 
-      float den = 1.f, inv = 1.f;
+      float den[4] = {1.f, 1.f, 1.f, 1.f}, inv[4] = {1.f, 1.f, 1.f, 1.f};
       bool slow = false;
       if (C::kInt8Out && in_range) {
         // ---------------------------------------------------------------- phase 1: row maxima of the unit
-        float amax = 0.f;
+        float amax[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll 1
-        for (int h = 0; h < kUnitN / NC; ++h) {
-          uint32_t r[NC];
-          ptx::tmem_ld_cols<NC>(taddr + h * NC, r);
+        for (int h = 0; h < kUnitN / 32; ++h) {
+          uint32_t a0[16], a1[16];
+          ptx::tmem_ld_16x256b_x4(taddr + h * 32, a0);
+          ptx::tmem_ld_16x256b_x4(taddr + (16u << 16) + h * 32, a1);
           ptx::tmem_ld_wait();
 #pragma unroll
-          for (int e = 0; e < NC; e += 4) {
-            const float4 f4 = *reinterpret_cast<const float4*>(ps_fs + h * NC + e);
-            const float4 b4 = *reinterpret_cast<const float4*>(ps_fb + h * NC + e);
-            const float2 z01 = z_pair(r[e], r[e + 1], xs2, f4.x, f4.y, b4.x, b4.y);   // columns >= N give 0 * 0 + 0
-            const float2 z23 = z_pair(r[e + 2], r[e + 3], xs2, f4.z, f4.w, b4.z, b4.w);
-            amax = fmaxf(fmaxf(amax, fmaxf(fabsf(z01.x), fabsf(z01.y))), fmaxf(fabsf(z23.x), fabsf(z23.y)));
+          for (int i = 0; i < 4; ++i) {
+            float2 z[4];
+            z_block(a0 + 4 * i, a1 + 4 * i, h * 32 + 8 * i, z);
+#pragma unroll
+            for (int k = 0; k < 4; ++k) amax[k] = fmaxf(amax[k], fmaxf(fabsf(z[k].x), fabsf(z[k].y)));
+            // z replaces the accumulators in TMEM: phase 2 reads it back instead of recomputing it
+            a0[4 * i] = __float_as_uint(z[0].x);
+            a0[4 * i + 1] = __float_as_uint(z[0].y);
+            a0[4 * i + 2] = __float_as_uint(z[1].x);
+            a0[4 * i + 3] = __float_as_uint(z[1].y);
+            a1[4 * i] = __float_as_uint(z[2].x);
+            a1[4 * i + 1] = __float_as_uint(z[2].y);
+            a1[4 * i + 2] = __float_as_uint(z[3].x);
+            a1[4 * i + 3] = __float_as_uint(z[3].y);
           }
+          ptx::tmem_st_16x256b_x4(taddr + h * 32, a0);
+          ptx::tmem_st_16x256b_x4(taddr + (16u << 16) + h * 32, a1);
         }
+        ptx::tmem_st_wait();
+        // the four lanes that share a row (same q) combine; lane (q, c) then speaks for row q + 8c
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          amax[k] = fmaxf(amax[k], __shfl_xor_sync(0xffffffffu, amax[k], 1));
+          amax[k] = fmaxf(amax[k], __shfl_xor_sync(0xffffffffu, amax[k], 2));
+        }
+        const float amax_mine = c == 0 ? amax[0] : (c == 1 ? amax[1] : (c == 2 ? amax[2] : amax[3]));
+        const int my = q + 8 * c;             // row (inside the warp's 32) this lane publishes and fetches
+        const int row = y0 + my;
         // Exchange of the row maxima between the CTAs of a row strip (all words start at zero):
         //  - up to 16 units per strip: every unit stores (tag 1, its maximum) in an 8-byte word of its own per
         //    row -- a single aligned 8-byte access is indivisible, so no fence is needed -- and a thread polls
@@ -508,12 +547,12 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         //    the strip's counter; the unit that completes the strip raises the strip's flag, the others poll it.
         const int strip_units = (int)p.counter_target;            // units of a row strip inside the matrix
         const int words = p.gather_words;                         // words per row: strip_units, or 0
-        unsigned long long* slot = p.partial + ((size_t)tm * words) * kBM + qd * 32 + lane;
+        unsigned long long* slot = p.partial + ((size_t)tm * words) * kBM + qd * 32 + my;
         float amax_row = 0.f;
         int good = 1;
         if (words > 0) {
           ptx::st_relaxed_gpu_u64(slot + (size_t)(n0 / kUnitN) * kBM,
-                                  (1ull << 32) | (unsigned long long)__float_as_uint(amax));
+                                  (1ull << 32) | (unsigned long long)__float_as_uint(amax_mine));
           // all words of the row are requested together (one L2 round trip when they are all there)
           uint32_t polls = 0;
           uint64_t t0 = 0;
@@ -543,7 +582,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
           }
         } else {
-          if (row < p.M) atomicMax(p.rowmax + row, __float_as_uint(amax));
+          if (row < p.M) atomicMax(p.rowmax + row, __float_as_uint(amax_mine));
           __syncwarp();
           if (lane == 0) {
             __threadfence();                  // this warp's maxima before the arrival below
@@ -591,92 +630,103 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // ---------------------------------------------------------------- phase 2: scale, codes
         const float ys = __fdiv_rn(amax_row, 127.f);
         if (n0 == 0 && row < p.M) p.y_scale[row] = ys;
-        den = ys > 0.f ? ys : 1.f;          // a zero row has z == 0 everywhere: codes 0
-        inv = __frcp_rn(den);
+        const float den_mine = ys > 0.f ? ys : 1.f;          // a zero row has z == 0 everywhere: codes 0
+        const float inv_mine = __frcp_rn(den_mine);
         // a scale so small that its reciprocal overflows (never on real data): divide directly
-        slow = __any_sync(0xffffffffu, !(inv <= 3.0e38f));
+        slow = __any_sync(0xffffffffu, !(inv_mine <= 3.0e38f));
+        // row q + 8k was handled by lane (q, k)
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          den[k] = __shfl_sync(0xffffffffu, den_mine, (lane & ~3) + k);
+          inv[k] = __shfl_sync(0xffffffffu, inv_mine, (lane & ~3) + k);
+        }
       }
 
       // ------------------------------------------------------------------ conversion and store, box by box
       if (in_range) {
-        const float2 inv2 = make_float2(inv, inv);
-        const float2 nden2 = make_float2(-den, -den);
-        const float2 magic2 = make_float2(12582912.f, 12582912.f);
         // z / den rounded to nearest: q0 = z * (1/den), then one residual correction with fused multiply-adds;
-        // adding 1.5 * 2^23 leaves rne(q) in the low mantissa bits (|q| <= 127 by construction)
+        // adding 1.5 * 2^23 leaves rne(q) in the low mantissa bits (|q| <= 127 by construction).
         // (the whole box loop is instantiated twice so that the common case carries no branch per element)
         auto convert_and_store = [&](auto slow_tag) {
-        constexpr bool SLOW = decltype(slow_tag)::value;
-        auto quant = [&](float2 z) -> float2 {
-          float2 q;
-          if (SLOW) {
-            q = make_float2(__fdiv_rn(z.x, den), __fdiv_rn(z.y, den));
-          } else {
-            const float2 q0 = __fmul2_rn(z, inv2);
-            const float2 rem = __ffma2_rn(q0, nden2, z);
-            q = __ffma2_rn(rem, inv2, q0);
-          }
-          return __fadd2_rn(q, magic2);
-        };
-        constexpr int LDC = BC < NC ? BC : NC;       // columns per load inside a box
+          constexpr bool SLOW = decltype(slow_tag)::value;
+          const float2 magic2 = make_float2(12582912.f, 12582912.f);
+          auto quant = [&](float2 z, int k) -> uint32_t {      // two codes in the low 16 bits
+            float2 qq;
+            if (SLOW) {
+              qq = make_float2(__fdiv_rn(z.x, den[k]), __fdiv_rn(z.y, den[k]));
+            } else {
+              const float2 i2 = make_float2(inv[k], inv[k]);
+              const float2 q0 = __fmul2_rn(z, i2);
+              const float2 rem = __ffma2_rn(q0, make_float2(-den[k], -den[k]), z);
+              qq = __ffma2_rn(rem, i2, q0);
+            }
+            const float2 m = __fadd2_rn(qq, magic2);
+            return __byte_perm(__float_as_uint(m.x), __float_as_uint(m.y), 0x0040) & 0xffffu;
+          };
+          constexpr int LDC = BC < 32 ? BC : 32;       // columns per pair of loads inside a box
+          constexpr int NB = LDC / 8;                  // 8-column blocks per load
+          // byte address of (row r of the warp's 32, byte b of the box row) in the swizzled staging slot
+          auto stage_at = [&](int r, int b) -> uint8_t* {
+            return stg + r * BOXB + ((((uint32_t)b >> 4) ^ swizzle_xor<BOXB>(r)) << 4) + (b & 15);
+          };
 #pragma unroll 1
-        for (int bx = 0; bx < kUnitN / BC; ++bx) {
-          if (n0 + bx * BC >= p.N) break;
-          uint8_t* dst = stg + lane * BOXB;
+          for (int bx = 0; bx < kUnitN / BC; ++bx) {
+            if (n0 + bx * BC >= p.N) break;
 #pragma unroll 1
-          for (int h = 0; h < BC / LDC; ++h) {
-            const int c0 = bx * BC + h * LDC;         // first column (inside the unit) of this load
-            uint32_t r[LDC];
-            ptx::tmem_ld_cols<LDC>(taddr + c0, r);
-            ptx::tmem_ld_wait();
-            constexpr int EPC = 16 / ESZ;            // elements per 16-byte chunk
+            for (int h = 0; h < BC / LDC; ++h) {
+              const int c0 = bx * BC + h * LDC;         // first column (inside the unit) of this pair of loads
+              uint32_t a0[4 * NB], a1[4 * NB];
+              ptx::tmem_ld_frag<NB>(taddr + c0, a0);
+              ptx::tmem_ld_frag<NB>(taddr + (16u << 16) + c0, a1);
+              ptx::tmem_ld_wait();
 #pragma unroll
-            for (int c = 0; c < LDC / EPC; ++c) {
-              uint32_t w[4];
-              if (OUT == QWT_OUT_INT32_ACC) {
+              for (int i = 0; i < NB; ++i) {
+                const int colb = h * LDC + 8 * i;      // first column of the block inside the box
+                if (OUT == QWT_OUT_INT32_ACC) {
+                  // W4: every term is a multiple of 16, the shift is exact
+                  auto fix = [](uint32_t v) { return W4 ? (uint32_t)((int)v >> 4) : v; };
+                  const int b = (colb + 2 * c) * 4;
+                  *reinterpret_cast<uint2*>(stage_at(q, b)) = make_uint2(fix(a0[4 * i]), fix(a0[4 * i + 1]));
+                  *reinterpret_cast<uint2*>(stage_at(q + 8, b)) = make_uint2(fix(a0[4 * i + 2]), fix(a0[4 * i + 3]));
+                  *reinterpret_cast<uint2*>(stage_at(q + 16, b)) = make_uint2(fix(a1[4 * i]), fix(a1[4 * i + 1]));
+                  *reinterpret_cast<uint2*>(stage_at(q + 24, b)) = make_uint2(fix(a1[4 * i + 2]), fix(a1[4 * i + 3]));
+                } else {
+                  float2 z[4];
+                  if (C::kInt8Out) {      // phase 1 left z in TMEM
+                    z[0] = make_float2(__uint_as_float(a0[4 * i]), __uint_as_float(a0[4 * i + 1]));
+                    z[1] = make_float2(__uint_as_float(a0[4 * i + 2]), __uint_as_float(a0[4 * i + 3]));
+                    z[2] = make_float2(__uint_as_float(a1[4 * i]), __uint_as_float(a1[4 * i + 1]));
+                    z[3] = make_float2(__uint_as_float(a1[4 * i + 2]), __uint_as_float(a1[4 * i + 3]));
+                  } else {
+                    z_block(a0 + 4 * i, a1 + 4 * i, c0 + 8 * i, z);
+                  }
+                  if (OUT == QWT_OUT_FP32) {
+                    const int b = (colb + 2 * c) * 4;
 #pragma unroll
-                for (int t = 0; t < 4; ++t)           // W4: every term is a multiple of 16, the shift is exact
-                  w[t] = W4 ? (uint32_t)((int)r[c * 4 + t] >> 4) : r[c * 4 + t];
-              } else if (OUT == QWT_OUT_FP32) {
-                const int e = c * 4;
-                const float4 f4 = *reinterpret_cast<const float4*>(ps_fs + c0 + e);
-                const float4 b4 = *reinterpret_cast<const float4*>(ps_fb + c0 + e);
-                const float2 z01 = z_pair(r[e], r[e + 1], xs2, f4.x, f4.y, b4.x, b4.y);
-                const float2 z23 = z_pair(r[e + 2], r[e + 3], xs2, f4.z, f4.w, b4.z, b4.w);
-                w[0] = __float_as_uint(z01.x);
-                w[1] = __float_as_uint(z01.y);
-                w[2] = __float_as_uint(z23.x);
-                w[3] = __float_as_uint(z23.y);
-              } else if (OUT == QWT_OUT_BF16) {
+                    for (int k = 0; k < 4; ++k) *reinterpret_cast<float2*>(stage_at(q + 8 * k, b)) = z[k];
+                  } else if (OUT == QWT_OUT_BF16) {
+                    const int b = (colb + 2 * c) * 2;
 #pragma unroll
-                for (int t = 0; t < 2; ++t) {
-                  const int e = c * 8 + t * 4;
-                  const float4 f4 = *reinterpret_cast<const float4*>(ps_fs + c0 + e);
-                  const float4 b4 = *reinterpret_cast<const float4*>(ps_fb + c0 + e);
-                  const float2 z01 = z_pair(r[e], r[e + 1], xs2, f4.x, f4.y, b4.x, b4.y);
-                  const float2 z23 = z_pair(r[e + 2], r[e + 3], xs2, f4.z, f4.w, b4.z, b4.w);
-                  w[2 * t] = pack_bf16x2(z01.x, z01.y);
-                  w[2 * t + 1] = pack_bf16x2(z23.x, z23.y);
-                }
-              } else {  // INT8 codes
-#pragma unroll
-                for (int t = 0; t < 4; ++t) {
-                  const int e = c * 16 + t * 4;
-                  const float4 f4 = *reinterpret_cast<const float4*>(ps_fs + c0 + e);
-                  const float4 b4 = *reinterpret_cast<const float4*>(ps_fb + c0 + e);
-                  const float2 m01 = quant(z_pair(r[e], r[e + 1], xs2, f4.x, f4.y, b4.x, b4.y));
-                  const float2 m23 = quant(z_pair(r[e + 2], r[e + 3], xs2, f4.z, f4.w, b4.z, b4.w));
-                  const uint32_t lo = __byte_perm(__float_as_uint(m01.x), __float_as_uint(m01.y), 0x0040);
-                  const uint32_t hi = __byte_perm(__float_as_uint(m23.x), __float_as_uint(m23.y), 0x0040);
-                  w[t] = __byte_perm(lo, hi, 0x5410);
+                    for (int k = 0; k < 4; ++k)
+                      *reinterpret_cast<uint32_t*>(stage_at(q + 8 * k, b)) = pack_bf16x2(z[k].x, z[k].y);
+                  } else {
+                    // INT8: neighbouring lanes (c even / odd) swap halves so that each ends up with 4 consecutive
+                    // codes of two rows: the even lane keeps rows q, q + 16, the odd lane rows q + 8, q + 24
+                    const uint32_t h0 = quant(z[0], 0), h1 = quant(z[1], 1), h2 = quant(z[2], 2), h3 = quant(z[3], 3);
+                    const bool odd = (c & 1) != 0;
+                    const uint32_t send = odd ? (h0 | (h2 << 16)) : (h1 | (h3 << 16));
+                    const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
+                    const uint32_t wa = odd ? ((recv & 0xffffu) | (h1 << 16)) : (h0 | (recv << 16));
+                    const uint32_t wb = odd ? ((recv >> 16) | (h3 << 16)) : (h2 | (recv & 0xffff0000u));
+                    const int b = colb + 2 * (c & ~1);
+                    *reinterpret_cast<uint32_t*>(stage_at(odd ? q + 8 : q, b)) = wa;
+                    *reinterpret_cast<uint32_t*>(stage_at(odd ? q + 24 : q + 16, b)) = wb;
+                  }
                 }
               }
-              const uint32_t chunk = (uint32_t)(h * (LDC / EPC) + c);     // 16-byte chunk inside the box row
-              st_shared_v4(dst + ((chunk ^ swz) << 4), w[0], w[1], w[2], w[3]);
             }
+            store_box((n0 + bx * BC) * ESZ, y0);
           }
-          store_box((n0 + bx * BC) * ESZ, y0);
-        }
         };
         if (C::kInt8Out && slow) convert_and_store(std::true_type{});
         else convert_and_store(std::false_type{});
