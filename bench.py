@@ -181,11 +181,18 @@ def build_layer(B, torch, WL, spec, seed, device, calib_rows=None):
     return L
 
 
-def phase_a(B, layers, stream):
-    for L in layers:
+def phase_a(B, layers, stream, side=None):
+    """Calibrate + fold every layer.  The layers are independent, so with a second stream (`side`) they alternate
+    between the two: the small solve / fold kernels of one layer then run under the next layer's statistics pass."""
+    if side is not None:
+        side.wait_stream(stream)
+    for i, L in enumerate(layers):
         s = L.spec
-        B.qwt_cwac_calibrate(L.fp_out, L.q_out, L.R, s.N, s.N, L.a, L.b, None, L.cws, L.cws_bytes, stream)
-        B.qwt_cwac_fold(L.ws, L.bias, L.a, L.b, s.N, L.fs, L.fb, stream)
+        st = stream if (side is None or i % 2 == 0) else side
+        B.qwt_cwac_calibrate(L.fp_out, L.q_out, L.R, s.N, s.N, L.a, L.b, None, L.cws, L.cws_bytes, st)
+        B.qwt_cwac_fold(L.ws, L.bias, L.a, L.b, s.N, L.fs, L.fb, st)
+    if side is not None:
+        stream.wait_stream(side)
 
 
 def phase_b(B, layers, stream):
@@ -364,12 +371,16 @@ def run_ours(args):
         cap.wait_stream(stream)
         graphs = []
         B.qwt_launch_count_reset()
+        side = torch.cuda.Stream()
         with torch.cuda.stream(cap):
-            for phase in (phase_a, phase_b):
-                g = torch.cuda.CUDAGraph()
-                with torch.cuda.graph(g, stream=cap):
-                    phase(B, layers, cap)
-                graphs.append(g)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=cap):
+                phase_a(B, layers, cap, side)
+            graphs.append(g)
+            g = torch.cuda.CUDAGraph()
+            with torch.cuda.graph(g, stream=cap):
+                phase_b(B, layers, cap)
+            graphs.append(g)
         launches_per_step = B.qwt_launch_count()      # launches recorded = launches per replayed step
         stream.wait_stream(cap)
         for g in graphs:                               # one untimed replay

@@ -155,11 +155,11 @@ __device__ __forceinline__ void cwac_solve_channel(double n, double Sq, double S
   *b = (float)(mf - alpha * mq);
 }
 
-// Adds the partials of all row chunks.  A block owns 32 channels; its 8 row lanes each add every 8th
+// Adds the partials of all row chunks.  A block owns 32 channels; its 32 row lanes each add every 32nd
 // chunk, then the lanes are combined in a fixed order, so the result does not depend on scheduling.
 // stats_io (may be NULL): running statistics to update.  a, b (may be NULL): solve after the reduction.
 constexpr int kRedTX = 32;
-constexpr int kRedTY = 8;
+constexpr int kRedTY = 32;
 __global__ void __launch_bounds__(kRedTX * kRedTY)
 cwac_reduce_kernel(const double* __restrict__ partial, int chunks, int cpad, int channels, double n_rows,
                    double* __restrict__ stats_io, float* __restrict__ a, float* __restrict__ b,
