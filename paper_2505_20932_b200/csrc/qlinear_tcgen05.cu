@@ -431,7 +431,9 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
       for (int i = 0; i < CPR; ++i) {
         const int r = i * RPI + lane / CPR;
-        const uint4 v = *reinterpret_cast<const uint4*>(stg + r * BOXB + ((chunk ^ swizzle_xor<BOXB>(r)) << 4));
+        uint4 v = *reinterpret_cast<const uint4*>(stg + r * BOXB + ((chunk ^ swizzle_xor<BOXB>(r)) << 4));
+        // INT8 boxes: rows 8-15 and 24-31 were written with the 8-byte halves of every chunk exchanged
+        if (C::kInt8Out && (r & 8) != 0) v = make_uint4(v.z, v.w, v.x, v.y);
         if (col_ok && y + r < p.M) *reinterpret_cast<uint4*>(out + (size_t)(y + r) * p.N * ESZ) = v;
       }
       __syncwarp();                                  // the slot may be rewritten
@@ -718,7 +720,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
                     const uint32_t wa = odd ? ((recv & 0xffffu) | (h1 << 16)) : (h0 | (recv << 16));
                     const uint32_t wb = odd ? ((recv >> 16) | (h3 << 16)) : (h2 | (recv & 0xffff0000u));
-                    const int b = colb + 2 * (c & ~1);
+                    // One store covers rows q (even lanes) and q + 8 (odd lanes): 16 rows x 8 bytes.  The odd
+                    // lanes' rows use the other 8-byte half of the chunk (undone in store_box), which spreads the
+                    // 16 pieces over all banks.
+                    const int b = (colb + 2 * (c & ~1)) ^ (odd ? 8 : 0);
                     *reinterpret_cast<uint32_t*>(stage_at(odd ? q + 8 : q, b)) = wa;
                     *reinterpret_cast<uint32_t*>(stage_at(odd ? q + 24 : q + 16, b)) = wb;
                   }
