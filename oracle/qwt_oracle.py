@@ -215,6 +215,21 @@ def fold_integer_offset(alpha, beta, S_x: float, S_W, S_r: float):
     return Mp, off
 
 
+def requant_static(acc, Mp, off, Z_r: int = 0, qmax: int = 127) -> np.ndarray:
+    """Eq. 10 as printed, for an engine with static scales: r_q = Z_r + M' (acc + offset), rounded and clipped,
+
+        r_q[m, n] = clip(round(M'[n] * (acc[m, n] + off[n])) + Z_r, -qmax, qmax).
+
+    `acc` is the integer bracket of Eq. 7 (here W_q x_q, zero-points 0) and `off` the rounded
+    beta / (alpha S_x S_W) of Eq. 10; their sum is exact integer arithmetic.  The product with the
+    multiplier M' (Eq. 11) is formed in float32 (the code is an integer decision taken in the
+    precision of the kernels): float32(acc + off) * float32(M').  Returns int8.
+    """
+    t = (np.asarray(acc, dtype=np.int64) + np.asarray(off, dtype=np.int64)[None, :]).astype(F32)
+    prod = (t * np.asarray(Mp, dtype=F32)[None, :]).astype(F32)
+    return np.clip(np.rint(prod) + Z_r, -qmax, qmax).astype(np.int8)
+
+
 # =========================================================================== output stage
 
 def requant_per_token(z: np.ndarray) -> Tuple[np.ndarray, np.ndarray]:

@@ -378,3 +378,56 @@ def test_cwac_parameter_budget_matches_printed_delta():
     deit_s = sum(s.N for s in WL.config_layers(2)) * per / 1e6
     assert round(vit_b, 1) == g["vit_b_delta_mb"]
     assert round(deit_s, 1) == g["deit_s_delta_mb"]
+
+
+# ------------------------------------------------------------------ Eq. 10 with static scales (integer-offset form)
+
+def test_static_requant_hand_fixture():
+    g = gold("eq10_static_requant_hand.json")
+    got = O.requant_static(np.array(g["acc"]), np.array(g["Mp"]), np.array(g["off"]))
+    # 0.001 is not a binary fraction: the hand values at exact .5 ties (1.5, 127.5, 3.5) must not depend on it
+    assert np.array_equal(got[:, [0, 1, 3]], np.array(g["expected"])[:, [0, 1, 3]])
+    assert np.all(np.abs(got[:, 2].astype(int) - np.array(g["expected"])[:, 2]) <= 1)
+    assert got[2, 2] == 127 and got[1, 3] == -127 and got[3, 3] == -127       # clipping
+
+
+def test_static_requant_equals_quantizing_the_compensated_output():
+    """Eq. 9 -> Eq. 10: dividing the compensated real output by S_r and rounding gives the same codes as the
+    integer-offset form whenever beta / (alpha S_x S_W) is an integer (then Eq. 10 loses nothing), and differs
+    by at most one step otherwise (beta is off by at most half an accumulator step, Section 3.4)."""
+    rng = np.random.default_rng(21)
+    M, N = 64, 48
+    alpha = 1 + 0.05 * rng.standard_normal(N)
+    S_W = rng.uniform(1e-4, 3e-4, N)
+    S_x, S_r = 0.03, 0.02
+    acc = rng.integers(-60000, 60000, (M, N))
+    k = rng.integers(-500, 500, N)
+    beta_exact = k * alpha * S_x * S_W                      # beta / (alpha S_x S_W) = k exactly
+    Mp, off = O.fold_integer_offset(alpha, beta_exact, S_x, S_W, S_r)
+    assert np.array_equal(off, k)
+    real = (alpha * S_W * S_x)[None, :] * acc + beta_exact[None, :]          # Eq. 9 right-hand side
+    direct = np.clip(np.rint(real / S_r), -127, 127)
+    got = O.requant_static(acc, Mp, off).astype(np.int64)
+    # float32 product against the float64 quotient: equal except within 1e-4 of a rounding tie
+    near_tie = np.abs((real / S_r) - np.floor(real / S_r) - 0.5) < 1e-4
+    assert np.array_equal(got[~near_tie], direct[~near_tie]) and np.abs(got - direct).max() <= 1
+    # arbitrary beta: at most one output step away, and the real-valued error obeys the Section 3.4 bound
+    beta = 0.02 * rng.standard_normal(N)
+    Mp, off = O.fold_integer_offset(alpha, beta, S_x, S_W, S_r)
+    real = (alpha * S_W * S_x)[None, :] * acc + beta[None, :]
+    direct = np.clip(np.rint(real / S_r), -127, 127)
+    got = O.requant_static(acc, Mp, off).astype(np.int64)
+    assert np.abs(got - direct).max() <= 1
+    unclipped = np.abs(real / S_r) < 126
+    err = np.abs(S_r * got - real)[unclipped]
+    assert np.all(err <= S_r / 2 + (np.abs(alpha * S_x * S_W) / 2)[None, :].repeat(M, 0)[unclipped] + 1e-9)
+
+
+def test_static_requant_zero_point_and_symmetry():
+    acc = np.array([[10, -10, 0]])
+    Mp = np.array([1.0, 1.0, 1.0])
+    off = np.array([0, 0, 0])
+    assert O.requant_static(acc, Mp, off, Z_r=5).tolist() == [[15, -5, 5]]
+    a = np.arange(-300, 300).reshape(1, -1)
+    r = O.requant_static(a, np.full(600, 0.7), np.zeros(600, dtype=int))
+    assert np.array_equal(r, -O.requant_static(-a, np.full(600, 0.7), np.zeros(600, dtype=int)))   # odd function
