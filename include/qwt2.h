@@ -46,7 +46,8 @@ enum { QWT_W_INT8 = 0,         /* [N, K] int8 codes in [-127, 127] */
 enum { QWT_OUT_INT8_PER_TOKEN = 0, /* int8 codes [M, N] + float y_scale[M] (dynamic per-token absmax) */
        QWT_OUT_BF16 = 1,           /* bfloat16 [M, N], round to nearest even */
        QWT_OUT_FP32 = 2,           /* float [M, N]: the compensated real-valued output z */
-       QWT_OUT_INT32_ACC = 3       /* int32 [M, N]: raw integer accumulators (verification) */ };
+       QWT_OUT_INT32_ACC = 3,      /* int32 [M, N]: raw integer accumulators (verification) */
+       QWT_OUT_INT8_STATIC = 4     /* int8 codes [M, N] with STATIC scales: Eq. 10 as printed (see qwt_cwac_fold_static) */ };
 
 const char* qwt_version(void);
 const char* qwt_status_string(qwt_status s);
@@ -128,6 +129,21 @@ qwt_status qwt_cwac_calibrate_noalloc(const float* fp_out, const float* q_out, i
 qwt_status qwt_cwac_fold(const float* w_scale, const float* bias, const float* a, const float* b, int32_t n,
                          float* fscale, float* fbias, void* stream);
 
+/* Fold for an engine with STATIC per-tensor scales -- Section 3.4, Eq. 10-11 exactly as printed (zero-points 0):
+ *     mult[n]   = a[n] * S_x * w_scale[n] / S_r                               (the multiplier M' of Eq. 11)
+ *     offset[n] = rne((a[n] * bias[n] + b[n]) / (a[n] * S_x * w_scale[n]))    (the rounded term of Eq. 10, INT32;
+ *                 the layer bias rides with beta because CWAC acts on the module output)
+ * computed in float64 on the device.  A channel whose a * S_x * w_scale is 0 gets offset 0.
+ * The forward call with QWT_OUT_INT8_STATIC then produces
+ *     Y[m, n] = clip(rne(mult[n] * (acc[m, n] + offset[n])), -127, 127)
+ * (the sum in exact integer arithmetic, the product in FP32), i.e. S_r * Y approximates the compensated output
+ * with beta off by at most half an accumulator step, |a S_x w_scale| / 2 (Section 3.4).
+ *   S_x, S_r > 0: static activation / output scales; bias [n] or NULL; a, b [n] or both NULL (= 1, 0)
+ *   mult float [n] out, offset int32 [n] out.
+ * Errors: NULL, SHAPE (n < 1, S_x <= 0, S_r <= 0), ARCH, CUDA. */
+qwt_status qwt_cwac_fold_static(const float* w_scale, const float* bias, const float* a, const float* b, int32_t n,
+                                float S_x, float S_r, float* mult, int32_t* offset, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Forward -- Section 3.4, Eq. 6-11 with all zero-points 0 (symmetric codes).
  *     acc[m, n] = sum_k X[m, k] * W[n, k]                       (int8 x int8 -> int32, exact; the W_q x_q of Eq. 7)
@@ -136,6 +152,9 @@ qwt_status qwt_cwac_fold(const float* w_scale, const float* bias, const float* a
  *                           (Eq. 1-2 applied to the output with zero-point 0: the 1/S_r of Eq. 10-11, per token);
  *                           a row of zeros gives y_scale 0 and codes 0.
  *   QWT_OUT_BF16 / FP32   : Y = z rounded to bfloat16 / as is.       QWT_OUT_INT32_ACC: Y = acc.
+ *   QWT_OUT_INT8_STATIC   : Y[m, n] = clip(rne(fscale[n] * (acc[m, n] + offset[n])), -127, 127) with fscale = mult and
+ *                           fbias = the INT32 offset array of qwt_cwac_fold_static passed through the same pointer
+ *                           (reinterpreted); x_scale and y_scale are not used (NULL).  No workspace traffic.
  *
  *   X [M, K] int8; x_scale [M] float (may be NULL for INT32_ACC)
  *   W [N, K] int8, or [N, K/2] packed int4 (expanded to int8 on chip)

@@ -23,7 +23,7 @@ QWT_OK, QWT_ERR_NULL, QWT_ERR_SHAPE, QWT_ERR_ALIGN, QWT_ERR_UNSUPPORTED = 0, 1, 
 QWT_ERR_WORKSPACE, QWT_ERR_CUDA, QWT_ERR_TIMEOUT, QWT_ERR_ARCH, QWT_ERR_TOO_LARGE = 5, 6, 7, 8, 9
 QWT_NOALLOC_SCRATCH_BYTES = 4 << 20
 QWT_W_INT8, QWT_W_INT4_PACKED = 0, 1
-QWT_OUT_INT8_PER_TOKEN, QWT_OUT_BF16, QWT_OUT_FP32, QWT_OUT_INT32_ACC = 0, 1, 2, 3
+QWT_OUT_INT8_PER_TOKEN, QWT_OUT_BF16, QWT_OUT_FP32, QWT_OUT_INT32_ACC, QWT_OUT_INT8_STATIC = 0, 1, 2, 3, 4
 
 _p, _i32, _i64, _sz = C.c_void_p, C.c_int32, C.c_int64, C.c_size_t
 
@@ -40,6 +40,7 @@ SIGNATURES = {
     "qwt_cwac_calibrate_host": (_i32, [_p, _p, _i64, _i32, _i64, _p, _p, _p, _p, _sz, _p]),
     "qwt_cwac_calibrate_noalloc": (_i32, [_p, _p, _i64, _i32, _i64, _p, _p, _p, _p]),
     "qwt_cwac_fold": (_i32, [_p, _p, _p, _p, _i32, _p, _p, _p]),
+    "qwt_cwac_fold_static": (_i32, [_p, _p, _p, _p, _i32, C.c_float, C.c_float, _p, _p, _p]),
     "qwt_qlinear_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32, _i32]),
     "qwt_qlinear_cwac_forward": (_i32, [_p, _p, _p, _i32, _p, _p, _i32, _i32, _i32, _i32, _p, _p, _p, _sz, _p]),
     "qwt_qlinear_check_status": (_i32, [_p, _p, C.POINTER(_i32)]),
@@ -161,6 +162,14 @@ def qwt_cwac_fold(w_scale, bias, a, b, n, fscale, fbias, stream=None, check=True
     s = lib.qwt_cwac_fold(_ptr(w_scale), _ptr(bias), _ptr(a), _ptr(b), n, _ptr(fscale), _ptr(fbias), _stream(stream))
     if check:
         _check(s, "qwt_cwac_fold")
+    return s
+
+
+def qwt_cwac_fold_static(w_scale, bias, a, b, n, S_x, S_r, mult, offset, stream=None, check=True) -> int:
+    s = lib.qwt_cwac_fold_static(_ptr(w_scale), _ptr(bias), _ptr(a), _ptr(b), n, S_x, S_r, _ptr(mult), _ptr(offset),
+                                 _stream(stream))
+    if check:
+        _check(s, "qwt_cwac_fold_static")
     return s
 
 

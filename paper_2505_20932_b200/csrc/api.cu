@@ -246,6 +246,17 @@ qwt_status qwt_cwac_fold(const float* w_scale, const float* bias, const float* a
   return launch_cwac_fold(w_scale, bias, a, b, n, fscale, fbias, as_stream(stream));
 }
 
+qwt_status qwt_cwac_fold_static(const float* w_scale, const float* bias, const float* a, const float* b, int32_t n,
+                                float S_x, float S_r, float* mult, int32_t* offset, void* stream) {
+  if (w_scale == nullptr || mult == nullptr || offset == nullptr) return QWT_ERR_NULL;
+  if ((a == nullptr) != (b == nullptr)) return QWT_ERR_NULL;
+  if (n < 1 || !(S_x > 0.f) || !(S_r > 0.f)) return QWT_ERR_SHAPE;
+  DeviceInfo dev;
+  qwt_status s = current_device(&dev);
+  if (s != QWT_OK) return s;
+  return launch_cwac_fold_static(w_scale, bias, a, b, n, S_x, S_r, mult, offset, as_stream(stream));
+}
+
 // ------------------------------------------------------------------------------------------------ forward
 
 static qwt_status check_forward_args(const void* X, const float* x_scale, const void* W, int32_t wfmt,
@@ -253,16 +264,17 @@ static qwt_status check_forward_args(const void* X, const float* x_scale, const 
                                      int32_t out_mode, const void* Y, const float* y_scale, bool host_io) {
   if (X == nullptr || W == nullptr || Y == nullptr) return QWT_ERR_NULL;
   if (wfmt != QWT_W_INT8 && wfmt != QWT_W_INT4_PACKED) return QWT_ERR_UNSUPPORTED;
-  if (out_mode < QWT_OUT_INT8_PER_TOKEN || out_mode > QWT_OUT_INT32_ACC) return QWT_ERR_UNSUPPORTED;
-  if (out_mode != QWT_OUT_INT32_ACC && (x_scale == nullptr || fscale == nullptr || fbias == nullptr))
-    return QWT_ERR_NULL;
+  if (out_mode < QWT_OUT_INT8_PER_TOKEN || out_mode > QWT_OUT_INT8_STATIC) return QWT_ERR_UNSUPPORTED;
+  if (out_mode != QWT_OUT_INT32_ACC && (fscale == nullptr || fbias == nullptr)) return QWT_ERR_NULL;
+  if (out_mode != QWT_OUT_INT32_ACC && out_mode != QWT_OUT_INT8_STATIC && x_scale == nullptr) return QWT_ERR_NULL;
   if (out_mode == QWT_OUT_INT8_PER_TOKEN && y_scale == nullptr) return QWT_ERR_NULL;
   if (M < 1 || N < 1 || K < 1) return QWT_ERR_SHAPE;
   if ((int64_t)M * (int64_t)N >= (int64_t)1 << 40) return QWT_ERR_SHAPE;
   if (K > 131072) return QWT_ERR_SHAPE;   // 127^2 * K must stay below 2^31
   const int kmul = wfmt == QWT_W_INT8 ? 16 : 32;
   if (K % kmul != 0) return QWT_ERR_UNSUPPORTED;
-  const int nmul = out_mode == QWT_OUT_INT8_PER_TOKEN ? 16 : (out_mode == QWT_OUT_BF16 ? 8 : 4);
+  const bool codes = out_mode == QWT_OUT_INT8_PER_TOKEN || out_mode == QWT_OUT_INT8_STATIC;
+  const int nmul = codes ? 16 : (out_mode == QWT_OUT_BF16 ? 8 : 4);
   if (N % nmul != 0) return QWT_ERR_UNSUPPORTED;
   if (!aligned(W, 16)) return QWT_ERR_ALIGN;
   if (!host_io && (!aligned(X, 16) || !aligned(Y, 16))) return QWT_ERR_ALIGN;
@@ -314,7 +326,8 @@ struct HostFwdLayout {
 HostFwdLayout host_fwd_layout(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode) {
   HostFwdLayout L{};
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
-  const size_t esz = out_mode == QWT_OUT_INT8_PER_TOKEN ? 1 : (out_mode == QWT_OUT_BF16 ? 2 : 4);
+  const size_t esz = (out_mode == QWT_OUT_INT8_PER_TOKEN || out_mode == QWT_OUT_INT8_STATIC)
+                         ? 1 : (out_mode == QWT_OUT_BF16 ? 2 : 4);
   L.x_bytes = (size_t)M * K;
   L.y_bytes = (size_t)M * N * esz;
   size_t off = 0;

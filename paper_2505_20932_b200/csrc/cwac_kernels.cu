@@ -227,6 +227,22 @@ cwac_fold_kernel(const float* __restrict__ w_scale, const float* __restrict__ bi
   fbias[i] = fmaf(ai, bs, bi);
 }
 
+// Eq. 10-11 as printed, static scales: multiplier M' and the rounded accumulator offset, in float64.
+__global__ void __launch_bounds__(256)
+cwac_fold_static_kernel(const float* __restrict__ w_scale, const float* __restrict__ bias, const float* __restrict__ a,
+                        const float* __restrict__ b, int n, double S_x, double S_r, float* __restrict__ mult,
+                        int32_t* __restrict__ offset) {
+  const int i = blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n) return;
+  const double ai = a ? (double)a[i] : 1.0;
+  const double bi = b ? (double)b[i] : 0.0;
+  const double bs = bias ? (double)bias[i] : 0.0;
+  const double step = ai * S_x * (double)w_scale[i];      // real value of one accumulator step after compensation
+  mult[i] = (float)(step / S_r);
+  const double off = step != 0.0 ? rint((ai * bs + bi) / step) : 0.0;
+  offset[i] = (int32_t)fmin(fmax(off, -2147483647.0), 2147483647.0);
+}
+
 // Eq. 1-2 with zero-point 0: one warp per row, two passes over the row (the second hits cache).
 __global__ void __launch_bounds__(256)
 quantize_rows_kernel(const float* __restrict__ X, int64_t rows, int cols, int64_t ld, float qmax,
@@ -325,6 +341,14 @@ qwt_status launch_cwac_solve(const double* stats, int32_t channels, float* a, fl
 qwt_status launch_cwac_fold(const float* w_scale, const float* bias, const float* a, const float* b, int32_t n,
                             float* fscale, float* fbias, cudaStream_t st) {
   cwac_fold_kernel<<<(n + 255) / 256, 256, 0, st>>>(w_scale, bias, a, b, n, fscale, fbias);
+  QWT_LAUNCH_CHECK();
+  return QWT_OK;
+}
+
+qwt_status launch_cwac_fold_static(const float* w_scale, const float* bias, const float* a, const float* b, int32_t n,
+                                   float S_x, float S_r, float* mult, int32_t* offset, cudaStream_t st) {
+  cwac_fold_static_kernel<<<(n + 255) / 256, 256, 0, st>>>(w_scale, bias, a, b, n, (double)S_x, (double)S_r, mult,
+                                                          offset);
   QWT_LAUNCH_CHECK();
   return QWT_OK;
 }

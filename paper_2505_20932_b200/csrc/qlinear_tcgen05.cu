@@ -93,9 +93,11 @@ struct QlParams {
 // Compile-time geometry of one instantiation.
 template <int BN, int OUT, bool W4, bool WIDE>
 struct Cfg {
-  static constexpr bool kInt8Out = OUT == QWT_OUT_INT8_PER_TOKEN;
+  static constexpr bool kInt8Out = OUT == QWT_OUT_INT8_PER_TOKEN;     // dynamic per-token scale: two-phase epilogue
+  static constexpr bool kStatic8 = OUT == QWT_OUT_INT8_STATIC;       // Eq. 10 as printed: static multiplier + offset
+  static constexpr bool kCodes = kInt8Out || kStatic8;               // one byte per output element
   static constexpr bool kHasParams = OUT != QWT_OUT_INT32_ACC;       // x_scale / fscale / fbias are used
-  static constexpr int kEsz = kInt8Out ? 1 : (OUT == QWT_OUT_BF16 ? 2 : 4);
+  static constexpr int kEsz = kCodes ? 1 : (OUT == QWT_OUT_BF16 ? 2 : 4);
   static constexpr int kAcc = kTmemCols / BN;                        // accumulator buffers (tiles) in TMEM
   static constexpr int kUPT = BN / kUnitN;                           // epilogue units per tile
   static constexpr int kConvWarp0 = 2 + kEpiWarps;                   // first converter warp (W4 only)
@@ -412,7 +414,12 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       for (int i = 0; i < kUnitN / 32; ++i) {
         const int c = n0 + i * 32 + lane;
         pre_fs[i] = c < p.N ? __ldg(p.fscale + c) * (W4 ? 0.0625f : 1.0f) : 0.f;   // W4 operands hold 16 x code
-        pre_fb[i] = c < p.N ? __ldg(p.fbias + c) : 0.f;
+        if (C::kStatic8) {   // integer accumulator offsets travel as bit patterns (x16 with the x16 W4 operands)
+          const int o = c < p.N ? __ldg(reinterpret_cast<const int*>(p.fbias) + c) : 0;
+          pre_fb[i] = __int_as_float(W4 ? o * 16 : o);
+        } else {
+          pre_fb[i] = c < p.N ? __ldg(p.fbias + c) : 0.f;
+        }
       }
     };
     if (C::kHasParams && lead && g < n_units) prefetch_params(g);
@@ -433,7 +440,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int r = i * RPI + lane / CPR;
         uint4 v = *reinterpret_cast<const uint4*>(stg + r * BOXB + ((chunk ^ swizzle_xor<BOXB>(r)) << 4));
         // INT8 boxes: rows 8-15 and 24-31 were written with the 8-byte halves of every chunk exchanged
-        if (C::kInt8Out && (r & 8) != 0) v = make_uint4(v.z, v.w, v.x, v.y);
+        if (C::kCodes && (r & 8) != 0) v = make_uint4(v.z, v.w, v.x, v.y);
         if (col_ok && y + r < p.M) *reinterpret_cast<uint4*>(out + (size_t)(y + r) * p.N * ESZ) = v;
       }
       __syncwarp();                                  // the slot may be rewritten
@@ -448,7 +455,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint32_t buf = j % kAcc, tpar = (j / kAcc) & 1u, upar = use & 1u;
       const int y0 = tm * kBM + qd * 32;
       float xs4[4] = {0.f, 0.f, 0.f, 0.f};    // x_scale of the thread's four rows, requested before the waits below
-      if (C::kHasParams) {
+      if (C::kHasParams && !C::kStatic8) {
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const int r = y0 + (lane >> 2) + 8 * k;
@@ -494,6 +501,18 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       auto z_block = [&](const uint32_t* a0, const uint32_t* a1, int col, float2 (&z)[4]) {
         const float2 f2 = *reinterpret_cast<const float2*>(ps_fs + col + 2 * c);
         const float2 b2 = *reinterpret_cast<const float2*>(ps_fb + col + 2 * c);
+        if (C::kStatic8) {
+          // Eq. 10: M' (acc + offset); the sum is exact integer arithmetic, the product one FP32 rounding
+          const int o0 = __float_as_int(b2.x), o1 = __float_as_int(b2.y);
+          auto mo = [&](uint32_t x0, uint32_t x1) {
+            return __fmul2_rn(make_float2(__int2float_rn((int)x0 + o0), __int2float_rn((int)x1 + o1)), f2);
+          };
+          z[0] = mo(a0[0], a0[1]);
+          z[1] = mo(a0[2], a0[3]);
+          z[2] = mo(a1[0], a1[1]);
+          z[3] = mo(a1[2], a1[3]);
+          return;
+        }
         z[0] = z_pair(a0[0], a0[1], xs2[0], f2.x, f2.y, b2.x, b2.y);     // columns >= N give 0 * 0 + 0
         z[1] = z_pair(a0[2], a0[3], xs2[1], f2.x, f2.y, b2.x, b2.y);
         z[2] = z_pair(a1[0], a1[1], xs2[2], f2.x, f2.y, b2.x, b2.y);
@@ -654,7 +673,9 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const float2 magic2 = make_float2(12582912.f, 12582912.f);
           auto quant = [&](float2 z, int k) -> uint32_t {      // two codes in the low 16 bits
             float2 qq;
-            if (SLOW) {
+            if (C::kStatic8) {      // already in output steps: clip to the code range, then round
+              qq = make_float2(fminf(fmaxf(z.x, -127.f), 127.f), fminf(fmaxf(z.y, -127.f), 127.f));
+            } else if (SLOW) {
               qq = make_float2(__fdiv_rn(z.x, den[k]), __fdiv_rn(z.y, den[k]));
             } else {
               const float2 i2 = make_float2(inv[k], inv[k]);
@@ -859,6 +880,8 @@ qwt_status launch_bn(int out_mode, const CUtensorMap& tmA, const CUtensorMap& tm
       return launch_inst<BN, QWT_OUT_FP32, W4>(tmA, tmB, prm, grid, want_resident, st);
     case QWT_OUT_INT32_ACC:
       return launch_inst<BN, QWT_OUT_INT32_ACC, W4>(tmA, tmB, prm, grid, want_resident, st);
+    case QWT_OUT_INT8_STATIC:
+      return launch_inst<BN, QWT_OUT_INT8_STATIC, W4>(tmA, tmB, prm, grid, want_resident, st);
   }
   return QWT_ERR_UNSUPPORTED;
 }

@@ -59,6 +59,8 @@ qwt_status launch_cwac_solve(const double* stats, int32_t channels, float* a, fl
                              cudaStream_t st);
 qwt_status launch_cwac_fold(const float* w_scale, const float* bias, const float* a, const float* b, int32_t n,
                             float* fscale, float* fbias, cudaStream_t st);
+qwt_status launch_cwac_fold_static(const float* w_scale, const float* bias, const float* a, const float* b, int32_t n,
+                                   float S_x, float S_r, float* mult, int32_t* offset, cudaStream_t st);
 qwt_status launch_quantize_rows(const float* X, int64_t rows, int32_t cols, int64_t ld, int32_t qmax, int8_t* Xq,
                                 float* scale, cudaStream_t st);
 qwt_status launch_pack_int4(const int8_t* codes, int64_t rows, int32_t cols, uint8_t* packed, cudaStream_t st);

@@ -81,7 +81,17 @@ def gpu_fold(ws_, bias, a, b):
 
 
 _OUT_DTYPE = {B.QWT_OUT_INT8_PER_TOKEN: torch.int8, B.QWT_OUT_BF16: torch.bfloat16,
-              B.QWT_OUT_FP32: torch.float32, B.QWT_OUT_INT32_ACC: torch.int32}
+              B.QWT_OUT_FP32: torch.float32, B.QWT_OUT_INT32_ACC: torch.int32, B.QWT_OUT_INT8_STATIC: torch.int8}
+
+
+def gpu_fold_static(ws_, bias, a, b, S_x, S_r):
+    n = ws_.shape[0]
+    mult = torch.empty(n, dtype=torch.float32, device=DEV)
+    off = torch.empty(n, dtype=torch.int32, device=DEV)
+    B.qwt_cwac_fold_static(dev(ws_), None if bias is None else dev(bias), None if a is None else dev(a),
+                           None if b is None else dev(b), n, float(S_x), float(S_r), mult, off)
+    torch.cuda.synchronize()
+    return mult.cpu().numpy(), off.cpu().numpy()
 
 
 def gpu_forward(Xq, xs, W, fs, fb, out_mode, wfmt=B.QWT_W_INT8, K=None, check_guard=True):
@@ -93,7 +103,8 @@ def gpu_forward(Xq, xs, W, fs, fb, out_mode, wfmt=B.QWT_W_INT8, K=None, check_gu
     dX, dW = dev(Xq), dev(W)
     dxs = None if xs is None else dev(xs.astype(np.float32))
     dfs = None if fs is None else dev(fs.astype(np.float32))
-    dfb = None if fb is None else dev(fb.astype(np.float32))
+    # static INT8 mode: the "fbias" pointer carries the INT32 accumulator offsets
+    dfb = None if fb is None else dev(fb.astype(np.int32) if out_mode == B.QWT_OUT_INT8_STATIC else fb.astype(np.float32))
     dt = _OUT_DTYPE[out_mode]
     guard = 64
     Ybuf = torch.zeros(M * N + 2 * guard, dtype=dt, device=DEV)
