@@ -85,6 +85,20 @@ def config_layers(cfg: int, full: bool = True) -> List[LayerSpec]:
     raise ValueError(f"no forward layers for config {cfg}")
 
 
+def resnet50_pointwise_layers(batch: int = 32, calib_images: int = 32) -> List[LayerSpec]:
+    """ResNet-50 shaped 1x1 convolutions (the paper also places CWAC after every quantized convolution, Section 3.3
+    and Table 1).  In NHWC layout a 1x1 convolution over a B x H x W x C_in activation IS this linear layer with
+    M = B*H*W tokens, K = C_in, N = C_out, so no new kernel is involved: these shapes only widen the workload set
+    (first and last pointwise convolution of a bottleneck in each of the four stages)."""
+    out: List[LayerSpec] = []
+    for stage, (hw, cin, mid, cout) in enumerate([(56, 256, 64, 256), (28, 512, 128, 512), (14, 1024, 256, 1024),
+                                                  (7, 2048, 512, 2048)]):
+        M, R = batch * hw * hw, calib_images * hw * hw
+        out.append(LayerSpec(f"resnet50.s{stage}.reduce", M, cin, mid, 8, "int8", "lognormal_channel", R))
+        out.append(LayerSpec(f"resnet50.s{stage}.expand", M, mid, cout, 8, "int8", "lognormal_channel", R))
+    return out
+
+
 CALIB_SWEEP_ROWS = 2048 * TOKENS_PER_IMAGE   # config 5: 403,456 rows
 CALIB_SWEEP_WIDTHS = (768, 2304, 3072)
 CALIB_SWEEP_BITS = (8, 4)

@@ -235,3 +235,25 @@ def test_w4_quantize_pack_forward_chain(H, B):
     z_ref = O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb)
     dd = np.abs(bits.astype(np.int32) - O.to_bf16_bits(z_ref).astype(np.int32))
     assert dd.max() <= 1 and np.count_nonzero(dd) <= max(1, int(1e-4 * dd.size))
+
+
+# ------------------------------------------------------------------ CNN-shaped layers (1x1 convolutions)
+
+def test_resnet50_pointwise_convolutions(H, B):
+    """A 1x1 convolution in NHWC layout is the same quantized linear layer (M = B*H*W, K = C_in, N = C_out):
+    ResNet-50 bottleneck shapes at a small batch, quantize -> forward in both INT8 modes, against the oracle."""
+    for spec in WL.resnet50_pointwise_layers(batch=1, calib_images=1):
+        if spec.M > 1600:
+            spec = WL.LayerSpec(spec.name, 1600, spec.K, spec.N, 8, "int8", spec.act, 64)
+        d = WL.host_layer_inputs(spec, seed=11, calib_rows=8)
+        Xq, xs = O.quantize_rows_sym(d["X"], 127)
+        Wq, ws = O.quantize_rows_sym(d["W"], 127)
+        fs, fb = O.cwac_fold(ws, d["bias"], None, None)
+        fs, fb = fs.astype(np.float32), fb.astype(np.float32)
+        acc = O.int_matmul(Xq, Wq)
+        codes, ys = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_INT8_PER_TOKEN)
+        c_ref, ys_ref = O.requant_per_token(O.forward_folded(acc, xs, fs, fb))
+        assert np.allclose(ys, ys_ref, rtol=1e-5), spec.name
+        assert_codes_close(codes, c_ref, spec.name)
+        raw, _ = H.gpu_forward(Xq, None, Wq, None, None, B.QWT_OUT_INT32_ACC)
+        assert np.array_equal(raw.astype(np.int64), acc), spec.name
