@@ -464,6 +464,29 @@ def run_ours(args):
                "what": "phase B through qwt_qlinear_cwac_forward_host: pinned host X/x_scale in, host Y/y_scale out, per layer"}
         del staging, host
 
+    # ---- an on-box INT8 reference point: the library's plain int8 x int8 -> int32 matmul (no epilogue) at 8192^3,
+    # timed outside the timed region.  Context for the "% INT8 peak" figures, not part of the path.
+    lib_int8_tops = None
+    if rank == 0 and not args.no_library_int8:
+        try:
+            a8 = torch.randint(-127, 128, (8192, 8192), dtype=torch.int8, device=device)
+            b8 = torch.randint(-127, 128, (8192, 8192), dtype=torch.int8, device=device).t()
+            for _ in range(3):
+                torch._int_mm(a8, b8)
+            best = None
+            for _ in range(5):
+                q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                q0.record()
+                torch._int_mm(a8, b8)
+                q1.record()
+                torch.cuda.synchronize()
+                t = q0.elapsed_time(q1) * 1e-3
+                best = t if best is None else min(best, t)
+            lib_int8_tops = 2 * 8192 ** 3 / best / 1e12
+            del a8, b8
+        except Exception:
+            lib_int8_tops = None
+
     # ---- rooflines
     int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
     int8_peak_sus = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
@@ -519,6 +542,7 @@ def run_ours(args):
             "forward": {"ms_per_step": t_b / args.steps * 1e3, "frac_int8_peak_burst": fwd_tops_gpu / int8_peak,
                         "frac_int8_peak_sustained": fwd_tops_gpu / int8_peak_sus,
                         "frac_int8_datasheet_4500": fwd_tops_gpu / 4500.0,
+                        "library_int8_matmul_8192_tops": lib_int8_tops,
                         "min_time_ms": max(t_min_compute, t_min_hbm) * 1e3,
                         "frac_of_roofline": max(t_min_compute, t_min_hbm) / (t_b / args.steps)},
             "roofline": dominant, "rooflines": [roof_cal, roof_fwd],
@@ -544,6 +568,7 @@ def main():
     ap.add_argument("--out", default="", choices=["", "int8", "bf16"], help="override the output stage")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-library-int8", action="store_true", help="skip timing the library int8 matmul reference point")
     ap.add_argument("--no-graph", action="store_true", help="issue every library call from the host in the timed region")
     ap.add_argument("--no-cpu", action="store_true")
     ap.add_argument("--cpu-rows", type=int, default=4096)
