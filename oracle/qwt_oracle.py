@@ -123,6 +123,32 @@ def qlinear_eq7(Wq: np.ndarray, xq: np.ndarray, Zw: np.ndarray, Zx: int) -> np.n
     return Wq @ xq - Zw * xq.sum() - Zx * Wq.sum(axis=1) + K * Zx * Zw
 
 
+def quantize_rows_asym(X: np.ndarray, bits: int = 8) -> Tuple[np.ndarray, np.ndarray, np.ndarray]:
+    """Eq. 1-2 applied to every row on its own (per token for activations, per output channel for weights):
+    unsigned codes in [0, 2^b - 1], scale s_r = (max_r - min_r) / (2^b - 1), zero-point
+    z_r = clip(round(-min_r / s_r), 0, 2^b - 1).  The quotients are formed in float32 (integer decisions).
+    A constant row gets scale 1 (Eq. 2 would give 0).  Returns (codes uint8, scale float32, zero int32)."""
+    X = np.ascontiguousarray(X, dtype=F32)
+    qmax = F32(2 ** bits - 1)
+    lo = X.min(axis=1).astype(F32)
+    hi = X.max(axis=1).astype(F32)
+    s = ((hi - lo) / qmax).astype(F32)
+    s = np.where(s > 0, s, F32(1.0)).astype(F32)
+    z = np.clip(np.rint((-lo / s).astype(F32)), 0, qmax).astype(np.int32)
+    q = np.clip(np.rint((X / s[:, None]).astype(F32)) + z[:, None].astype(F32), 0, qmax)
+    return q.astype(np.uint8), s, z
+
+
+def int_matmul_asym(Xq: np.ndarray, Zx: np.ndarray, Wq: np.ndarray, Zw: np.ndarray) -> np.ndarray:
+    """The bracket of Eq. 6 by its definition: acc[m, n] = sum_k (Wq[n, k] - Zw[n]) (Xq[m, k] - Zx[m]),
+    exact (float64 product of small integers, every partial sum below 2^53).  Zx per row (a scalar broadcasts:
+    the paper's per-tensor activation zero-point), Zw per output channel."""
+    Xc = np.asarray(Xq, dtype=F64) - np.broadcast_to(np.asarray(Zx, dtype=F64), (np.shape(Xq)[0],))[:, None]
+    Wc = np.asarray(Wq, dtype=F64) - np.asarray(Zw, dtype=F64)[:, None]
+    assert 256 * 256 * Xc.shape[1] < 2 ** 53
+    return (Xc @ Wc.T).astype(np.int64)
+
+
 def dequant(acc: np.ndarray, x_scale: np.ndarray, w_scale: np.ndarray,
             bias: Optional[np.ndarray]) -> np.ndarray:
     """Eq. 6 with all zero-points 0: real-valued layer output

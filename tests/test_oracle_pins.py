@@ -431,3 +431,51 @@ def test_static_requant_zero_point_and_symmetry():
     a = np.arange(-300, 300).reshape(1, -1)
     r = O.requant_static(a, np.full(600, 0.7), np.zeros(600, dtype=int))
     assert np.array_equal(r, -O.requant_static(-a, np.full(600, 0.7), np.zeros(600, dtype=int)))   # odd function
+
+
+# ------------------------------------------------------------------ asymmetric codes (Eq. 1-2 and Eq. 6-7 in full)
+
+def test_rowwise_asymmetric_quantizer_is_eq1_eq2_per_row():
+    rng = np.random.default_rng(31)
+    X = (rng.standard_normal((6, 50)) * rng.lognormal(0, 1, (6, 1)) + rng.normal(0, 2, (6, 1))).astype(np.float32)
+    q, s, z = O.quantize_rows_asym(X, 8)
+    for r in range(X.shape[0]):
+        qr, sr, zr = O.uniform_quantize(X[r], 8)           # the per-tensor form pinned by the hand fixture
+        assert z[r] == zr and s[r] == pytest.approx(sr, rel=1e-6)
+        assert np.abs(q[r].astype(int) - qr).max() <= 1    # float32 vs float64 quotient: at most a tie apart
+        assert np.count_nonzero(q[r].astype(int) - qr) <= 1
+    assert q.min() == 0 and q.max() == 255                 # the extremes of a row take the end codes
+    back = s[:, None] * (q.astype(np.float64) - z[:, None])
+    # half a step from rounding x, half from rounding the zero-point, one more where the shifted end code clips
+    assert np.all(np.abs(back - X) <= 2.0 * s[:, None] * (1 + 1e-3))
+    assert np.mean(np.abs(back - X) <= s[:, None] * (1 + 1e-3)) > 0.97
+    qc, sc, zc = O.quantize_rows_asym(np.full((1, 8), 3.0, np.float32))
+    assert sc[0] == 1.0 and np.all(qc == qc[0, 0])
+
+
+def test_asymmetric_product_equals_eq7_expansion_and_brute_force():
+    rng = np.random.default_rng(32)
+    M, N, K = 5, 7, 48
+    Xq = rng.integers(0, 256, (M, K)).astype(np.uint8)
+    Wq = rng.integers(0, 256, (N, K)).astype(np.uint8)
+    Zx = rng.integers(0, 256, M)
+    Zw = rng.integers(0, 256, N)
+    acc = O.int_matmul_asym(Xq, Zx, Wq, Zw)
+    brute = np.zeros((M, N), dtype=np.int64)
+    for m in range(M):
+        for n in range(N):
+            for k in range(K):
+                brute[m, n] += (int(Wq[n, k]) - int(Zw[n])) * (int(Xq[m, k]) - int(Zx[m]))
+    assert np.array_equal(acc, brute)
+    for m in range(M):                                     # Eq. 7's four terms, pinned separately by eq7_hand.json
+        assert np.array_equal(acc[m], O.qlinear_eq7(Wq, Xq[m], Zw, int(Zx[m])))
+    # zero zero-points: the symmetric product
+    assert np.array_equal(O.int_matmul_asym(Xq, 0, Wq, np.zeros(N)), O.int_matmul(Xq.astype(np.int64), Wq.astype(np.int64)))
+    # the real-valued product is recovered: S_W (W_q - Z_W) S_x (x_q - Z_x) ~ W x  (Eq. 6)
+    X = rng.standard_normal((20, 64)).astype(np.float32) + 1.0
+    W = (0.02 * rng.standard_normal((12, 64))).astype(np.float32)
+    xq, xs, xz = O.quantize_rows_asym(X)
+    wq, ws, wz = O.quantize_rows_asym(W)
+    y = O.int_matmul_asym(xq, xz, wq, wz) * xs[:, None].astype(np.float64) * ws[None, :]
+    ref = X.astype(np.float64) @ W.astype(np.float64).T
+    assert np.abs(y - ref).max() < 0.02 * np.abs(ref).max() + 1e-3
