@@ -446,9 +446,14 @@ def test_rowwise_asymmetric_quantizer_is_eq1_eq2_per_row():
         assert np.count_nonzero(q[r].astype(int) - qr) <= 1
     assert q.min() == 0 and q.max() == 255                 # the extremes of a row take the end codes
     back = s[:, None] * (q.astype(np.float64) - z[:, None])
-    # half a step from rounding x, half from rounding the zero-point, one more where the shifted end code clips
-    assert np.all(np.abs(back - X) <= 2.0 * s[:, None] * (1 + 1e-3))
-    assert np.mean(np.abs(back - X) <= s[:, None] * (1 + 1e-3)) > 0.97
+    # rows whose range contains 0: half a step from rounding x, half from rounding the zero-point, one more where
+    # the shifted end code clips.  Rows that lie on one side of 0 have their zero-point clipped by Eq. 2 and are
+    # represented badly -- that is the quantizer as printed, kept as is.
+    spans0 = (X.min(axis=1) <= 0) & (X.max(axis=1) >= 0)
+    assert spans0.sum() >= 3 and (~spans0).sum() >= 1
+    err = np.abs(back - X) / s[:, None]
+    assert np.all(err[spans0] <= 2.0 * (1 + 1e-3)) and np.mean(err[spans0] <= 1 + 1e-3) > 0.97
+    assert np.all(np.isin(z[~spans0], (0, 255)))
     qc, sc, zc = O.quantize_rows_asym(np.full((1, 8), 3.0, np.float32))
     assert sc[0] == 1.0 and np.all(qc == qc[0, 0])
 
