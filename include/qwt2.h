@@ -198,6 +198,35 @@ qwt_status qwt_quantize_rows_i8(const float* X, int64_t rows, int32_t cols, int6
                                 int8_t* Xq, float* scale, void* stream);
 qwt_status qwt_pack_int4(const int8_t* codes, int64_t rows, int32_t cols, uint8_t* packed, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Asymmetric (unsigned) codes -- Eq. 1-2 and Eq. 6-7 as printed, with non-zero zero-points:
+ *     acc[m, n] = sum_k (W_q[n, k] - Z_W[n]) (x_q[m, k] - Z_x[m])
+ *               = sum_k W_q x_q  -  Z_W[n] sum_k x_q[m, k]  -  Z_x[m] sum_k W_q[n, k]  +  K Z_x[m] Z_W[n]      (Eq. 7)
+ * (codes in [0, 255]; Z_x per token -- pass the same value for every token for the paper's per-tensor activation
+ * zero-point -- and Z_W per output channel).  The unsigned product runs on the tensor cores, the three zero-point
+ * terms are added in the epilogue in exact integer arithmetic; everything after that (x_scale, fscale, fbias, the
+ * output stages) is as in qwt_qlinear_cwac_forward.
+ *
+ * qwt_quantize_rows_u8   Eq. 1-2 per row: scale[r] = (max - min) / 255 (1 for a constant row),
+ *                        zero[r] = clip(rne(-min / scale), 0, 255), Xq = clip(rne(x / scale) + zero, 0, 255);
+ *                        rowsum[r] = sum_c Xq[r, c] (may be NULL).  Rows = tokens for activations, output
+ *                        channels for weights.
+ * qwt_asym_weight_terms  w_terms int32 [2 N]: w_terms[n] = -Z_W[n], w_terms[N + n] = K Z_W[n] - sum_k W_q[n, k];
+ *                        computed once per layer.
+ * qwt_qlinear_cwac_forward_asym   X uint8 [M, K], x_zero / x_rowsum int32 [M], W uint8 [N, K] (no packed int4),
+ *                        out_mode any but QWT_OUT_INT8_STATIC; K <= 33000; other arguments, workspace and errors as
+ *                        for qwt_qlinear_cwac_forward.
+ */
+qwt_status qwt_quantize_rows_u8(const float* X, int64_t rows, int32_t cols, int64_t ld, uint8_t* Xq, float* scale,
+                                int32_t* zero, int32_t* rowsum, void* stream);
+qwt_status qwt_asym_weight_terms(const uint8_t* W, const int32_t* w_zero, int32_t N, int32_t K, int32_t* w_terms,
+                                 void* stream);
+qwt_status qwt_qlinear_cwac_forward_asym(const uint8_t* X, const float* x_scale, const int32_t* x_zero,
+                                         const int32_t* x_rowsum, const uint8_t* W, const int32_t* w_terms,
+                                         const float* fscale, const float* fbias, int32_t M, int32_t N, int32_t K,
+                                         int32_t out_mode, void* Y, float* y_scale, void* workspace,
+                                         size_t workspace_bytes, void* stream);
+
 /* Kernels launched by this library on the calling thread since the last reset (for launch accounting). */
 int64_t qwt_launch_count(void);
 void qwt_launch_count_reset(void);

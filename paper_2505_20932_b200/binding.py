@@ -46,6 +46,9 @@ SIGNATURES = {
     "qwt_qlinear_check_status": (_i32, [_p, _p, C.POINTER(_i32)]),
     "qwt_qlinear_host_staging_bytes": (_sz, [_i32, _i32, _i32, _i32, _i32]),
     "qwt_qlinear_cwac_forward_host": (_i32, [_p, _p, _p, _i32, _p, _p, _i32, _i32, _i32, _i32, _p, _p, _p, _sz, _p]),
+    "qwt_quantize_rows_u8": (_i32, [_p, _i64, _i32, _i64, _p, _p, _p, _p, _p]),
+    "qwt_asym_weight_terms": (_i32, [_p, _p, _i32, _i32, _p, _p]),
+    "qwt_qlinear_cwac_forward_asym": (_i32, [_p, _p, _p, _p, _p, _p, _p, _p, _i32, _i32, _i32, _i32, _p, _p, _p, _sz, _p]),
     "qwt_quantize_rows_i8": (_i32, [_p, _i64, _i32, _i64, _i32, _p, _p, _p]),
     "qwt_pack_int4": (_i32, [_p, _i64, _i32, _p, _p]),
     "qwt_launch_count": (_i64, []),
@@ -206,6 +209,30 @@ def qwt_qlinear_cwac_forward_host(X, x_scale, W, wfmt, fscale, fbias, M, N, K, o
                                           _stream(stream))
     if check:
         _check(s, "qwt_qlinear_cwac_forward_host")
+    return s
+
+
+def qwt_quantize_rows_u8(X, rows, cols, ld, Xq, scale, zero, rowsum, stream=None, check=True) -> int:
+    s = lib.qwt_quantize_rows_u8(_ptr(X), rows, cols, ld, _ptr(Xq), _ptr(scale), _ptr(zero), _ptr(rowsum), _stream(stream))
+    if check:
+        _check(s, "qwt_quantize_rows_u8")
+    return s
+
+
+def qwt_asym_weight_terms(W, w_zero, N, K, w_terms, stream=None, check=True) -> int:
+    s = lib.qwt_asym_weight_terms(_ptr(W), _ptr(w_zero), N, K, _ptr(w_terms), _stream(stream))
+    if check:
+        _check(s, "qwt_asym_weight_terms")
+    return s
+
+
+def qwt_qlinear_cwac_forward_asym(X, x_scale, x_zero, x_rowsum, W, w_terms, fscale, fbias, M, N, K, out_mode, Y, y_scale,
+                                  workspace, workspace_bytes, stream=None, check=True) -> int:
+    s = lib.qwt_qlinear_cwac_forward_asym(_ptr(X), _ptr(x_scale), _ptr(x_zero), _ptr(x_rowsum), _ptr(W), _ptr(w_terms),
+                                          _ptr(fscale), _ptr(fbias), M, N, K, out_mode, _ptr(Y), _ptr(y_scale),
+                                          _ptr(workspace), workspace_bytes, _stream(stream))
+    if check:
+        _check(s, "qwt_qlinear_cwac_forward_asym")
     return s
 
 

@@ -309,6 +309,48 @@ qwt_status qwt_qlinear_cwac_forward(const int8_t* X, const float* x_scale, const
                         as_stream(stream));
 }
 
+qwt_status qwt_qlinear_cwac_forward_asym(const uint8_t* X, const float* x_scale, const int32_t* x_zero,
+                                         const int32_t* x_rowsum, const uint8_t* W, const int32_t* w_terms,
+                                         const float* fscale, const float* fbias, int32_t M, int32_t N, int32_t K,
+                                         int32_t out_mode, void* Y, float* y_scale, void* workspace,
+                                         size_t workspace_bytes, void* stream) {
+  if (out_mode == QWT_OUT_INT8_STATIC) return QWT_ERR_UNSUPPORTED;
+  qwt_status s = check_forward_args(X, x_scale, W, QWT_W_INT8, fscale, fbias, M, N, K, out_mode, Y, y_scale, false);
+  if (s != QWT_OK) return s;
+  if (x_zero == nullptr || x_rowsum == nullptr || w_terms == nullptr || workspace == nullptr) return QWT_ERR_NULL;
+  if (K > 33000) return QWT_ERR_SHAPE;   // 255^2 * K must stay below 2^31
+  DeviceInfo dev{};
+  dev.sm_count = 148;
+  QlinearPlan plan;
+  if ((s = qlinear_plan(M, N, K, QWT_W_INT8, out_mode, dev, &plan)) != QWT_OK) return s;
+  if (workspace_bytes < plan.ws_total || !aligned(workspace, 256)) return QWT_ERR_WORKSPACE;
+  DeviceInfo real;
+  if ((s = current_device(&real)) != QWT_OK) return s;
+  if (real.sm_count < plan.grid) return QWT_ERR_ARCH;
+  return launch_qlinear(reinterpret_cast<const int8_t*>(X), x_scale, W, QWT_W_INT8, fscale, fbias, M, N, K, out_mode,
+                        Y, y_scale, workspace, plan, as_stream(stream), x_zero, x_rowsum, w_terms);
+}
+
+qwt_status qwt_asym_weight_terms(const uint8_t* W, const int32_t* w_zero, int32_t N, int32_t K, int32_t* w_terms,
+                                 void* stream) {
+  if (W == nullptr || w_zero == nullptr || w_terms == nullptr) return QWT_ERR_NULL;
+  if (N < 1 || K < 1 || K > 33000) return QWT_ERR_SHAPE;
+  DeviceInfo dev;
+  qwt_status s = current_device(&dev);
+  if (s != QWT_OK) return s;
+  return launch_asym_weight_terms(W, w_zero, N, K, w_terms, as_stream(stream));
+}
+
+qwt_status qwt_quantize_rows_u8(const float* X, int64_t rows, int32_t cols, int64_t ld, uint8_t* Xq, float* scale,
+                                int32_t* zero, int32_t* rowsum, void* stream) {
+  if (X == nullptr || Xq == nullptr || scale == nullptr || zero == nullptr) return QWT_ERR_NULL;
+  if (rows < 1 || cols < 1 || ld < cols || rows > (int64_t)8 * 2147483647) return QWT_ERR_SHAPE;
+  DeviceInfo dev;
+  qwt_status s = current_device(&dev);
+  if (s != QWT_OK) return s;
+  return launch_quantize_rows_u8(X, rows, cols, ld, Xq, scale, zero, rowsum, as_stream(stream));
+}
+
 qwt_status qwt_qlinear_check_status(const void* workspace, void* stream, int32_t* device_status) {
   if (workspace == nullptr) return QWT_ERR_NULL;
   QWT_CUDA_TRY(cudaStreamSynchronize(as_stream(stream)));

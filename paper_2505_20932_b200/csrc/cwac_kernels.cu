@@ -269,6 +269,64 @@ quantize_rows_kernel(const float* __restrict__ X, int64_t rows, int cols, int64_
   }
 }
 
+// Eq. 1-2 as printed, one row at a time (one warp per row): s = (max - min) / 255, z = clip(rne(-min / s), 0, 255),
+// code = clip(rne(x / s) + z, 0, 255); a constant row gets s = 1.  Also leaves the row's code sum, one of the
+// terms of Eq. 7.
+__global__ void __launch_bounds__(256)
+quantize_rows_u8_kernel(const float* __restrict__ X, int64_t rows, int cols, int64_t ld, uint8_t* __restrict__ Xq,
+                        float* __restrict__ scale, int32_t* __restrict__ zero, int32_t* __restrict__ rowsum) {
+  const int lane = threadIdx.x & 31;
+  const int64_t r = (int64_t)blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (r >= rows) return;
+  const float* x = X + r * ld;
+  float lo = x[0], hi = x[0];
+  for (int c = lane; c < cols; c += 32) {
+    lo = fminf(lo, x[c]);
+    hi = fmaxf(hi, x[c]);
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    lo = fminf(lo, __shfl_xor_sync(0xffffffffu, lo, o));
+    hi = fmaxf(hi, __shfl_xor_sync(0xffffffffu, hi, o));
+  }
+  float s = __fdiv_rn(__fsub_rn(hi, lo), 255.f);
+  if (!(s > 0.f)) s = 1.f;
+  const float zf = fminf(fmaxf(rintf(__fdiv_rn(-lo, s)), 0.f), 255.f);
+  uint8_t* q = Xq + r * (int64_t)cols;
+  int sum = 0;
+  for (int c = lane; c < cols; c += 32) {
+    const float v = fminf(fmaxf(__fadd_rn(rintf(__fdiv_rn(x[c], s)), zf), 0.f), 255.f);
+    q[c] = (uint8_t)(int)v;
+    sum += (int)v;
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if (lane == 0) {
+    scale[r] = s;
+    zero[r] = (int)zf;
+    if (rowsum != nullptr) rowsum[r] = sum;
+  }
+}
+
+// Weight-side terms of Eq. 7, one warp per output channel: terms[n] = -Z_W[n], terms[N + n] = K Z_W[n] - sum_k W_q[n, k].
+__global__ void __launch_bounds__(256)
+asym_weight_terms_kernel(const uint8_t* __restrict__ W, const int32_t* __restrict__ w_zero, int N, int K,
+                         int32_t* __restrict__ terms) {
+  const int lane = threadIdx.x & 31;
+  const int n = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+  if (n >= N) return;
+  const uint8_t* w = W + (size_t)n * K;
+  int sum = 0;
+  for (int k = lane; k < K; k += 32) sum += w[k];
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) sum += __shfl_xor_sync(0xffffffffu, sum, o);
+  if (lane == 0) {
+    const int z = w_zero[n];
+    terms[n] = -z;
+    terms[N + n] = K * z - sum;
+  }
+}
+
 __global__ void __launch_bounds__(256)
 pack_int4_kernel(const int8_t* __restrict__ codes, int64_t n_bytes, uint8_t* __restrict__ packed) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -358,6 +416,22 @@ qwt_status launch_quantize_rows(const float* X, int64_t rows, int32_t cols, int6
   const int rows_per_block = 8;
   const int64_t blocks = (rows + rows_per_block - 1) / rows_per_block;
   quantize_rows_kernel<<<(unsigned)blocks, rows_per_block * 32, 0, st>>>(X, rows, cols, ld, (float)qmax, Xq, scale);
+  QWT_LAUNCH_CHECK();
+  return QWT_OK;
+}
+
+qwt_status launch_quantize_rows_u8(const float* X, int64_t rows, int32_t cols, int64_t ld, uint8_t* Xq, float* scale,
+                                   int32_t* zero, int32_t* rowsum, cudaStream_t st) {
+  const int rows_per_block = 8;
+  const int64_t blocks = (rows + rows_per_block - 1) / rows_per_block;
+  quantize_rows_u8_kernel<<<(unsigned)blocks, rows_per_block * 32, 0, st>>>(X, rows, cols, ld, Xq, scale, zero, rowsum);
+  QWT_LAUNCH_CHECK();
+  return QWT_OK;
+}
+
+qwt_status launch_asym_weight_terms(const uint8_t* W, const int32_t* w_zero, int32_t N, int32_t K, int32_t* w_terms,
+                                    cudaStream_t st) {
+  asym_weight_terms_kernel<<<(N + 7) / 8, 256, 0, st>>>(W, w_zero, N, K, w_terms);
   QWT_LAUNCH_CHECK();
   return QWT_OK;
 }

@@ -217,6 +217,11 @@ __host__ __device__ constexpr uint32_t make_idesc_i8(int m, int n) {
   return (2u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
 }
 
+// Same with unsigned 8-bit A and B (format code 0 at bits 7 and 10).
+__host__ __device__ constexpr uint32_t make_idesc_u8(int m, int n) {
+  return (2u << 4) | ((uint32_t)(n >> 3) << 17) | ((uint32_t)(m >> 4) << 24);
+}
+
 // ---------------------------------------------------------------- global memory helpers
 __device__ __forceinline__ uint32_t ld_acquire_gpu(const uint32_t* p) {
   uint32_t v;

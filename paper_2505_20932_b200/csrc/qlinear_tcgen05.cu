@@ -88,15 +88,20 @@ struct QlParams {
   uint32_t* counters;            // [tiles_m] units of the strip that have published their row maxima
   uint32_t* flags;               // [tiles_m] raised by the unit that completes the strip
   unsigned long long timeout_ns;
+  // asymmetric (unsigned) codes, Eq. 7 in full: acc = sum W_q x_q - Z_W[n] rsx[m] + Z_x[m] (K Z_W[n] - csw[n])
+  const int* x_zero;             // [M] Z_x per token
+  const int* x_rowsum;           // [M] rsx[m] = sum_k x_q[m, k]
+  const int* w_terms;            // [2 N]: -Z_W[n], then K Z_W[n] - sum_k W_q[n, k]
 };
 
 // Compile-time geometry of one instantiation.
-template <int BN, int OUT, bool W4, bool WIDE>
+template <int BN, int OUT, bool W4, bool WIDE, bool ASYM = false>
 struct Cfg {
   static constexpr bool kInt8Out = OUT == QWT_OUT_INT8_PER_TOKEN;     // dynamic per-token scale: two-phase epilogue
   static constexpr bool kStatic8 = OUT == QWT_OUT_INT8_STATIC;       // Eq. 10 as printed: static multiplier + offset
   static constexpr bool kCodes = kInt8Out || kStatic8;               // one byte per output element
   static constexpr bool kHasParams = OUT != QWT_OUT_INT32_ACC;       // x_scale / fscale / fbias are used
+  static constexpr bool kNeedSlice = kHasParams || ASYM;             // per-column values staged in shared memory
   static constexpr int kEsz = kCodes ? 1 : (OUT == QWT_OUT_BF16 ? 2 : 4);
   static constexpr int kAcc = kTmemCols / BN;                        // accumulator buffers (tiles) in TMEM
   static constexpr int kUPT = BN / kUnitN;                           // epilogue units per tile
@@ -112,7 +117,9 @@ struct Cfg {
   static constexpr int kBBytes = BN * kBK;                           // expanded (int8) W tile of one stage
   static constexpr int kPBytes = W4 ? BN * (kBK / 2) : 0;            // packed (int4) W tile of one stage
   static constexpr int kStageBytes = kABytes + kBBytes + kPBytes;
-  static constexpr int kParamBytes = kGroups * 2 * kUnitN * 4;       // fscale | fbias slice of each group's unit
+  // per group and unit: fscale | fbias, and with asymmetric codes also the two integer column terms of Eq. 7
+  static constexpr int kParamArrays = ASYM ? 4 : 2;
+  static constexpr int kParamBytes = kGroups * kParamArrays * kUnitN * 4;
   static constexpr int kBarBytes = 512;
   static constexpr int kFixedBytes = kStagingBytes + kParamBytes + kBarBytes;
   static constexpr int kMaxStages = 12;
@@ -157,11 +164,11 @@ __device__ __forceinline__ float2 z_pair(uint32_t a0, uint32_t a1, float2 xs2, f
   return __ffma2_rn(__fmul2_rn(a, xs2), make_float2(f0, f1), make_float2(b0, b1));
 }
 
-template <int BN, int OUT, bool W4, bool WIDE>
-__global__ void __launch_bounds__((Cfg<BN, OUT, W4, WIDE>::kThreads), 1)
+template <int BN, int OUT, bool W4, bool WIDE, bool ASYM>
+__global__ void __launch_bounds__((Cfg<BN, OUT, W4, WIDE, ASYM>::kThreads), 1)
 qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const QlParams p) {
-  using C = Cfg<BN, OUT, W4, WIDE>;
+  using C = Cfg<BN, OUT, W4, WIDE, ASYM>;
   constexpr int kAcc = C::kAcc;
   constexpr int kMaxStages = C::kMaxStages;
   const int stages = p.stages;
@@ -293,7 +300,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
     if (lane == 0) {
-      constexpr uint32_t idesc = ptx::make_idesc_i8(kBM, BN);
+      constexpr uint32_t idesc = ASYM ? ptx::make_idesc_u8(kBM, BN) : ptx::make_idesc_i8(kBM, BN);
       const uint32_t a_base = ptx::smem_u32(sA), b_base = ptx::smem_u32(sB), w_base = ptx::smem_u32(sWres);
       uint32_t s = 0, ph = 0, it = 0;
       bool ok = true;
@@ -398,8 +405,11 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const bool lead = qd == 0;              // stages fscale / fbias and speaks for the group to the other CTAs
     uint8_t* stg = sStage + ew * C::kSlotBytes;
     const uint32_t swz = swizzle_xor<BOXB>(lane);
-    float* const ps_fs = sParam + g * 2 * kUnitN;   // this group's fscale slice, then its fbias slice
+    float* const ps_fs = sParam + g * C::kParamArrays * kUnitN;   // this group's fscale slice, then its fbias slice
     float* const ps_fb = ps_fs + kUnitN;
+    int* const ps_c1 = reinterpret_cast<int*>(ps_fs + 2 * kUnitN);   // ASYM: -Z_W, then K Z_W - column sum of W_q
+    int* const ps_cd = ps_c1 + kUnitN;
+    int pre_c1[kUnitN / 32], pre_cd[kUnitN / 32];
     const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + g * kUnitN;
     const int n_units = n_local * UPT;
     float pre_fs[kUnitN / 32], pre_fb[kUnitN / 32];
@@ -413,6 +423,11 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
       for (int i = 0; i < kUnitN / 32; ++i) {
         const int c = n0 + i * 32 + lane;
+        if (ASYM) {
+          pre_c1[i] = c < p.N ? __ldg(p.w_terms + c) : 0;
+          pre_cd[i] = c < p.N ? __ldg(p.w_terms + p.N + c) : 0;
+        }
+        if (!C::kHasParams) continue;
         pre_fs[i] = c < p.N ? __ldg(p.fscale + c) * (W4 ? 0.0625f : 1.0f) : 0.f;   // W4 operands hold 16 x code
         if (C::kStatic8) {   // integer accumulator offsets travel as bit patterns (x16 with the x16 W4 operands)
           const int o = c < p.N ? __ldg(reinterpret_cast<const int*>(p.fbias) + c) : 0;
@@ -422,7 +437,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       }
     };
-    if (C::kHasParams && lead && g < n_units) prefetch_params(g);
+    if (C::kNeedSlice && lead && g < n_units) prefetch_params(g);
 
     // Writes the warp's box (32 rows x BOXB bytes, swizzled in its staging slot) to global memory: lanes are
     // re-dealt so that one store instruction covers whole box rows (BOXB contiguous bytes each).
@@ -462,8 +477,19 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (r < p.M) xs4[k] = __ldg(p.x_scale + r);
         }
       }
+      int zx4[4] = {0, 0, 0, 0}, rs4[4] = {0, 0, 0, 0};   // ASYM: zero-point and code sum of the four rows
+      if (ASYM) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {
+          const int r = y0 + (lane >> 2) + 8 * k;
+          if (r < p.M) {
+            zx4[k] = __ldg(p.x_zero + r);
+            rs4[k] = __ldg(p.x_rowsum + r);
+          }
+        }
+      }
       bool ok = true;
-      if (C::kHasParams) {
+      if (C::kNeedSlice) {
         if (lead) {
           // the slice is free once the group's 4 warps have finished the unit that used it before
           if (!ptx::mbar_wait_bounded(&gdone[g], upar ^ 1u, cta_abort, tmo)) {
@@ -472,8 +498,14 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
 #pragma unroll
           for (int i = 0; i < kUnitN / 32; ++i) {
-            ps_fs[i * 32 + lane] = pre_fs[i];
-            ps_fb[i * 32 + lane] = pre_fb[i];
+            if (C::kHasParams) {
+              ps_fs[i * 32 + lane] = pre_fs[i];
+              ps_fb[i * 32 + lane] = pre_fb[i];
+            }
+            if (ASYM) {
+              ps_c1[i * 32 + lane] = pre_c1[i];
+              ps_cd[i * 32 + lane] = pre_cd[i];
+            }
           }
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&pfull[g]);
@@ -498,6 +530,20 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const bool in_range = n0 < p.N;        // a unit entirely right of the matrix has nothing to compute or store
       // z of one 8-column block for the thread's four rows; a = registers of lanes q, q + 8 (half 0) and of
       // lanes q + 16, q + 24 (half 1); col = first column of the block inside the unit
+      // Eq. 7: the unsigned product plus the three zero-point terms, for the block's two columns and four rows
+      // (in place, exact integer arithmetic): acc += -Z_W[n] rsx[m] + Z_x[m] (K Z_W[n] - csw[n])
+      auto asym_fix = [&](uint32_t* a0, uint32_t* a1, int col) {
+        const int2 c1 = *reinterpret_cast<const int2*>(ps_c1 + col + 2 * c);
+        const int2 cd = *reinterpret_cast<const int2*>(ps_cd + col + 2 * c);
+        auto fix = [&](uint32_t& v0, uint32_t& v1, int k) {
+          v0 = (uint32_t)((int)v0 + c1.x * rs4[k] + zx4[k] * cd.x);
+          v1 = (uint32_t)((int)v1 + c1.y * rs4[k] + zx4[k] * cd.y);
+        };
+        fix(a0[0], a0[1], 0);
+        fix(a0[2], a0[3], 1);
+        fix(a1[0], a1[1], 2);
+        fix(a1[2], a1[3], 3);
+      };
       auto z_block = [&](const uint32_t* a0, const uint32_t* a1, int col, float2 (&z)[4]) {
         const float2 f2 = *reinterpret_cast<const float2*>(ps_fs + col + 2 * c);
         const float2 b2 = *reinterpret_cast<const float2*>(ps_fb + col + 2 * c);
@@ -533,6 +579,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
           for (int i = 0; i < 4; ++i) {
             float2 z[4];
+            if (ASYM) asym_fix(a0 + 4 * i, a1 + 4 * i, h * 32 + 8 * i);
             z_block(a0 + 4 * i, a1 + 4 * i, h * 32 + 8 * i, z);
 #pragma unroll
             for (int k = 0; k < 4; ++k) amax[k] = fmaxf(amax[k], fmaxf(fabsf(z[k].x), fabsf(z[k].y)));
@@ -705,6 +752,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
               for (int i = 0; i < NB; ++i) {
                 const int colb = h * LDC + 8 * i;      // first column of the block inside the box
+                if (ASYM && !C::kInt8Out) asym_fix(a0 + 4 * i, a1 + 4 * i, c0 + 8 * i);
                 if (OUT == QWT_OUT_INT32_ACC) {
                   // W4: every term is a multiple of 16, the shift is exact
                   auto fix = [](uint32_t v) { return W4 ? (uint32_t)((int)v >> 4) : v; };
@@ -825,12 +873,12 @@ unsigned long long timeout_ns_from_env() {
   return v;
 }
 
-template <int BN, int OUT, bool W4, bool WIDE>
+template <int BN, int OUT, bool W4, bool WIDE, bool ASYM = false>
 qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams prm, int grid, int res_kb,
                       cudaStream_t st) {
-  using C = Cfg<BN, OUT, W4, WIDE>;
+  using C = Cfg<BN, OUT, W4, WIDE, ASYM>;
   constexpr int kThreads = C::kThreads;
-  auto kern = qlinear_cwac_kernel<BN, OUT, W4, WIDE>;
+  auto kern = qlinear_cwac_kernel<BN, OUT, W4, WIDE, ASYM>;
   prm.res_kb = res_kb;
   prm.stages = C::stages_for(res_kb);
   const int smem_bytes = C::dynamic_bytes(prm.stages, res_kb);
@@ -868,9 +916,30 @@ qwt_status launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const QlP
   return launch_cfg<BN, OUT, W4, false>(tmA, tmB, prm, grid, 0, st);
 }
 
+// Asymmetric (unsigned) codes: int8 weights only, streaming operand ring.
+template <int BN>
+qwt_status launch_asym(int out_mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
+                       cudaStream_t st) {
+  switch (out_mode) {
+    case QWT_OUT_INT8_PER_TOKEN:
+      return launch_cfg<BN, QWT_OUT_INT8_PER_TOKEN, false, false, true>(tmA, tmB, prm, grid, 0, st);
+    case QWT_OUT_BF16:
+      return launch_cfg<BN, QWT_OUT_BF16, false, false, true>(tmA, tmB, prm, grid, 0, st);
+    case QWT_OUT_FP32:
+      return launch_cfg<BN, QWT_OUT_FP32, false, false, true>(tmA, tmB, prm, grid, 0, st);
+    case QWT_OUT_INT32_ACC:
+      return launch_cfg<BN, QWT_OUT_INT32_ACC, false, false, true>(tmA, tmB, prm, grid, 0, st);
+  }
+  return QWT_ERR_UNSUPPORTED;
+}
+
 template <int BN, bool W4>
 qwt_status launch_bn(int out_mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
                      bool want_resident, cudaStream_t st) {
+  if (prm.w_terms != nullptr) {
+    if (W4) return QWT_ERR_UNSUPPORTED;
+    return launch_asym<BN>(out_mode, tmA, tmB, prm, grid, st);
+  }
   switch (out_mode) {
     case QWT_OUT_INT8_PER_TOKEN:
       return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN, W4>(tmA, tmB, prm, grid, want_resident, st);
@@ -944,7 +1013,8 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
 
 qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, int32_t wfmt, const float* fscale,
                           const float* fbias, int32_t M, int32_t N, int32_t K, int32_t out_mode, void* Y,
-                          float* y_scale, void* workspace, const QlinearPlan& plan, cudaStream_t st) {
+                          float* y_scale, void* workspace, const QlinearPlan& plan, cudaStream_t st,
+                          const int32_t* x_zero, const int32_t* x_rowsum, const int32_t* w_terms) {
   const bool w4 = wfmt == QWT_W_INT4_PACKED;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   CUtensorMap tmA, tmB;
@@ -976,6 +1046,9 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   prm.partial = reinterpret_cast<unsigned long long*>(ws + plan.ws_partial_off);
   prm.counter_target = (uint32_t)((N + kUnitN - 1) / kUnitN);   // units of a row strip that lie inside the matrix
   prm.gather_words = plan.gather_words;
+  prm.x_zero = x_zero;
+  prm.x_rowsum = x_rowsum;
+  prm.w_terms = w_terms;
   prm.rowmax = reinterpret_cast<uint32_t*>(ws + plan.ws_partial_off);
   prm.counters = prm.rowmax + (size_t)plan.tiles_m * kBM;
   prm.flags = prm.counters + plan.tiles_m;
