@@ -364,7 +364,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         const uint8_t* src = sP + s * C::kPBytes;
         uint8_t* dst = sB + s * C::kBBytes;
-#pragma unroll 2
+#pragma unroll
         for (int q = ct; q < BN * 4; q += 32 * kNumConvWarps) {
           const int n = q >> 2, c = q & 3;                 // row of the tile, 16-byte chunk of the packed row
           const uint4 w = *reinterpret_cast<const uint4*>(src + n * 64 + c * 16);
