@@ -40,8 +40,8 @@ INT8_OVER_BF16 = 2.0      # nominal dense ratio (4.5 POPS int8 : 2.25 PFLOPS bf1
 # DRAM bytes per algorithmic byte of cwac_stats_kernel, from the ncu capture summarised in
 # profiles/cwac_stats_kernel_cfg5_small.md (None until a capture exists).
 STATS_TRAFFIC_RATIO = 1.01
-# same for the forward kernel on a LLaMA-shaped layer, profiles/qlinear_cwac_kernel_*.md
-QLINEAR_TRAFFIC_RATIO = None
+# same for the forward kernel on the config-2 layers, profiles/qlinear_cwac_kernel_cfg2_int8.md
+QLINEAR_TRAFFIC_RATIO = 0.48    # the outputs stay in L2 for the length of the kernel (config-2 capture)
 
 
 def load_peaks():
