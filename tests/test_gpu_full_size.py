@@ -1,0 +1,108 @@
+"""GPU parity at the full sizes of the benchmark configurations, in the launch configuration bench.py times
+(device-resident inputs, the library's own plan for these shapes).  Where the oracle cannot evaluate a whole
+output in seconds it evaluates sampled rows (whole rows: the per-token scale depends on the complete row) or
+sampled channels (calibration is independent per channel)."""
+import numpy as np
+import pytest
+import torch
+
+from oracle import qwt_oracle as O
+from paper_2505_20932_b200 import workload as WL
+from tolerances import assert_ab_close, assert_codes_close
+
+pytestmark = pytest.mark.gpu
+DEV = "cuda"
+
+
+@pytest.fixture(scope="module")
+def B():
+    from paper_2505_20932_b200 import binding
+    return binding
+
+
+def device_layer(B, M, N, K, seed, w_bits=8):
+    g = torch.Generator(device=DEV)
+    g.manual_seed(seed)
+    qmax = 127 if w_bits == 8 else 7
+    Xq = torch.randint(-127, 128, (M, K), generator=g, device=DEV, dtype=torch.int8)
+    Wq = torch.randint(-qmax, qmax + 1, (N, K), generator=g, device=DEV, dtype=torch.int8)
+    xs = torch.rand(M, generator=g, device=DEV) * 0.04 + 0.01
+    fs = (torch.rand(N, generator=g, device=DEV) * 2e-4 + 1e-4) * (127 // qmax)
+    fb = torch.randn(N, generator=g, device=DEV) * 0.01
+    return Xq, Wq, xs, fs, fb
+
+
+def run_forward(B, Xq, xs, W, fs, fb, mode, wfmt, K):
+    M, N = Xq.shape[0], W.shape[0]
+    dt = {B.QWT_OUT_INT8_PER_TOKEN: torch.int8, B.QWT_OUT_BF16: torch.bfloat16}[mode]
+    Y = torch.empty((M, N), dtype=dt, device=DEV)
+    ys = torch.empty(M, dtype=torch.float32, device=DEV)
+    wsb = B.qwt_qlinear_workspace_bytes(M, N, K, wfmt, mode)
+    ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device=DEV)
+    for _ in range(2):      # twice on the same workspace, as the benchmark does
+        B.qwt_qlinear_cwac_forward(Xq, xs, W, wfmt, fs, fb, M, N, K, mode, Y, ys if mode == B.QWT_OUT_INT8_PER_TOKEN else None,
+                                   ws, wsb)
+    B.qwt_qlinear_check_status(ws)
+    return Y, ys
+
+
+@pytest.mark.parametrize("M,N,K", [(12608, 1152, 384), (12608, 384, 1536)])
+def test_config2_layers_whole_output(B, M, N, K):
+    Xq, Wq, xs, fs, fb = device_layer(B, M, N, K, seed=N + K)
+    Y, ys = run_forward(B, Xq, xs, Wq, fs, fb, B.QWT_OUT_INT8_PER_TOKEN, B.QWT_W_INT8, K)
+    z = O.forward_folded(O.int_matmul(Xq.cpu().numpy(), Wq.cpu().numpy()), xs.cpu().numpy(), fs.cpu().numpy(), fb.cpu().numpy())
+    c_ref, ys_ref = O.requant_per_token(z)
+    assert np.allclose(ys.cpu().numpy(), ys_ref, rtol=1e-5)
+    assert_codes_close(Y.cpu().numpy(), c_ref)
+
+
+@pytest.mark.parametrize("M,N,K", [(8192, 4096, 4096), (2048, 11008, 4096), (8192, 4096, 11008)])
+def test_config4_layers_sampled_rows(B, M, N, K):
+    Xq, Wq, xs, fs, fb = device_layer(B, M, N, K, seed=M + N)
+    Y, ys = run_forward(B, Xq, xs, Wq, fs, fb, B.QWT_OUT_INT8_PER_TOKEN, B.QWT_W_INT8, K)
+    rows = np.unique(np.concatenate([np.random.default_rng(5).integers(0, M, 60), [0, 127, 128, M - 1]]))
+    rt = torch.from_numpy(rows).to(DEV)
+    z = O.forward_folded(O.int_matmul(Xq[rt].cpu().numpy(), Wq.cpu().numpy()), xs[rt].cpu().numpy(), fs.cpu().numpy(),
+                         fb.cpu().numpy())
+    c_ref, ys_ref = O.requant_per_token(z)
+    assert np.allclose(ys[rt].cpu().numpy(), ys_ref, rtol=1e-5)
+    assert_codes_close(Y[rt].cpu().numpy(), c_ref)
+    # properties that hold for every row: the scale is positive and every row reaches an end code
+    assert bool((ys > 0).all()) and bool((Y.abs().amax(dim=1) == 127).all())
+
+
+def test_config3_layer_sampled_rows_w4_bf16(B):
+    M, N, K = 25216, 2304, 768
+    Xq, Wq, xs, fs, fb = device_layer(B, M, N, K, seed=3, w_bits=4)
+    Wp = torch.empty((N, K // 2), dtype=torch.uint8, device=DEV)
+    B.qwt_pack_int4(Wq, N, K, Wp)
+    Y, _ = run_forward(B, Xq, xs, Wp, fs, fb, B.QWT_OUT_BF16, B.QWT_W_INT4_PACKED, K)
+    rows = np.unique(np.concatenate([np.random.default_rng(6).integers(0, M, 60), [0, M - 1]]))
+    rt = torch.from_numpy(rows).to(DEV)
+    z = O.forward_folded(O.int_matmul(Xq[rt].cpu().numpy(), Wq.cpu().numpy()), xs[rt].cpu().numpy(), fs.cpu().numpy(),
+                         fb.cpu().numpy())
+    bits = Y[rt].view(torch.int16).cpu().numpy().view(np.uint16)
+    d = np.abs(bits.astype(np.int32) - O.to_bf16_bits(z).astype(np.int32))
+    assert d.max() <= 1 and np.count_nonzero(d) <= max(1, int(1e-4 * d.size))
+
+
+@pytest.mark.parametrize("C,bits", [(768, 4), (3072, 8)])
+def test_config5_calibration_sampled_channels(B, C, bits):
+    R = WL.CALIB_SWEEP_ROWS                       # 403,456 rows
+    fp, q, sig = WL.device_calib_pair(R, C, bits, seed=0, device=DEV)
+    a = torch.empty(C, dtype=torch.float32, device=DEV)
+    b = torch.empty(C, dtype=torch.float32, device=DEV)
+    wsb = B.qwt_cwac_workspace_bytes(R, C)
+    ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device=DEV)
+    B.qwt_cwac_calibrate(fp, q, R, C, C, a, b, None, ws, wsb)
+    torch.cuda.synchronize()
+    ch = np.unique(np.concatenate([np.random.default_rng(7).integers(0, C, 40), [0, 127, 128, C - 1]]))
+    ct = torch.from_numpy(ch).to(DEV)
+    fph, qh = fp[:, ct].cpu().numpy(), q[:, ct].cpu().numpy()
+    a_ref, b_ref, nd = O.cwac_fit(fph, qh)
+    assert nd == 0
+    assert_ab_close(a[ct].cpu().numpy(), b[ct].cpu().numpy(), a_ref, b_ref, np.maximum(np.abs(fph.mean(0)), fph.std(0)))
+    # every channel: the closed form for independent uniform noise, a = s^2 / (s^2 + D^2 / 12) with D = 8 s / (2^b - 1)
+    expect = 1.0 / (1.0 + (8.0 / (2 ** bits - 1)) ** 2 / 12.0)
+    assert np.abs(a.cpu().numpy() - expect).max() < 6.0 / np.sqrt(R) * (1.2 if bits == 4 else 0.1) + 1e-4
+    assert np.abs(b.cpu().numpy() / sig).max() < 6.0 / np.sqrt(R)
