@@ -973,7 +973,9 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
     const double pad_eff = (double)N / (double)(tn * bn);            // useful columns of the tiles
     return wave_eff * pad_eff;
   };
-  pl.bn = (N > 128 && score(256) + 0.15 >= score(128)) ? 256 : 128;
+  // 256-wide whenever the grid can still be filled; for small problems the narrower tile spreads over more SMs
+  const long tiles256 = (long)pl.tiles_m * ((N + 255) / 256);
+  pl.bn = (N > 128 && (tiles256 >= sms || score(256) + 0.15 >= score(128))) ? 256 : 128;
   const char* force = getenv("QWT_FORCE_BN");
   if (force != nullptr) {
     const int f = atoi(force);
