@@ -488,7 +488,6 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
       }
-      bool ok = true;
       if (C::kNeedSlice) {
         if (lead) {
           // the slice is free once the group's 4 warps have finished the unit that used it before
@@ -812,7 +811,6 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         ptx::mbar_arrive(&tempty[buf]);
         ptx::mbar_arrive(&gdone[g]);
       }
-      (void)ok;
     }
   }
 
