@@ -195,11 +195,18 @@ def phase_a(B, layers, stream, side=None):
         stream.wait_stream(side)
 
 
-def phase_b(B, layers, stream):
-    for L in layers:
+def phase_b(B, layers, stream, sides=()):
+    """Fused forward of every layer; like phase A the independent layers may be dealt over several streams, so
+    that one call's launch latency and tail run under its neighbours."""
+    lanes = [stream] + list(sides)
+    for sd in sides:
+        sd.wait_stream(stream)
+    for i, L in enumerate(layers):
         s = L.spec
         B.qwt_qlinear_cwac_forward(L.Xq, L.xs, L.W, L.wfmt, L.fs, L.fb, s.M, s.N, s.K, L.out_mode, L.Y, L.ys,
-                                   L.fws, L.fws_bytes, stream)
+                                   L.fws, L.fws_bytes, lanes[i % len(lanes)])
+    for sd in sides:
+        stream.wait_stream(sd)
 
 
 def workload_layers(WL, name):
@@ -372,6 +379,7 @@ def run_ours(args):
         graphs = []
         B.qwt_launch_count_reset()
         side = torch.cuda.Stream()
+        more_sides = [torch.cuda.Stream() for _ in range(2)]
         with torch.cuda.stream(cap):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=cap):
@@ -379,7 +387,7 @@ def run_ours(args):
             graphs.append(g)
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=cap):
-                phase_b(B, layers, cap)
+                phase_b(B, layers, cap, [side] + more_sides[: args.forward_streams - 2] if args.forward_streams > 1 else ())
             graphs.append(g)
         launches_per_step = B.qwt_launch_count()      # launches recorded = launches per replayed step
         stream.wait_stream(cap)
@@ -568,6 +576,8 @@ def main():
     ap.add_argument("--out", default="", choices=["", "int8", "bf16"], help="override the output stage")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--forward-streams", type=int, default=2, choices=[1, 2, 3, 4],
+                    help="streams the forward calls of phase B alternate over inside the graph")
     ap.add_argument("--no-library-int8", action="store_true", help="skip timing the library int8 matmul reference point")
     ap.add_argument("--no-graph", action="store_true", help="issue every library call from the host in the timed region")
     ap.add_argument("--no-cpu", action="store_true")
