@@ -563,13 +563,68 @@ def run_ours(args):
     return 0
 
 
+def run_calibration_sweep(args):
+    """Config 5: the calibration sweep (2048 images x 197 tokens, widths 768 / 2304 / 3072, quantization noise at 8
+    and 4 bits).  A step = qwt_cwac_calibrate on each of the six pairs; the value is GB/s (8 bytes per row and
+    channel), single GPU.  The pairs are drawn on the device one at a time (they are 2.5-9.9 GB each)."""
+    import torch
+    from paper_2505_20932_b200 import binding as B
+    from paper_2505_20932_b200 import workload as WL
+    torch.cuda.set_device(0)
+    device = "cuda:0"
+    peaks = load_peaks()
+    stream = torch.cuda.current_stream()
+    R = WL.CALIB_SWEEP_ROWS
+    rows, total_bytes, total_s = [], 0, 0.0
+    sampler = ClockSampler(0)
+    sampler.start()
+    B.qwt_launch_count_reset()
+    for C in WL.CALIB_SWEEP_WIDTHS:
+        for bits in WL.CALIB_SWEEP_BITS:
+            fp, q, _ = WL.device_calib_pair(R, C, bits, seed=args.seed, device=device)
+            a = torch.empty(C, dtype=torch.float32, device=device)
+            b = torch.empty(C, dtype=torch.float32, device=device)
+            wsb = B.qwt_cwac_workspace_bytes(R, C)
+            ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device=device)
+            for _ in range(args.warmup):
+                B.qwt_cwac_calibrate(fp, q, R, C, C, a, b, None, ws, wsb, stream)
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            for _ in range(args.steps):
+                B.qwt_cwac_calibrate(fp, q, R, C, C, a, b, None, ws, wsb, stream)
+            e1.record(stream)
+            torch.cuda.synchronize()
+            t = e0.elapsed_time(e1) * 1e-3 / args.steps
+            byt = 8 * R * C
+            rows.append({"channels": C, "bits": bits, "ms": t * 1e3, "gbs": byt / t / 1e9,
+                         "frac_hbm_peak": byt / t / 1e9 / peaks["hbm_gbs"], "a_mean": float(a.mean().item())})
+            total_bytes += byt
+            total_s += t
+            del fp, q, a, b, ws
+    launches = B.qwt_launch_count()
+    clocks = sampler.stop()
+    gbs = total_bytes / total_s / 1e9
+    line = {"metric": METRIC, "value": gbs, "unit": "GB/s", "n_gpus": 1, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": total_s * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f32",
+            "data": "synthetic",
+            "config": {"workload": "config 5: CWAC calibration sweep, 403456 rows x {768, 2304, 3072} channels, 8- and 4-bit noise",
+                       "l2": "inputs larger than L2 (2.5-9.9 GB per pair)"},
+            "roofline": {"kernel": "cwac_stats_kernel", "bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"],
+                         "unit": "GB/s", "frac": gbs / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
+                         "traffic": STATS_TRAFFIC_RATIO * total_bytes / len(rows)},
+            "pairs": rows, "cpu_baseline": None, "e2e": None, "gpu_launches": int(launches), "clocks": clocks}
+    print(json.dumps(line))
+    return 0
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=20)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
-    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4"])
+    ap.add_argument("--workload", default="cfg2", choices=["cfg1", "cfg2", "cfg3", "cfg4", "cfg5"])
     ap.add_argument("--layers", type=int, default=0, help="only the first L layers of the workload (0 = all)")
     ap.add_argument("--first-layer", type=int, default=0, help="skip this many layers of the workload")
     ap.add_argument("--calib-rows", type=int, default=0, help="cap the calibration rows per layer (0 = the config's)")
@@ -588,6 +643,8 @@ def main():
         args.warmup = 3
     if args.impl == "reference":
         return run_reference(args)
+    if args.workload == "cfg5":
+        return run_calibration_sweep(args)
     return run_ours(args)
 
 
