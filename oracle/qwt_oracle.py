@@ -112,6 +112,28 @@ def int_matmul(Xq: np.ndarray, Wq: np.ndarray) -> np.ndarray:
     return acc.astype(np.int64)
 
 
+def conv2d_int_nhwc(Xq: np.ndarray, Wq: np.ndarray, stride: int = 1, pad: int = 0) -> np.ndarray:
+    """Integer convolution by its definition (the paper places CWAC after every quantized convolution as well,
+    Section 3.3): acc[b, ho, wo, n] = sum_{i, j, c} Xq[b, ho*stride + i - pad, wo*stride + j - pad, c] * Wq[n, i, j, c],
+    positions outside the image contribute 0 (symmetric codes: zero-point 0).  Xq [B, H, W, C], Wq [N, kh, kw, C].
+    Returns int64 [B, Ho, Wo, N]."""
+    Xq = np.asarray(Xq, dtype=np.int64)
+    Wq = np.asarray(Wq, dtype=np.int64)
+    Bn, H, W, C = Xq.shape
+    N, kh, kw, C2 = Wq.shape
+    assert C == C2
+    Ho = (H + 2 * pad - kh) // stride + 1
+    Wo = (W + 2 * pad - kw) // stride + 1
+    Xp = np.zeros((Bn, H + 2 * pad, W + 2 * pad, C), dtype=np.int64)
+    Xp[:, pad:pad + H, pad:pad + W, :] = Xq
+    acc = np.zeros((Bn, Ho, Wo, N), dtype=np.int64)
+    for i in range(kh):
+        for j in range(kw):
+            patch = Xp[:, i:i + stride * (Ho - 1) + 1:stride, j:j + stride * (Wo - 1) + 1:stride, :]   # [B, Ho, Wo, C]
+            acc += patch @ Wq[:, i, j, :].T
+    return acc
+
+
 def qlinear_eq7(Wq: np.ndarray, xq: np.ndarray, Zw: np.ndarray, Zx: int) -> np.ndarray:
     """Bracket of Eq. 7 for one input vector, with the sums the paper's notation leaves
     implicit:  sum_k (Wq[n,k] - Zw[n]) (xq[k] - Zx)

@@ -484,3 +484,35 @@ def test_asymmetric_product_equals_eq7_expansion_and_brute_force():
     y = O.int_matmul_asym(xq, xz, wq, wz) * xs[:, None].astype(np.float64) * ws[None, :]
     ref = X.astype(np.float64) @ W.astype(np.float64).T
     assert np.abs(y - ref).max() < 0.02 * np.abs(ref).max() + 1e-3
+
+
+# ------------------------------------------------------------------ convolution (CWAC after quantized convolutions)
+
+def test_integer_convolution_definition():
+    rng = np.random.default_rng(51)
+    Bn, H, W, C, N = 2, 5, 6, 3, 4
+    X = rng.integers(-127, 128, (Bn, H, W, C))
+    # 1x1: the linear layer over B*H*W tokens
+    W1 = rng.integers(-127, 128, (N, 1, 1, C))
+    assert np.array_equal(O.conv2d_int_nhwc(X, W1).reshape(-1, N), O.int_matmul(X.reshape(-1, C), W1.reshape(N, C)))
+    # 3x3, stride 2, padding 1: brute force over every index
+    W3 = rng.integers(-127, 128, (N, 3, 3, C))
+    got = O.conv2d_int_nhwc(X, W3, stride=2, pad=1)
+    Ho, Wo = (H + 2 - 3) // 2 + 1, (W + 2 - 3) // 2 + 1
+    assert got.shape == (Bn, Ho, Wo, N)
+    for b in range(Bn):
+        for ho in range(Ho):
+            for wo in range(Wo):
+                for n in range(N):
+                    t = 0
+                    for i in range(3):
+                        for j in range(3):
+                            y, x = ho * 2 + i - 1, wo * 2 + j - 1
+                            if 0 <= y < H and 0 <= x < W:
+                                t += int(np.dot(X[b, y, x], W3[n, i, j]))
+                    assert got[b, ho, wo, n] == t
+    # a kernel that is 1 at its centre tap of channel c copies that channel (catches a flipped or shifted window)
+    Wd = np.zeros((C, 3, 3, C), dtype=np.int64)
+    for c in range(C):
+        Wd[c, 1, 1, c] = 1
+    assert np.array_equal(O.conv2d_int_nhwc(X, Wd, stride=1, pad=1), X)
