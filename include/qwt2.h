@@ -227,6 +227,20 @@ qwt_status qwt_qlinear_cwac_forward_asym(const uint8_t* X, const float* x_scale,
                                          int32_t out_mode, void* Y, float* y_scale, void* workspace,
                                          size_t workspace_bytes, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Convolutions (the paper places CWAC after every quantized convolution too, Section 3.3).  In NHWC layout a 1x1
+ * convolution is qwt_qlinear_cwac_forward itself with M = batch*H*W, K = C_in, N = C_out.  For a kh x kw
+ * convolution qwt_im2col_i8 writes the patch matrix
+ *     patches[(b, ho, wo), (i, j, c)] = X[b, ho*stride + i - pad, wo*stride + j - pad, c]   (0 outside the image)
+ * of shape [batch*Ho*Wo, kh*kw*C] (Ho = (H + 2 pad - kh) / stride + 1, likewise Wo), after which the convolution is
+ * the same forward call with K = kh*kw*C and the weights laid out [C_out, kh, kw, C_in].  The per-token scale of
+ * the layer's input belongs to the pixel the patch is centred on only if the scale is per tensor: use one
+ * x_scale value for all rows (the paper's per-tensor activation scale).  Symmetric codes (zero-point 0).
+ *   X int8 [batch, H, W, C], C % 16 == 0, 16-byte aligned; patches int8, 16-byte aligned.
+ * Errors: NULL, SHAPE, UNSUPPORTED (C % 16), ALIGN, ARCH, CUDA. */
+qwt_status qwt_im2col_i8(const int8_t* X, int32_t batch, int32_t H, int32_t W, int32_t C, int32_t kh, int32_t kw,
+                         int32_t stride, int32_t pad, int8_t* patches, void* stream);
+
 /* Kernels launched by this library on the calling thread since the last reset (for launch accounting). */
 int64_t qwt_launch_count(void);
 void qwt_launch_count_reset(void);

@@ -50,6 +50,7 @@ SIGNATURES = {
     "qwt_asym_weight_terms": (_i32, [_p, _p, _i32, _i32, _p, _p]),
     "qwt_qlinear_cwac_forward_asym": (_i32, [_p, _p, _p, _p, _p, _p, _p, _p, _i32, _i32, _i32, _i32, _p, _p, _p, _sz, _p]),
     "qwt_quantize_rows_i8": (_i32, [_p, _i64, _i32, _i64, _i32, _p, _p, _p]),
+    "qwt_im2col_i8": (_i32, [_p, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _p, _p]),
     "qwt_pack_int4": (_i32, [_p, _i64, _i32, _p, _p]),
     "qwt_launch_count": (_i64, []),
     "qwt_launch_count_reset": (None, []),
@@ -240,6 +241,13 @@ def qwt_quantize_rows_i8(X, rows, cols, ld, qmax, Xq, scale, stream=None, check=
     s = lib.qwt_quantize_rows_i8(_ptr(X), rows, cols, ld, qmax, _ptr(Xq), _ptr(scale), _stream(stream))
     if check:
         _check(s, "qwt_quantize_rows_i8")
+    return s
+
+
+def qwt_im2col_i8(X, batch, H, W, C, kh, kw, stride, pad, patches, stream=None, check=True) -> int:
+    s = lib.qwt_im2col_i8(_ptr(X), batch, H, W, C, kh, kw, stride, pad, _ptr(patches), _stream(stream))
+    if check:
+        _check(s, "qwt_im2col_i8")
     return s
 
 

@@ -429,6 +429,19 @@ qwt_status qwt_quantize_rows_i8(const float* X, int64_t rows, int32_t cols, int6
   return launch_quantize_rows(X, rows, cols, ld, qmax, Xq, scale, as_stream(stream));
 }
 
+qwt_status qwt_im2col_i8(const int8_t* X, int32_t batch, int32_t H, int32_t W, int32_t C, int32_t kh, int32_t kw,
+                         int32_t stride, int32_t pad, int8_t* patches, void* stream) {
+  if (X == nullptr || patches == nullptr) return QWT_ERR_NULL;
+  if (batch < 1 || H < 1 || W < 1 || C < 1 || kh < 1 || kw < 1 || stride < 1 || pad < 0) return QWT_ERR_SHAPE;
+  if (H + 2 * pad < kh || W + 2 * pad < kw) return QWT_ERR_SHAPE;
+  if ((C % 16) != 0) return QWT_ERR_UNSUPPORTED;
+  if (!aligned(X, 16) || !aligned(patches, 16)) return QWT_ERR_ALIGN;
+  DeviceInfo dev;
+  qwt_status s = current_device(&dev);
+  if (s != QWT_OK) return s;
+  return launch_im2col_i8(X, batch, H, W, C, kh, kw, stride, pad, patches, as_stream(stream));
+}
+
 qwt_status qwt_pack_int4(const int8_t* codes, int64_t rows, int32_t cols, uint8_t* packed, void* stream) {
   if (codes == nullptr || packed == nullptr) return QWT_ERR_NULL;
   if (rows < 1 || cols < 2) return QWT_ERR_SHAPE;

@@ -327,6 +327,30 @@ asym_weight_terms_kernel(const uint8_t* __restrict__ W, const int32_t* __restric
   }
 }
 
+// Patch matrix of a convolution (NHWC codes, zero-point 0): row (b, ho, wo), column (i, j, c) holds
+// X[b, ho*stride + i - pad, wo*stride + j - pad, c], 0 outside the image.  16 bytes per thread (C % 16 == 0).
+__global__ void __launch_bounds__(256)
+im2col_i8_kernel(const int8_t* __restrict__ X, int Bn, int H, int W, int C, int kh, int kw, int stride, int pad, int Ho,
+                 int Wo, int8_t* __restrict__ P) {
+  const int chunks = C >> 4;                                   // 16-byte chunks per pixel
+  const int64_t per_row = (int64_t)kh * kw * chunks;
+  const int64_t total = (int64_t)Bn * Ho * Wo * per_row;
+  const int64_t t = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (t >= total) return;
+  const int64_t rowi = t / per_row;
+  const int rem = (int)(t - rowi * per_row);
+  const int tap = rem / chunks, ch = rem - tap * chunks;
+  const int i = tap / kw, j = tap - i * kw;
+  const int wo = (int)(rowi % Wo);
+  const int64_t bh = rowi / Wo;
+  const int ho = (int)(bh % Ho), b = (int)(bh / Ho);
+  const int y = ho * stride + i - pad, x = wo * stride + j - pad;
+  uint4 v = make_uint4(0u, 0u, 0u, 0u);
+  if (y >= 0 && y < H && x >= 0 && x < W)
+    v = *reinterpret_cast<const uint4*>(X + (((int64_t)b * H + y) * W + x) * C + ch * 16);
+  *reinterpret_cast<uint4*>(P + rowi * ((int64_t)kh * kw * C) + (int64_t)tap * C + ch * 16) = v;
+}
+
 __global__ void __launch_bounds__(256)
 pack_int4_kernel(const int8_t* __restrict__ codes, int64_t n_bytes, uint8_t* __restrict__ packed) {
   const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -432,6 +456,15 @@ qwt_status launch_quantize_rows_u8(const float* X, int64_t rows, int32_t cols, i
 qwt_status launch_asym_weight_terms(const uint8_t* W, const int32_t* w_zero, int32_t N, int32_t K, int32_t* w_terms,
                                     cudaStream_t st) {
   asym_weight_terms_kernel<<<(N + 7) / 8, 256, 0, st>>>(W, w_zero, N, K, w_terms);
+  QWT_LAUNCH_CHECK();
+  return QWT_OK;
+}
+
+qwt_status launch_im2col_i8(const int8_t* X, int32_t Bn, int32_t H, int32_t W, int32_t C, int32_t kh, int32_t kw,
+                            int32_t stride, int32_t pad, int8_t* P, cudaStream_t st) {
+  const int Ho = (H + 2 * pad - kh) / stride + 1, Wo = (W + 2 * pad - kw) / stride + 1;
+  const int64_t total = (int64_t)Bn * Ho * Wo * kh * kw * (C / 16);
+  im2col_i8_kernel<<<(unsigned)((total + 255) / 256), 256, 0, st>>>(X, Bn, H, W, C, kh, kw, stride, pad, Ho, Wo, P);
   QWT_LAUNCH_CHECK();
   return QWT_OK;
 }

@@ -63,6 +63,8 @@ qwt_status launch_cwac_fold_static(const float* w_scale, const float* bias, cons
                                    float S_x, float S_r, float* mult, int32_t* offset, cudaStream_t st);
 qwt_status launch_quantize_rows(const float* X, int64_t rows, int32_t cols, int64_t ld, int32_t qmax, int8_t* Xq,
                                 float* scale, cudaStream_t st);
+qwt_status launch_im2col_i8(const int8_t* X, int32_t Bn, int32_t H, int32_t W, int32_t C, int32_t kh, int32_t kw,
+                            int32_t stride, int32_t pad, int8_t* P, cudaStream_t st);
 qwt_status launch_pack_int4(const int8_t* codes, int64_t rows, int32_t cols, uint8_t* packed, cudaStream_t st);
 
 // ---- forward (qlinear_tcgen05.cu)

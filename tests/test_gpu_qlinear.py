@@ -257,3 +257,29 @@ def test_resnet50_pointwise_convolutions(H, B):
         assert_codes_close(codes, c_ref, spec.name)
         raw, _ = H.gpu_forward(Xq, None, Wq, None, None, B.QWT_OUT_INT32_ACC)
         assert np.array_equal(raw.astype(np.int64), acc), spec.name
+
+
+@pytest.mark.parametrize("Bn,Hh,Ww,C,N,k,stride,pad", [(2, 14, 14, 64, 64, 3, 1, 1), (1, 15, 13, 32, 48, 3, 2, 1),
+                                                        (2, 8, 8, 16, 32, 5, 1, 2), (1, 7, 7, 128, 16, 7, 2, 3)])
+def test_convolution_through_the_patch_matrix(H, B, Bn, Hh, Ww, C, N, k, stride, pad):
+    """k x k convolution = qwt_im2col_i8 + the same forward call with K = k*k*C: raw accumulators against the
+    oracle's convolution by definition (bit-exact), then the folded FP32 output with a per-tensor input scale."""
+    import torch
+    rng = np.random.default_rng(Bn * 1000 + Hh * 10 + k)
+    X = rng.integers(-127, 128, (Bn, Hh, Ww, C)).astype(np.int8)
+    Wq = rng.integers(-127, 128, (N, k, k, C)).astype(np.int8)
+    Ho, Wo = (Hh + 2 * pad - k) // stride + 1, (Ww + 2 * pad - k) // stride + 1
+    M, K = Bn * Ho * Wo, k * k * C
+    P = torch.full((M, K), 0x5A, dtype=torch.int8, device=H.DEV)
+    B.qwt_im2col_i8(H.dev(X), Bn, Hh, Ww, C, k, k, stride, pad, P)
+    torch.cuda.synchronize()
+    Ph = P.cpu().numpy()
+    acc_ref = O.conv2d_int_nhwc(X, Wq, stride, pad).reshape(M, N)
+    assert np.array_equal(O.int_matmul(Ph, Wq.reshape(N, K)), acc_ref)          # the patch matrix itself
+    acc, _ = H.gpu_forward(Ph, None, Wq.reshape(N, K), None, None, B.QWT_OUT_INT32_ACC)
+    assert np.array_equal(acc.astype(np.int64), acc_ref)
+    xs = np.full(M, 0.02, np.float32)                                            # per-tensor activation scale
+    fs = rng.uniform(1e-4, 3e-4, N).astype(np.float32)
+    fb = (0.01 * rng.standard_normal(N)).astype(np.float32)
+    z, _ = H.gpu_forward(Ph, xs, Wq.reshape(N, K), fs, fb, B.QWT_OUT_FP32)
+    assert_fp32_close(z, O.forward_folded(acc_ref, xs, fs, fb))
