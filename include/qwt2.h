@@ -188,6 +188,31 @@ qwt_status qwt_qlinear_cwac_forward_host(const int8_t* X /*HOST*/, const float* 
                                          void* stream);
 
 /* ---------------------------------------------------------------------------------------------
+ * Calibration fused into the layer (Section 3.3 applied to the layer of Eq. 6-8, in one pass):
+ * the quantized layer runs on the calibration rows and, instead of writing its output
+ *     q[m, n] = S_x[m] S_W[n] acc[m, n] + bias[n]              (the layer before compensation, FP32)
+ * the kernel reads the stored full-precision output fp_out[m, n] of the same rows and accumulates the
+ * per-channel sums of Eq. 4-5 in its epilogue; q never exists in memory.  Results equal
+ * qwt_qlinear_cwac_forward(QWT_OUT_FP32, fscale = w_scale, fbias = bias) followed by qwt_cwac_calibrate
+ * within the calibration tolerance (same q values, different but fixed summation order: strips of 128 rows,
+ * then the strips in order; results are bitwise reproducible).
+ *   X, x_scale, W, w_format : as for qwt_qlinear_cwac_forward (x_scale required)
+ *   w_scale  float [N]      : S_W;   bias float [N] or NULL (= 0)
+ *   fp_out   float [M, ld]  : 16-byte aligned, ld >= N, ld % 4 == 0;   N % 4 == 0
+ *   stats    float64 [5 * N] or NULL: running statistics, updated in place (layout of qwt_cwac_stats_accumulate)
+ *   a, b     float [N] or both NULL : solved from (stats + this call) when given; one of stats / (a, b) is required
+ *   n_degenerate            : as for qwt_cwac_calibrate, may be NULL
+ *   workspace               : device, 256-byte aligned, >= qwt_qlinear_cwac_calibrate_workspace_bytes; its first
+ *                             word is the status word of qwt_qlinear_check_status
+ */
+size_t qwt_qlinear_cwac_calibrate_workspace_bytes(int32_t M, int32_t N, int32_t K, int32_t w_format);
+qwt_status qwt_qlinear_cwac_calibrate(const int8_t* X, const float* x_scale, const void* W, int32_t w_format,
+                                      const float* w_scale, const float* bias, const float* fp_out, int64_t ld,
+                                      int32_t M, int32_t N, int32_t K, double* stats, float* a, float* b,
+                                      int32_t* n_degenerate, void* workspace, size_t workspace_bytes,
+                                      void* stream);
+
+/* ---------------------------------------------------------------------------------------------
  * Support: symmetric row-wise quantizer -- Eq. 1-2 with zero-point 0 and signed codes.
  *     scale[r] = max_c |X[r, c]| / qmax;   Xq[r, c] = clip(rne(X[r, c] / scale[r]), -qmax, qmax)
  * Per-token activations: X = activations, qmax = 127.  Per-channel weights: X = W [N, K], qmax = 127 or 7.

@@ -43,6 +43,9 @@ SIGNATURES = {
     "qwt_cwac_fold_static": (_i32, [_p, _p, _p, _p, _i32, C.c_float, C.c_float, _p, _p, _p]),
     "qwt_qlinear_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32, _i32]),
     "qwt_qlinear_cwac_forward": (_i32, [_p, _p, _p, _i32, _p, _p, _i32, _i32, _i32, _i32, _p, _p, _p, _sz, _p]),
+    "qwt_qlinear_cwac_calibrate_workspace_bytes": (_sz, [_i32, _i32, _i32, _i32]),
+    "qwt_qlinear_cwac_calibrate": (_i32, [_p, _p, _p, _i32, _p, _p, _p, _i64, _i32, _i32, _i32, _p, _p, _p, _p, _p,
+                                          _sz, _p]),
     "qwt_qlinear_check_status": (_i32, [_p, _p, C.POINTER(_i32)]),
     "qwt_qlinear_host_staging_bytes": (_sz, [_i32, _i32, _i32, _i32, _i32]),
     "qwt_qlinear_cwac_forward_host": (_i32, [_p, _p, _p, _i32, _p, _p, _i32, _i32, _i32, _i32, _p, _p, _p, _sz, _p]),
@@ -129,6 +132,20 @@ def qwt_cwac_stats_accumulate(fp_out, q_out, rows, channels, ld, stats, workspac
                                       workspace_bytes, _stream(stream))
     if check:
         _check(s, "qwt_cwac_stats_accumulate")
+    return s
+
+
+def qwt_qlinear_cwac_calibrate_workspace_bytes(M, N, K, w_format) -> int:
+    return int(lib.qwt_qlinear_cwac_calibrate_workspace_bytes(M, N, K, w_format))
+
+
+def qwt_qlinear_cwac_calibrate(X, x_scale, W, w_format, w_scale, bias, fp_out, ld, M, N, K, stats, a, b, n_degenerate,
+                               workspace, workspace_bytes, stream=None, check=True) -> int:
+    s = lib.qwt_qlinear_cwac_calibrate(_ptr(X), _ptr(x_scale), _ptr(W), w_format, _ptr(w_scale), _ptr(bias),
+                                       _ptr(fp_out), ld, M, N, K, _ptr(stats), _ptr(a), _ptr(b), _ptr(n_degenerate),
+                                       _ptr(workspace), workspace_bytes, _stream(stream))
+    if check:
+        _check(s, "qwt_qlinear_cwac_calibrate")
     return s
 
 

@@ -331,6 +331,66 @@ qwt_status qwt_qlinear_cwac_forward_asym(const uint8_t* X, const float* x_scale,
                         Y, y_scale, workspace, plan, as_stream(stream), x_zero, x_rowsum, w_terms);
 }
 
+// Calibration fused into the layer (Section 3.3 on top of Eq. 6-8): workspace = [status 256 B][partials].
+namespace {
+struct FusedCalibLayout {
+  QlinearPlan plan;
+  CwacPlan red;          // the strips of 128 rows play the part of the row chunks
+  size_t off_partial, total;
+};
+qwt_status fused_calib_layout(int32_t M, int32_t N, int32_t K, int32_t wfmt, FusedCalibLayout* L) {
+  DeviceInfo dev{};
+  dev.sm_count = 148;
+  qwt_status s = qlinear_plan(M, N, K, wfmt, kOutCalibStats, dev, &L->plan);
+  if (s != QWT_OK) return s;
+  L->red = CwacPlan{};
+  L->red.slabs = (N + 127) / 128;
+  L->red.cpad = L->red.slabs * 128;
+  L->red.chunks = L->plan.tiles_m;
+  L->red.chunk_rows = 128;
+  L->red.partial_bytes = (size_t)L->red.chunks * 4 * L->red.cpad * sizeof(double);
+  L->off_partial = 256;
+  L->total = L->off_partial + L->red.partial_bytes;
+  return QWT_OK;
+}
+}  // namespace
+
+size_t qwt_qlinear_cwac_calibrate_workspace_bytes(int32_t M, int32_t N, int32_t K, int32_t wfmt) {
+  if (M < 1 || N < 1 || K < 1) return 0;
+  FusedCalibLayout L;
+  if (fused_calib_layout(M, N, K, wfmt, &L) != QWT_OK) return 0;
+  return L.total;
+}
+
+qwt_status qwt_qlinear_cwac_calibrate(const int8_t* X, const float* x_scale, const void* W, int32_t wfmt,
+                                      const float* w_scale, const float* bias, const float* fp_out, int64_t ld,
+                                      int32_t M, int32_t N, int32_t K, double* stats, float* a, float* b,
+                                      int32_t* n_degenerate, void* workspace, size_t workspace_bytes, void* stream) {
+  if (X == nullptr || x_scale == nullptr || W == nullptr || w_scale == nullptr || fp_out == nullptr ||
+      workspace == nullptr)
+    return QWT_ERR_NULL;
+  if (stats == nullptr && (a == nullptr || b == nullptr)) return QWT_ERR_NULL;
+  if ((a == nullptr) != (b == nullptr)) return QWT_ERR_NULL;
+  if (wfmt != QWT_W_INT8 && wfmt != QWT_W_INT4_PACKED) return QWT_ERR_UNSUPPORTED;
+  if (M < 1 || N < 1 || K < 1 || ld < N || K > 131072) return QWT_ERR_SHAPE;
+  if (K % (wfmt == QWT_W_INT8 ? 16 : 32) != 0 || N % 4 != 0 || ld % 4 != 0) return QWT_ERR_UNSUPPORTED;
+  if (!aligned(X, 16) || !aligned(W, 16) || !aligned(fp_out, 16)) return QWT_ERR_ALIGN;
+  FusedCalibLayout L;
+  qwt_status s = fused_calib_layout(M, N, K, wfmt, &L);
+  if (s != QWT_OK) return s;
+  if (workspace_bytes < L.total || !aligned(workspace, 256)) return QWT_ERR_WORKSPACE;
+  DeviceInfo real;
+  if ((s = current_device(&real)) != QWT_OK) return s;
+  if (real.sm_count < L.plan.grid) return QWT_ERR_ARCH;
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  QlinearStatsArgs sa{fp_out, ld, reinterpret_cast<double*>(ws + L.off_partial), L.red.cpad};
+  cudaStream_t st = as_stream(stream);
+  if ((s = launch_qlinear(X, x_scale, W, wfmt, w_scale, bias, M, N, K, kOutCalibStats, nullptr, nullptr, workspace,
+                          L.plan, st, nullptr, nullptr, nullptr, &sa)) != QWT_OK)
+    return s;
+  return launch_cwac_reduce(ws + L.off_partial, L.red, N, M, stats, a, b, n_degenerate, st);
+}
+
 qwt_status qwt_asym_weight_terms(const uint8_t* W, const int32_t* w_zero, int32_t N, int32_t K, int32_t* w_terms,
                                  void* stream) {
   if (W == nullptr || w_zero == nullptr || w_terms == nullptr) return QWT_ERR_NULL;

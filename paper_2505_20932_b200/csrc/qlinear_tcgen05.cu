@@ -92,6 +92,11 @@ struct QlParams {
   const int* x_zero;             // [M] Z_x per token
   const int* x_rowsum;           // [M] rsx[m] = sum_k x_q[m, k]
   const int* w_terms;            // [2 N]: -Z_W[n], then K Z_W[n] - sum_k W_q[n, k]
+  // calibration statistics instead of an output matrix (Section 3.3, Eq. 4-5)
+  const float* F;                // [M, ldf] full-precision output of the same layer on the same rows
+  long long ldf;
+  double* sums;                  // [tiles_m][4][cpad]: sum q, sum f, sum q f, sum q q over the rows of a strip
+  int cpad;
 };
 
 // Compile-time geometry of one instantiation.
@@ -100,6 +105,7 @@ struct Cfg {
   static constexpr bool kInt8Out = OUT == QWT_OUT_INT8_PER_TOKEN;     // dynamic per-token scale: two-phase epilogue
   static constexpr bool kStatic8 = OUT == QWT_OUT_INT8_STATIC;       // Eq. 10 as printed: static multiplier + offset
   static constexpr bool kCodes = kInt8Out || kStatic8;               // one byte per output element
+  static constexpr bool kStats = OUT == kOutCalibStats;              // no output matrix: per-channel sums of Eq. 4-5
   static constexpr bool kHasParams = OUT != QWT_OUT_INT32_ACC;       // x_scale / fscale / fbias are used
   static constexpr bool kNeedSlice = kHasParams || ASYM;             // per-column values staged in shared memory
   static constexpr int kEsz = kCodes ? 1 : (OUT == QWT_OUT_BF16 ? 2 : 4);
@@ -110,7 +116,8 @@ struct Cfg {
   // output staging: one box of 32 rows per epilogue warp, through which a warp turns "thread = row" into
   // row-contiguous global stores.  128-byte rows for 128-wide tiles; 256-wide tiles use 32-byte rows when the
   // operand ring needs the room (long K: the epilogue hides behind the mainloop) and 64-byte rows otherwise
-  static constexpr int kBoxBytes = BN == 128 ? 128 : (WIDE ? 64 : 32);
+  // (statistics: the slot holds the warp's four sums and two shifts of the unit's 128 columns, 3 KB)
+  static constexpr int kBoxBytes = kStats ? 96 : (BN == 128 ? 128 : (WIDE ? 64 : 32));
   static constexpr int kBC = kBoxBytes / kEsz;                       // columns per box
   static constexpr int kSlotBytes = 32 * kBoxBytes;
   static constexpr int kStagingBytes = kEpiWarps * kSlotBytes;
@@ -433,7 +440,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           const int o = c < p.N ? __ldg(reinterpret_cast<const int*>(p.fbias) + c) : 0;
           pre_fb[i] = __int_as_float(W4 ? o * 16 : o);
         } else {
-          pre_fb[i] = c < p.N ? __ldg(p.fbias + c) : 0.f;
+          pre_fb[i] = (c < p.N && p.fbias != nullptr) ? __ldg(p.fbias + c) : 0.f;   // statistics: no bias = 0
         }
       }
     };
@@ -709,8 +716,130 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       }
 
+      if constexpr (C::kStats) {
+        // -------------------------------------------------------------- calibration statistics of the unit
+        // q = the layer's quantized output before compensation (fscale = S_W, fbias = bias), f = the stored
+        // full-precision output of the same rows.  Eq. 4-5 need, per channel, the sums of q, f, q f and q q.
+        // A warp shifts q and f by their values in its own first row (a constant column then sums to exactly
+        // zero, as Eq. 4's degenerate case needs), adds the shifted terms in FP32 over its 32 rows (4 in the
+        // thread, then a halving butterfly over the 8 lanes that share a column pair: pairwise order, at most
+        // 5 roundings deep) and leaves sums and shifts in shared memory; the group's 128 threads then take one
+        // column each, undo the shifts in FP64, add the four warps in order and write the strip's partial.  A
+        // second kernel adds the strips in a fixed order.  Rows >= M and columns >= N contribute nothing.
+        constexpr int NB = 2;                                  // 8-column blocks per step
+        float* const wsum = reinterpret_cast<float*>(stg);      // [4 sums | shift of q | shift of f][128 columns]
+        bool rv[4];
+#pragma unroll
+        for (int k = 0; k < 4; ++k) rv[k] = y0 + q + 8 * k < p.M;
+        if (in_range) {
+#pragma unroll 1
+          for (int h = 0; h < kUnitN / (8 * NB); ++h) {
+            const int c0 = h * 8 * NB;                          // first column of the step inside the unit
+            float2 fv[NB][4];
+#pragma unroll
+            for (int i = 0; i < NB; ++i) {
+              const int col = n0 + c0 + 8 * i + 2 * c;          // N is even: a column pair is all in or all out
+#pragma unroll
+              for (int k = 0; k < 4; ++k)
+                fv[i][k] = (col < p.N && rv[k]) ? __ldcs(reinterpret_cast<const float2*>(
+                                                      p.F + (size_t)(y0 + q + 8 * k) * (size_t)p.ldf + col))
+                                                : make_float2(0.f, 0.f);
+            }
+            uint32_t a0[4 * NB], a1[4 * NB];
+            ptx::tmem_ld_frag<NB>(taddr + c0, a0);
+            ptx::tmem_ld_frag<NB>(taddr + (16u << 16) + c0, a1);
+            ptx::tmem_ld_wait();
+            float v[8 * NB];                                    // [(block, column of the pair)][sum]
+#pragma unroll
+            for (int i = 0; i < NB; ++i) {
+              float2 z[4];
+              z_block(a0 + 4 * i, a1 + 4 * i, c0 + 8 * i, z);
+              // the warp's first row sits in lanes 0-3 (q = 0), row slot k = 0
+              const float2 kq = make_float2(__shfl_sync(0xffffffffu, z[0].x, c), __shfl_sync(0xffffffffu, z[0].y, c));
+              const float2 kf = make_float2(__shfl_sync(0xffffffffu, fv[i][0].x, c),
+                                            __shfl_sync(0xffffffffu, fv[i][0].y, c));
+              if (q == 0) {
+                *reinterpret_cast<float2*>(wsum + 4 * kUnitN + c0 + 8 * i + 2 * c) = kq;
+                *reinterpret_cast<float2*>(wsum + 5 * kUnitN + c0 + 8 * i + 2 * c) = kf;
+              }
+              auto four_rows = [&](float z0, float z1, float z2, float z3, float f0, float f1, float f2, float f3,
+                                   float shq, float shf, float* out) {
+                const float zz[4] = {z0, z1, z2, z3}, ff[4] = {f0, f1, f2, f3};
+                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+#pragma unroll
+                for (int k = 0; k < 4; ++k) {
+                  const float dq = rv[k] ? zz[k] - shq : 0.f;
+                  const float df = rv[k] ? ff[k] - shf : 0.f;
+                  s0 += dq;
+                  s1 += df;
+                  s2 = fmaf(dq, df, s2);
+                  s3 = fmaf(dq, dq, s3);
+                }
+                out[0] = s0;
+                out[1] = s1;
+                out[2] = s2;
+                out[3] = s3;
+              };
+              four_rows(z[0].x, z[1].x, z[2].x, z[3].x, fv[i][0].x, fv[i][1].x, fv[i][2].x, fv[i][3].x, kq.x, kf.x,
+                        v + (2 * i) * 4);
+              four_rows(z[0].y, z[1].y, z[2].y, z[3].y, fv[i][0].y, fv[i][1].y, fv[i][2].y, fv[i][3].y, kq.y, kf.y,
+                        v + (2 * i + 1) * 4);
+            }
+            // halving butterfly over lane bits 4, 3, 2 (the row index q): at every level a lane hands one half
+            // of its values to its partner and adds the partner's other half to the half it keeps
+#pragma unroll
+            for (int lvl = 0; lvl < 3; ++lvl) {
+              const int mask = 16 >> lvl;
+              const int half = (8 * NB) >> (lvl + 1);
+              const bool up = (lane & mask) != 0;
+#pragma unroll
+              for (int j = 0; j < half; ++j) {
+                const float lo = v[j], hi = v[j + half];
+                const float got = __shfl_xor_sync(0xffffffffu, up ? lo : hi, mask);
+                v[j] = (up ? hi : lo) + got;
+              }
+            }
+            // the lane is left with values j + NB q of the original numbering
+#pragma unroll
+            for (int j = 0; j < NB; ++j) {
+              const int idx = j + NB * q;
+              const int ie = idx >> 2;
+              wsum[(idx & 3) * kUnitN + c0 + 8 * (ie >> 1) + 2 * c + (ie & 1)] = v[j];
+            }
+          }
+        }
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&pub[g]);
+        if (!ptx::mbar_wait_bounded(&pub[g], upar, cta_abort, tmo)) {
+          give_up(kStWaitStrip);
+          break;
+        }
+        const int t = qd * 32 + lane;                           // the group's 128 threads take one column each
+        if (in_range && n0 + t < p.N) {
+          double Sq = 0.0, Sf = 0.0, Sqf = 0.0, Sqq = 0.0;
+#pragma unroll
+          for (int w = 0; w < kGroupWarps; ++w) {
+            // the slot of epilogue warp g * 4 + w holds the rows of TMEM quadrant (g * 4 + w + 2) % 4
+            const int row0 = tm * kBM + ((g * kGroupWarps + w + 2) & 3) * 32;
+            const int left = p.M - row0;
+            if (left <= 0) continue;                            // nothing of this warp is inside the matrix
+            const double nw = (double)(left < 32 ? left : 32);
+            const float* ws4 = reinterpret_cast<const float*>(sStage + (g * kGroupWarps + w) * C::kSlotBytes) + t;
+            const double d0 = ws4[0], d1 = ws4[kUnitN], d2 = ws4[2 * kUnitN], d3 = ws4[3 * kUnitN];
+            const double Kq = ws4[4 * kUnitN], Kf = ws4[5 * kUnitN];
+            Sq += d0 + nw * Kq;
+            Sf += d1 + nw * Kf;
+            Sqf += d2 + Kf * d0 + Kq * d1 + nw * Kq * Kf;
+            Sqq += d3 + 2.0 * Kq * d0 + nw * Kq * Kq;
+          }
+          double* out = p.sums + (size_t)tm * 4 * (size_t)p.cpad + n0 + t;
+          out[0] = Sq;
+          out[(size_t)p.cpad] = Sf;
+          out[2 * (size_t)p.cpad] = Sqf;
+          out[3 * (size_t)p.cpad] = Sqq;
+        }
+      } else if (in_range) {
       // ------------------------------------------------------------------ conversion and store, box by box
-      if (in_range) {
         // z / den rounded to nearest: q0 = z * (1/den), then one residual correction with fused multiply-adds;
         // adding 1.5 * 2^23 leaves rne(q) in the low mantissa bits (|q| <= 127 by construction).
         // (the whole box loop is instantiated twice so that the common case carries no branch per element)
@@ -949,6 +1078,10 @@ qwt_status launch_bn(int out_mode, const CUtensorMap& tmA, const CUtensorMap& tm
       return launch_inst<BN, QWT_OUT_INT32_ACC, W4>(tmA, tmB, prm, grid, want_resident, st);
     case QWT_OUT_INT8_STATIC:
       return launch_inst<BN, QWT_OUT_INT8_STATIC, W4>(tmA, tmB, prm, grid, want_resident, st);
+    case kOutCalibStats:
+      // packed weights with 256-wide tiles leave no room for the per-warp sums: the plan picks 128 there
+      if constexpr (W4 && BN == 256) return QWT_ERR_UNSUPPORTED;
+      else return launch_inst<BN, kOutCalibStats, W4>(tmA, tmB, prm, grid, want_resident, st);
   }
   return QWT_ERR_UNSUPPORTED;
 }
@@ -974,10 +1107,11 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   // 256-wide whenever the grid can still be filled; for small problems the narrower tile spreads over more SMs
   const long tiles256 = (long)pl.tiles_m * ((N + 255) / 256);
   pl.bn = (N > 128 && (tiles256 >= sms || score(256) + 0.15 >= score(128))) ? 256 : 128;
+  if (out_mode == kOutCalibStats && wfmt == QWT_W_INT4_PACKED) pl.bn = 128;
   const char* force = getenv("QWT_FORCE_BN");
   if (force != nullptr) {
     const int f = atoi(force);
-    if (f == 128 || f == 256) pl.bn = f;
+    if ((f == 128 || f == 256) && !(out_mode == kOutCalibStats && wfmt == QWT_W_INT4_PACKED)) pl.bn = f;
   }
   pl.tiles_n = (N + pl.bn - 1) / pl.bn;
   const long tiles = (long)pl.tiles_m * pl.tiles_n;
@@ -1014,7 +1148,8 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
 qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, int32_t wfmt, const float* fscale,
                           const float* fbias, int32_t M, int32_t N, int32_t K, int32_t out_mode, void* Y,
                           float* y_scale, void* workspace, const QlinearPlan& plan, cudaStream_t st,
-                          const int32_t* x_zero, const int32_t* x_rowsum, const int32_t* w_terms) {
+                          const int32_t* x_zero, const int32_t* x_rowsum, const int32_t* w_terms,
+                          const QlinearStatsArgs* stats) {
   const bool w4 = wfmt == QWT_W_INT4_PACKED;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   CUtensorMap tmA, tmB;
@@ -1053,6 +1188,12 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   prm.counters = prm.rowmax + (size_t)plan.tiles_m * kBM;
   prm.flags = prm.counters + plan.tiles_m;
   prm.timeout_ns = timeout_ns_from_env();
+  if (stats != nullptr) {
+    prm.F = stats->F;
+    prm.ldf = stats->ldf;
+    prm.sums = stats->sums;
+    prm.cpad = stats->cpad;
+  }
 
   int mode = out_mode;
   prm.Y = Y;

@@ -79,11 +79,19 @@ struct QlinearPlan {
 };
 qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
                         QlinearPlan* plan);
+// Internal output mode of the forward kernel: no output matrix, the per-channel sums of Eq. 4-5 instead.
+constexpr int kOutCalibStats = 5;
+struct QlinearStatsArgs {
+  const float* F;      // [M, ldf] full-precision output
+  int64_t ldf;
+  double* sums;        // [tiles_m][4][cpad] partials, one per strip of 128 rows
+  int cpad;
+};
 qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, int32_t wfmt, const float* fscale,
                           const float* fbias, int32_t M, int32_t N, int32_t K, int32_t out_mode, void* Y,
                           float* y_scale, void* workspace, const QlinearPlan& plan, cudaStream_t st,
                           const int32_t* x_zero = nullptr, const int32_t* x_rowsum = nullptr,
-                          const int32_t* w_terms = nullptr);
+                          const int32_t* w_terms = nullptr, const QlinearStatsArgs* stats = nullptr);
 qwt_status launch_quantize_rows_u8(const float* X, int64_t rows, int32_t cols, int64_t ld, uint8_t* Xq, float* scale,
                                    int32_t* zero, int32_t* rowsum, cudaStream_t st);
 qwt_status launch_asym_weight_terms(const uint8_t* W, const int32_t* w_zero, int32_t N, int32_t K, int32_t* w_terms,

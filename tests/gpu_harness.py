@@ -129,3 +129,25 @@ def gpu_forward(Xq, xs, W, fs, fb, out_mode, wfmt=B.QWT_W_INT8, K=None, check_gu
     else:
         Yh = Y.cpu().numpy().reshape(M, N)
     return Yh, (None if ys is None else ys.cpu().numpy())
+
+
+def gpu_calibrate_fused(Xq, xs, W, w_scale, bias, fp, wfmt=B.QWT_W_INT8, K=None, stats=None, solve=True):
+    """Calibration inside the layer's epilogue: returns (a, b, n_degenerate, stats [5, N] or None).
+    fp: float32 [M, ld] with ld >= N.  stats: running statistics (numpy [5, N]) to continue from, or None."""
+    M = Xq.shape[0]
+    K = Xq.shape[1] if K is None else K
+    N = W.shape[0]
+    ld = fp.shape[1]
+    dX, dW, dxs, dws, dfp = dev(Xq), dev(W), dev(xs.astype(np.float32)), dev(w_scale.astype(np.float32)), dev(fp)
+    dbias = None if bias is None else dev(bias.astype(np.float32))
+    dstats = None if stats is None else dev(np.ascontiguousarray(stats, dtype=np.float64).reshape(-1))
+    a = torch.full((N,), 7.0, dtype=torch.float32, device=DEV) if solve else None
+    b = torch.full((N,), 7.0, dtype=torch.float32, device=DEV) if solve else None
+    nd = torch.full((1,), -1, dtype=torch.int32, device=DEV) if solve else None
+    wsb = B.qwt_qlinear_cwac_calibrate_workspace_bytes(M, N, K, wfmt)
+    ws = empty_bytes(wsb)
+    ws.fill_(0xFF)
+    B.qwt_qlinear_cwac_calibrate(dX, dxs, dW, wfmt, dws, dbias, dfp, ld, M, N, K, dstats, a, b, nd, ws, wsb)
+    B.qwt_qlinear_check_status(ws)
+    return (None if a is None else a.cpu().numpy(), None if b is None else b.cpu().numpy(),
+            None if nd is None else int(nd.item()), None if dstats is None else dstats.cpu().numpy().reshape(5, N))
