@@ -484,6 +484,28 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (r < p.M) xs4[k] = __ldg(p.x_scale + r);
         }
       }
+      // statistics: the thread's rows inside the matrix, and the first step's values of f (requested before the
+      // waits below; every later step is requested one step ahead)
+      constexpr int NB = 2;                   // statistics: 8-column blocks per step
+      bool rv[4] = {true, true, true, true};
+      const bool rows_full = y0 + 32 <= p.M;
+      float2 fnext[NB][4];
+      auto load_f = [&](int col0, float2 (&dst)[NB][4]) {
+#pragma unroll
+        for (int i = 0; i < NB; ++i) {
+          const int col = col0 + 8 * i + 2 * (lane & 3);    // N is even: a column pair is all in or all out
+#pragma unroll
+          for (int k = 0; k < 4; ++k)
+            dst[i][k] = (col < p.N && rv[k]) ? __ldcs(reinterpret_cast<const float2*>(
+                                                   p.F + (size_t)(y0 + (lane >> 2) + 8 * k) * (size_t)p.ldf + col))
+                                             : make_float2(0.f, 0.f);
+        }
+      };
+      if constexpr (C::kStats) {
+#pragma unroll
+        for (int k = 0; k < 4; ++k) rv[k] = y0 + (lane >> 2) + 8 * k < p.M;
+        load_f(n0, fnext);
+      }
       int zx4[4] = {0, 0, 0, 0}, rs4[4] = {0, 0, 0, 0};   // ASYM: zero-point and code sum of the four rows
       if (ASYM) {
 #pragma unroll
@@ -726,25 +748,17 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // 5 roundings deep) and leaves sums and shifts in shared memory; the group's 128 threads then take one
         // column each, undo the shifts in FP64, add the four warps in order and write the strip's partial.  A
         // second kernel adds the strips in a fixed order.  Rows >= M and columns >= N contribute nothing.
-        constexpr int NB = 2;                                  // 8-column blocks per step
         float* const wsum = reinterpret_cast<float*>(stg);      // [4 sums | shift of q | shift of f][128 columns]
-        bool rv[4];
-#pragma unroll
-        for (int k = 0; k < 4; ++k) rv[k] = y0 + q + 8 * k < p.M;
         if (in_range) {
-#pragma unroll 1
+#pragma unroll 2
           for (int h = 0; h < kUnitN / (8 * NB); ++h) {
             const int c0 = h * 8 * NB;                          // first column of the step inside the unit
             float2 fv[NB][4];
 #pragma unroll
-            for (int i = 0; i < NB; ++i) {
-              const int col = n0 + c0 + 8 * i + 2 * c;          // N is even: a column pair is all in or all out
+            for (int i = 0; i < NB; ++i)
 #pragma unroll
-              for (int k = 0; k < 4; ++k)
-                fv[i][k] = (col < p.N && rv[k]) ? __ldcs(reinterpret_cast<const float2*>(
-                                                      p.F + (size_t)(y0 + q + 8 * k) * (size_t)p.ldf + col))
-                                                : make_float2(0.f, 0.f);
-            }
+              for (int k = 0; k < 4; ++k) fv[i][k] = fnext[i][k];
+            if (h + 1 < kUnitN / (8 * NB)) load_f(n0 + c0 + 8 * NB, fnext);   // in flight during this step
             uint32_t a0[4 * NB], a1[4 * NB];
             ptx::tmem_ld_frag<NB>(taddr + c0, a0);
             ptx::tmem_ld_frag<NB>(taddr + (16u << 16) + c0, a1);
@@ -762,28 +776,28 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 *reinterpret_cast<float2*>(wsum + 4 * kUnitN + c0 + 8 * i + 2 * c) = kq;
                 *reinterpret_cast<float2*>(wsum + 5 * kUnitN + c0 + 8 * i + 2 * c) = kf;
               }
-              auto four_rows = [&](float z0, float z1, float z2, float z3, float f0, float f1, float f2, float f3,
-                                   float shq, float shf, float* out) {
-                const float zz[4] = {z0, z1, z2, z3}, ff[4] = {f0, f1, f2, f3};
-                float s0 = 0.f, s1 = 0.f, s2 = 0.f, s3 = 0.f;
+              if (!rows_full) {                                 // last strip only: rows >= M get shifted value 0
 #pragma unroll
-                for (int k = 0; k < 4; ++k) {
-                  const float dq = rv[k] ? zz[k] - shq : 0.f;
-                  const float df = rv[k] ? ff[k] - shf : 0.f;
-                  s0 += dq;
-                  s1 += df;
-                  s2 = fmaf(dq, df, s2);
-                  s3 = fmaf(dq, dq, s3);
-                }
-                out[0] = s0;
-                out[1] = s1;
-                out[2] = s2;
-                out[3] = s3;
-              };
-              four_rows(z[0].x, z[1].x, z[2].x, z[3].x, fv[i][0].x, fv[i][1].x, fv[i][2].x, fv[i][3].x, kq.x, kf.x,
-                        v + (2 * i) * 4);
-              four_rows(z[0].y, z[1].y, z[2].y, z[3].y, fv[i][0].y, fv[i][1].y, fv[i][2].y, fv[i][3].y, kq.y, kf.y,
-                        v + (2 * i + 1) * 4);
+                for (int k = 0; k < 4; ++k)
+                  if (!rv[k]) {
+                    z[k] = kq;
+                    fv[i][k] = kf;
+                  }
+              }
+              const float2 nkq = make_float2(-kq.x, -kq.y), nkf = make_float2(-kf.x, -kf.y);
+              float2 s0 = make_float2(0.f, 0.f), s1 = s0, s2 = s0, s3 = s0;     // .x / .y = the pair's two columns
+#pragma unroll
+              for (int k = 0; k < 4; ++k) {
+                const float2 dq = __fadd2_rn(z[k], nkq);
+                const float2 df = __fadd2_rn(fv[i][k], nkf);
+                s0 = __fadd2_rn(s0, dq);
+                s1 = __fadd2_rn(s1, df);
+                s2 = __ffma2_rn(dq, df, s2);
+                s3 = __ffma2_rn(dq, dq, s3);
+              }
+              float* o = v + (2 * i) * 4;
+              o[0] = s0.x; o[1] = s1.x; o[2] = s2.x; o[3] = s3.x;
+              o[4] = s0.y; o[5] = s1.y; o[6] = s2.y; o[7] = s3.y;
             }
             // halving butterfly over lane bits 4, 3, 2 (the row index q): at every level a lane hands one half
             // of its values to its partner and adds the partner's other half to the half it keeps
