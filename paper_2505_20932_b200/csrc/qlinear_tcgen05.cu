@@ -461,8 +461,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       for (int i = 0; i < CPR; ++i) {
         const int r = i * RPI + lane / CPR;
         uint4 v = *reinterpret_cast<const uint4*>(stg + r * BOXB + ((chunk ^ swizzle_xor<BOXB>(r)) << 4));
-        // INT8 boxes: rows 8-15 and 24-31 were written with the 8-byte halves of every chunk exchanged
-        if (C::kCodes && (r & 8) != 0) v = make_uint4(v.z, v.w, v.x, v.y);
+        // static-scale INT8 boxes: rows 8-15 and 24-31 were written with the 8-byte halves of every chunk exchanged
+        if (C::kStatic8 && (r & 8) != 0) v = make_uint4(v.z, v.w, v.x, v.y);
         if (col_ok && y + r < p.M) *reinterpret_cast<uint4*>(out + (size_t)(y + r) * p.N * ESZ) = v;
       }
       __syncwarp();                                  // the slot may be rewritten
@@ -593,7 +593,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         z[3] = z_pair(a1[2], a1[3], xs2[3], f2.x, f2.y, b2.x, b2.y);
       };
 
-      float den[4] = {1.f, 1.f, 1.f, 1.f}, inv[4] = {1.f, 1.f, 1.f, 1.f};
+      float den_row = 1.f, inv_row = 1.f;
       bool slow = false;
       if (C::kInt8Out && in_range) {
         // ---------------------------------------------------------------- phase 1: row maxima of the unit
@@ -730,12 +730,9 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const float inv_mine = __frcp_rn(den_mine);
         // a scale so small that its reciprocal overflows (never on real data): divide directly
         slow = __any_sync(0xffffffffu, !(inv_mine <= 3.0e38f));
-        // row q + 8k was handled by lane (q, k)
-#pragma unroll
-        for (int k = 0; k < 4; ++k) {
-          den[k] = __shfl_sync(0xffffffffu, den_mine, (lane & ~3) + k);
-          inv[k] = __shfl_sync(0xffffffffu, inv_mine, (lane & ~3) + k);
-        }
+        // phase 2 works on row `lane` of the warp's 32; that row's maximum sits in lane (q, c) = (lane % 8, lane / 8)
+        den_row = __shfl_sync(0xffffffffu, den_mine, 4 * (lane & 7) + (lane >> 3));
+        inv_row = __shfl_sync(0xffffffffu, inv_mine, 4 * (lane & 7) + (lane >> 3));
       }
 
       if constexpr (C::kStats) {
@@ -852,26 +849,51 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           out[2 * (size_t)p.cpad] = Sqf;
           out[3 * (size_t)p.cpad] = Sqq;
         }
-      } else if (in_range) {
-      // ------------------------------------------------------------------ conversion and store, box by box
-        // z / den rounded to nearest: q0 = z * (1/den), then one residual correction with fused multiply-adds;
-        // adding 1.5 * 2^23 leaves rne(q) in the low mantissa bits (|q| <= 127 by construction).
-        // (the whole box loop is instantiated twice so that the common case carries no branch per element)
-        auto convert_and_store = [&](auto slow_tag) {
+      } else if (C::kInt8Out && in_range) {
+        // ---------------------------------------------------------------- phase 2: codes, box by box
+        // z is read back in the 32x32b layout: thread = row, 32 consecutive columns in registers, so a row has
+        // one scale and its codes leave the thread as whole 16-byte pieces (no per-column value is needed any
+        // more).  code = rne(z * (1 / y_scale)) in one fused multiply-add: adding 1.5 * 2^23 leaves the integer
+        // in the low mantissa bits (|z / y_scale| <= 127 by construction).
+        auto codes_and_store = [&](auto slow_tag) {
           constexpr bool SLOW = decltype(slow_tag)::value;
           const float2 magic2 = make_float2(12582912.f, 12582912.f);
-          auto quant = [&](float2 z, int k) -> uint32_t {      // two codes in the low 16 bits
-            float2 qq;
-            if (C::kStatic8) {      // already in output steps: clip to the code range, then round
-              qq = make_float2(fminf(fmaxf(z.x, -127.f), 127.f), fminf(fmaxf(z.y, -127.f), 127.f));
-            } else if (SLOW) {
-              qq = make_float2(__fdiv_rn(z.x, den[k]), __fdiv_rn(z.y, den[k]));
-            } else {
-              const float2 i2 = make_float2(inv[k], inv[k]);
-              const float2 q0 = __fmul2_rn(z, i2);
-              const float2 rem = __ffma2_rn(q0, make_float2(-den[k], -den[k]), z);
-              qq = __ffma2_rn(rem, i2, q0);
+          const float2 inv2 = make_float2(inv_row, inv_row);
+          auto two = [&](uint32_t x, uint32_t y) -> uint32_t {        // two codes in the low 16 bits
+            const float2 z2 = make_float2(__uint_as_float(x), __uint_as_float(y));
+            const float2 m = SLOW ? __fadd2_rn(make_float2(__fdiv_rn(z2.x, den_row), __fdiv_rn(z2.y, den_row)), magic2)
+                                  : __ffma2_rn(z2, inv2, magic2);
+            return __byte_perm(__float_as_uint(m.x), __float_as_uint(m.y), 0x0040);
+          };
+          uint8_t* const row_base = stg + lane * BOXB;
+#pragma unroll 1
+          for (int bx = 0; bx < kUnitN / BC; ++bx) {
+            if (n0 + bx * BC >= p.N) break;
+#pragma unroll 1
+            for (int h = 0; h < BC / 32; ++h) {
+              uint32_t zr[32];
+              ptx::tmem_ld_32x32b_x32(taddr + bx * BC + h * 32, zr);
+              ptx::tmem_ld_wait();
+              uint32_t w[8];
+#pragma unroll
+              for (int j = 0; j < 8; ++j)
+                w[j] = __byte_perm(two(zr[4 * j], zr[4 * j + 1]), two(zr[4 * j + 2], zr[4 * j + 3]), 0x5410);
+              *reinterpret_cast<uint4*>(row_base + (((uint32_t)(2 * h) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
+              *reinterpret_cast<uint4*>(row_base + (((uint32_t)(2 * h + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
             }
+            store_box(n0 + bx * BC, y0);
+          }
+        };
+        if (slow) codes_and_store(std::true_type{});
+        else codes_and_store(std::false_type{});
+      } else if (in_range) {
+      // ------------------------------------------------------------------ conversion and store, box by box
+        {
+          const float2 magic2 = make_float2(12582912.f, 12582912.f);
+          // static scales: z is already in output steps; clip to the code range, then round (adding 1.5 * 2^23
+          // leaves the integer in the low mantissa bits)
+          auto quant = [&](float2 z) -> uint32_t {             // two codes in the low 16 bits
+            const float2 qq = make_float2(fminf(fmaxf(z.x, -127.f), 127.f), fminf(fmaxf(z.y, -127.f), 127.f));
             const float2 m = __fadd2_rn(qq, magic2);
             return __byte_perm(__float_as_uint(m.x), __float_as_uint(m.y), 0x0040) & 0xffffu;
           };
@@ -894,7 +916,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
               for (int i = 0; i < NB; ++i) {
                 const int colb = h * LDC + 8 * i;      // first column of the block inside the box
-                if (ASYM && !C::kInt8Out) asym_fix(a0 + 4 * i, a1 + 4 * i, c0 + 8 * i);
+                if (ASYM) asym_fix(a0 + 4 * i, a1 + 4 * i, c0 + 8 * i);
                 if (OUT == QWT_OUT_INT32_ACC) {
                   // W4: every term is a multiple of 16, the shift is exact
                   auto fix = [](uint32_t v) { return W4 ? (uint32_t)((int)v >> 4) : v; };
@@ -905,14 +927,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                   *reinterpret_cast<uint2*>(stage_at(q + 24, b)) = make_uint2(fix(a1[4 * i + 2]), fix(a1[4 * i + 3]));
                 } else {
                   float2 z[4];
-                  if (C::kInt8Out) {      // phase 1 left z in TMEM
-                    z[0] = make_float2(__uint_as_float(a0[4 * i]), __uint_as_float(a0[4 * i + 1]));
-                    z[1] = make_float2(__uint_as_float(a0[4 * i + 2]), __uint_as_float(a0[4 * i + 3]));
-                    z[2] = make_float2(__uint_as_float(a1[4 * i]), __uint_as_float(a1[4 * i + 1]));
-                    z[3] = make_float2(__uint_as_float(a1[4 * i + 2]), __uint_as_float(a1[4 * i + 3]));
-                  } else {
-                    z_block(a0 + 4 * i, a1 + 4 * i, c0 + 8 * i, z);
-                  }
+                  z_block(a0 + 4 * i, a1 + 4 * i, c0 + 8 * i, z);
                   if (OUT == QWT_OUT_FP32) {
                     const int b = (colb + 2 * c) * 4;
 #pragma unroll
@@ -925,7 +940,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                   } else {
                     // INT8: neighbouring lanes (c even / odd) swap halves so that each ends up with 4 consecutive
                     // codes of two rows: the even lane keeps rows q, q + 16, the odd lane rows q + 8, q + 24
-                    const uint32_t h0 = quant(z[0], 0), h1 = quant(z[1], 1), h2 = quant(z[2], 2), h3 = quant(z[3], 3);
+                    const uint32_t h0 = quant(z[0]), h1 = quant(z[1]), h2 = quant(z[2]), h3 = quant(z[3]);
                     const bool odd = (c & 1) != 0;
                     const uint32_t send = odd ? (h0 | (h2 << 16)) : (h1 | (h3 << 16));
                     const uint32_t recv = __shfl_xor_sync(0xffffffffu, send, 1);
@@ -943,9 +958,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
             store_box((n0 + bx * BC) * ESZ, y0);
           }
-        };
-        if (C::kInt8Out && slow) convert_and_store(std::true_type{});
-        else convert_and_store(std::false_type{});
+        }
       }
       // the accumulator buffer and the group's parameter slice are free again
       ptx::tc_fence_before();
