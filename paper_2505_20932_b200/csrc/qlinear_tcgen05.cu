@@ -593,6 +593,16 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         z[3] = z_pair(a1[2], a1[3], xs2[3], f2.x, f2.y, b2.x, b2.y);
       };
 
+      // The accumulator buffer is handed back to the tensor pipe as soon as this warp has read the last of it
+      // (the arithmetic and the stores of the last box then overlap the next tile's MMAs).
+      bool released = false;
+      auto release_acc = [&]() {
+        ptx::tc_fence_before();
+        __syncwarp();
+        if (lane == 0) ptx::mbar_arrive(&tempty[buf]);
+        released = true;
+      };
+      const int boxes_in = in_range ? ((p.N - n0 + BC - 1) / BC < kUnitN / BC ? (p.N - n0 + BC - 1) / BC : kUnitN / BC) : 0;
       float den_row = 1.f, inv_row = 1.f;
       bool slow = false;
       if (C::kInt8Out && in_range) {
@@ -760,6 +770,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             ptx::tmem_ld_frag<NB>(taddr + c0, a0);
             ptx::tmem_ld_frag<NB>(taddr + (16u << 16) + c0, a1);
             ptx::tmem_ld_wait();
+            if (h + 1 == kUnitN / (8 * NB)) release_acc();
             float v[8 * NB];                                    // [(block, column of the pair)][sum]
 #pragma unroll
             for (int i = 0; i < NB; ++i) {
@@ -874,6 +885,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               uint32_t zr[32];
               ptx::tmem_ld_32x32b_x32(taddr + bx * BC + h * 32, zr);
               ptx::tmem_ld_wait();
+              if (bx + 1 == boxes_in && h + 1 == BC / 32) release_acc();
               uint32_t w[8];
 #pragma unroll
               for (int j = 0; j < 8; ++j)
@@ -913,6 +925,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               ptx::tmem_ld_frag<NB>(taddr + c0, a0);
               ptx::tmem_ld_frag<NB>(taddr + (16u << 16) + c0, a1);
               ptx::tmem_ld_wait();
+              if (bx + 1 == boxes_in && h + 1 == BC / LDC) release_acc();
 #pragma unroll
               for (int i = 0; i < NB; ++i) {
                 const int colb = h * LDC + 8 * i;      // first column of the block inside the box
@@ -960,13 +973,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
       }
-      // the accumulator buffer and the group's parameter slice are free again
-      ptx::tc_fence_before();
+      // the group's parameter slice is free again (and the accumulator buffer, if nothing of the unit was read)
+      if (!released) release_acc();
       __syncwarp();
-      if (lane == 0) {
-        ptx::mbar_arrive(&tempty[buf]);
-        ptx::mbar_arrive(&gdone[g]);
-      }
+      if (lane == 0) ptx::mbar_arrive(&gdone[g]);
     }
   }
 
