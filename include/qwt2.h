@@ -150,7 +150,9 @@ qwt_status qwt_cwac_fold_static(const float* w_scale, const float* bias, const f
  *     z[m, n]   = fma((float)acc[m, n] * x_scale[m], fscale[n], fbias[n])      (Eq. 9 after the fold)
  *   QWT_OUT_INT8_PER_TOKEN: y_scale[m] = max_n |z[m, n]| / 127;  Y[m, n] = clip(rne(z / y_scale[m]), -127, 127)
  *                           (Eq. 1-2 applied to the output with zero-point 0: the 1/S_r of Eq. 10-11, per token);
- *                           a row of zeros gives y_scale 0 and codes 0.
+ *                           a row of zeros gives y_scale 0 and codes 0.  The kernel rounds z * (1 / y_scale[m])
+ *                           (FP32 reciprocal, one fused multiply-add), which differs from the FP32 quotient by
+ *                           one step in about one code per million.
  *   QWT_OUT_BF16 / FP32   : Y = z rounded to bfloat16 / as is.       QWT_OUT_INT32_ACC: Y = acc.
  *   QWT_OUT_INT8_STATIC   : Y[m, n] = clip(rne(fscale[n] * (acc[m, n] + offset[n])), -127, 127) with fscale = mult and
  *                           fbias = the INT32 offset array of qwt_cwac_fold_static passed through the same pointer

@@ -106,6 +106,7 @@ struct Cfg {
   static constexpr bool kStatic8 = OUT == QWT_OUT_INT8_STATIC;       // Eq. 10 as printed: static multiplier + offset
   static constexpr bool kCodes = kInt8Out || kStatic8;               // one byte per output element
   static constexpr bool kStats = OUT == kOutCalibStats;              // no output matrix: per-channel sums of Eq. 4-5
+  static constexpr bool kTmaStore = !kStatic8 && !kStats;            // staging boxes leave by cp.async.bulk.tensor
   static constexpr bool kHasParams = OUT != QWT_OUT_INT32_ACC;       // x_scale / fscale / fbias are used
   static constexpr bool kNeedSlice = kHasParams || ASYM;             // per-column values staged in shared memory
   static constexpr int kEsz = kCodes ? 1 : (OUT == QWT_OUT_BF16 ? 2 : 4);
@@ -174,7 +175,7 @@ __device__ __forceinline__ float2 z_pair(uint32_t a0, uint32_t a1, float2 xs2, f
 template <int BN, int OUT, bool W4, bool WIDE, bool ASYM>
 __global__ void __launch_bounds__((Cfg<BN, OUT, W4, WIDE, ASYM>::kThreads), 1)
 qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
-                    const QlParams p) {
+                    const __grid_constant__ CUtensorMap tmY, const QlParams p) {
   using C = Cfg<BN, OUT, W4, WIDE, ASYM>;
   constexpr int kAcc = C::kAcc;
   constexpr int kMaxStages = C::kMaxStages;
@@ -231,6 +232,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     ptx::fence_mbar_init();
     ptx::prefetch_tensormap(&tmA);
     ptx::prefetch_tensormap(&tmB);
+    if (C::kTmaStore) ptx::prefetch_tensormap(&tmY);
   }
   if (warp == 1) {
     ptx::tmem_alloc(tmem_slot, kTmemCols);
@@ -466,6 +468,22 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (col_ok && y + r < p.M) *reinterpret_cast<uint4*>(out + (size_t)(y + r) * p.N * ESZ) = v;
       }
       __syncwarp();                                  // the slot may be rewritten
+    };
+
+    // The same box by a bulk tensor store issued by one lane: the LSU sees nothing of it and the warp goes on
+    // at once.  The staging slot may be rewritten when the copy has read it: slot_free() before the next box's
+    // first write (by then the copy has usually had the next box's TMEM load and arithmetic to finish reading).
+    auto tma_box = [&](int x_bytes, int y) {
+      ptx::fence_proxy_async_smem();                 // this lane's writes to the slot, for the async proxy
+      __syncwarp();
+      if (lane == 0) {
+        if (y < p.M) ptx::tma_store_2d(&tmY, stg, x_bytes, y);
+        ptx::bulk_commit_group();
+      }
+    };
+    auto slot_free = [&]() {
+      if (lane == 0) ptx::bulk_wait_read_all();
+      __syncwarp();
     };
 
     int use = 0;                            // units this group has handled
@@ -890,10 +908,11 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
               for (int j = 0; j < 8; ++j)
                 w[j] = __byte_perm(two(zr[4 * j], zr[4 * j + 1]), two(zr[4 * j + 2], zr[4 * j + 3]), 0x5410);
+              if (h == 0) slot_free();
               *reinterpret_cast<uint4*>(row_base + (((uint32_t)(2 * h) ^ swz) << 4)) = make_uint4(w[0], w[1], w[2], w[3]);
               *reinterpret_cast<uint4*>(row_base + (((uint32_t)(2 * h + 1) ^ swz) << 4)) = make_uint4(w[4], w[5], w[6], w[7]);
             }
-            store_box(n0 + bx * BC, y0);
+            tma_box(n0 + bx * BC, y0);
           }
         };
         if (slow) codes_and_store(std::true_type{});
@@ -926,6 +945,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               ptx::tmem_ld_frag<NB>(taddr + (16u << 16) + c0, a1);
               ptx::tmem_ld_wait();
               if (bx + 1 == boxes_in && h + 1 == BC / LDC) release_acc();
+              if (C::kTmaStore && h == 0) slot_free();
 #pragma unroll
               for (int i = 0; i < NB; ++i) {
                 const int colb = h * LDC + 8 * i;      // first column of the block inside the box
@@ -969,7 +989,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 }
               }
             }
-            store_box((n0 + bx * BC) * ESZ, y0);
+            if (C::kTmaStore) tma_box((n0 + bx * BC) * ESZ, y0);
+            else store_box((n0 + bx * BC) * ESZ, y0);
           }
         }
       }
@@ -978,6 +999,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       __syncwarp();
       if (lane == 0) ptx::mbar_arrive(&gdone[g]);
     }
+    if (C::kTmaStore && lane == 0) ptx::bulk_wait_all();     // the stores of this warp's boxes are complete
   }
 
   // ------------------------------------------------------------------ teardown
@@ -1043,6 +1065,16 @@ qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams p
   using C = Cfg<BN, OUT, W4, WIDE, ASYM>;
   constexpr int kThreads = C::kThreads;
   auto kern = qlinear_cwac_kernel<BN, OUT, W4, WIDE, ASYM>;
+  // output map: Y as a byte matrix, one staging box (32 rows x kBoxBytes, in the box's own swizzle) per copy
+  CUtensorMap tmY = tmA;
+  if (C::kTmaStore) {
+    constexpr CUtensorMapSwizzle swz = C::kBoxBytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
+                                       : (C::kBoxBytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
+    if (!make_byte_map(&tmY, prm.Y, (uint64_t)prm.M, (uint64_t)prm.N * C::kEsz, C::kBoxBytes, 32, swz)) {
+      set_cuda_error((int)cudaErrorInvalidValue);
+      return QWT_ERR_CUDA;
+    }
+  }
   prm.res_kb = res_kb;
   prm.stages = C::stages_for(res_kb);
   const int smem_bytes = C::dynamic_bytes(prm.stages, res_kb);
@@ -1056,11 +1088,11 @@ qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams p
   }
   if (C::kInt8Out) {
     // the row-maximum exchange needs every CTA of the grid resident
-    void* args[] = {(void*)&tmA, (void*)&tmB, (void*)&prm};
+    void* args[] = {(void*)&tmA, (void*)&tmB, (void*)&tmY, (void*)&prm};
     QWT_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, smem_bytes, st));
     count_launch();
   } else {
-    kern<<<grid, kThreads, smem_bytes, st>>>(tmA, tmB, prm);
+    kern<<<grid, kThreads, smem_bytes, st>>>(tmA, tmB, tmY, prm);
     QWT_LAUNCH_CHECK();
   }
   return QWT_OK;
