@@ -59,7 +59,9 @@ constexpr int kUmmaK = 32;         // K of one kind::i8 instruction
 constexpr int kTmemCols = 512;
 constexpr int kGroupWarps = 4;        // warps of an epilogue group (one per TMEM lane quadrant)
 constexpr int kGroups = 4;            // epilogue groups; a group works on one 128-column unit of a tile at a time
-constexpr int kUnitN = 128;           // columns of an epilogue unit (512 TMEM columns = 4 units in flight)
+// Columns of an epilogue unit: 128 in every mode (512 TMEM columns = 4 units in flight, one per group).  64-column
+// units, which let the four groups share one tile, were measured slower on short-K layers and are left selectable here.
+__host__ __device__ constexpr int unit_cols(int /*out_mode*/) { return 128; }
 constexpr int kEpiWarps = kGroupWarps * kGroups;
 constexpr int kNumConvWarps = 4;      // W4 -> INT8 converter warps (packed weights only)
 constexpr int kABytes = kBM * kBK;
@@ -111,6 +113,7 @@ struct Cfg {
   static constexpr bool kNeedSlice = kHasParams || ASYM;             // per-column values staged in shared memory
   static constexpr int kEsz = kCodes ? 1 : (OUT == QWT_OUT_BF16 ? 2 : 4);
   static constexpr int kAcc = kTmemCols / BN;                        // accumulator buffers (tiles) in TMEM
+  static constexpr int kUnitN = unit_cols(OUT);                      // columns of an epilogue unit
   static constexpr int kUPT = BN / kUnitN;                           // epilogue units per tile
   static constexpr int kConvWarp0 = 2 + kEpiWarps;                   // first converter warp (W4 only)
   static constexpr int kThreads = 32 * (2 + kEpiWarps + (W4 ? kNumConvWarps : 0));
@@ -118,7 +121,7 @@ struct Cfg {
   // row-contiguous global stores.  128-byte rows for 128-wide tiles; 256-wide tiles use 32-byte rows when the
   // operand ring needs the room (long K: the epilogue hides behind the mainloop) and 64-byte rows otherwise
   // (statistics: the slot holds the warp's four sums and two shifts of the unit's 128 columns, 3 KB)
-  static constexpr int kBoxBytes = kStats ? 96 : (BN == 128 ? 128 : (WIDE ? 64 : 32));
+  static constexpr int kBoxBytes = kStats ? 96 : (BN == 128 ? (kStatic8 && kUnitN < 128 ? 64 : 128) : (WIDE ? 64 : 32));
   static constexpr int kBC = kBoxBytes / kEsz;                       // columns per box
   static constexpr int kSlotBytes = 32 * kBoxBytes;
   static constexpr int kStagingBytes = kEpiWarps * kSlotBytes;
@@ -402,9 +405,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
   } else {
     // ------------------------------------------------------------------ epilogue warps
-    // Work item = one unit: 128 columns of a tile.  The CTA's units are numbered u = j * kUPT + half
-    // (j = local tile); group g takes u = g, g + 4, ...  Unit u lives in TMEM columns (u % 4) * 128.
+    // Work item = one unit: kUnitN columns of a tile.  The CTA's units are numbered u = j * kUPT + part
+    // (j = local tile); group g takes u = g, g + 4, ...  Unit u lives in its tile's accumulator buffer, part by part.
     constexpr int UPT = C::kUPT;
+    constexpr int kUnitN = C::kUnitN;
     constexpr int BOXB = C::kBoxBytes;
     constexpr int BC = C::kBC;              // columns per staging box
     constexpr int ESZ = C::kEsz;
@@ -419,7 +423,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     int* const ps_c1 = reinterpret_cast<int*>(ps_fs + 2 * kUnitN);   // ASYM: -Z_W, then K Z_W - column sum of W_q
     int* const ps_cd = ps_c1 + kUnitN;
     int pre_c1[kUnitN / 32], pre_cd[kUnitN / 32];
-    const uint32_t taddr = tmem_base + ((uint32_t)(qd * 32) << 16) + g * kUnitN;
+    const uint32_t taddr_q = tmem_base + ((uint32_t)(qd * 32) << 16);   // this warp's lane quadrant, column 0
     const int n_units = n_local * UPT;
     float pre_fs[kUnitN / 32], pre_fb[kUnitN / 32];
 
@@ -494,6 +498,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int n0 = unit_col0(u);
       const uint32_t buf = j % kAcc, tpar = (j / kAcc) & 1u, upar = use & 1u;
       const int y0 = tm * kBM + qd * 32;
+      const uint32_t taddr = taddr_q + buf * BN + (uint32_t)(u % UPT) * kUnitN;   // the unit's columns in TMEM
       float xs4[4] = {0.f, 0.f, 0.f, 0.f};    // x_scale of the thread's four rows, requested before the waits below
       if (C::kHasParams && !C::kStatic8) {
 #pragma unroll
@@ -945,31 +950,33 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
               ptx::tmem_ld_frag<NB>(taddr + (16u << 16) + c0, a1);
               ptx::tmem_ld_wait();
               if (bx + 1 == boxes_in && h + 1 == BC / LDC) release_acc();
-              if (C::kTmaStore && h == 0) slot_free();
+              // words of one 8-column block of the thread: 2 per row (FP32, INT32) or 1 per row (BF16)
+              constexpr int WPB = C::kEsz == 4 ? 8 : 4;
+              uint32_t ow[C::kTmaStore ? NB * WPB : 1];
 #pragma unroll
               for (int i = 0; i < NB; ++i) {
                 const int colb = h * LDC + 8 * i;      // first column of the block inside the box
                 if (ASYM) asym_fix(a0 + 4 * i, a1 + 4 * i, c0 + 8 * i);
-                if (OUT == QWT_OUT_INT32_ACC) {
+                if constexpr (OUT == QWT_OUT_INT32_ACC) {
                   // W4: every term is a multiple of 16, the shift is exact
                   auto fix = [](uint32_t v) { return W4 ? (uint32_t)((int)v >> 4) : v; };
-                  const int b = (colb + 2 * c) * 4;
-                  *reinterpret_cast<uint2*>(stage_at(q, b)) = make_uint2(fix(a0[4 * i]), fix(a0[4 * i + 1]));
-                  *reinterpret_cast<uint2*>(stage_at(q + 8, b)) = make_uint2(fix(a0[4 * i + 2]), fix(a0[4 * i + 3]));
-                  *reinterpret_cast<uint2*>(stage_at(q + 16, b)) = make_uint2(fix(a1[4 * i]), fix(a1[4 * i + 1]));
-                  *reinterpret_cast<uint2*>(stage_at(q + 24, b)) = make_uint2(fix(a1[4 * i + 2]), fix(a1[4 * i + 3]));
+#pragma unroll
+                  for (int k = 0; k < 4; ++k) {
+                    ow[i * WPB + 2 * k] = fix(k < 2 ? a0[4 * i + 2 * k] : a1[4 * i + 2 * k - 4]);
+                    ow[i * WPB + 2 * k + 1] = fix(k < 2 ? a0[4 * i + 2 * k + 1] : a1[4 * i + 2 * k - 3]);
+                  }
                 } else {
                   float2 z[4];
                   z_block(a0 + 4 * i, a1 + 4 * i, c0 + 8 * i, z);
-                  if (OUT == QWT_OUT_FP32) {
-                    const int b = (colb + 2 * c) * 4;
+                  if constexpr (OUT == QWT_OUT_FP32) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k) *reinterpret_cast<float2*>(stage_at(q + 8 * k, b)) = z[k];
-                  } else if (OUT == QWT_OUT_BF16) {
-                    const int b = (colb + 2 * c) * 2;
+                    for (int k = 0; k < 4; ++k) {
+                      ow[i * WPB + 2 * k] = __float_as_uint(z[k].x);
+                      ow[i * WPB + 2 * k + 1] = __float_as_uint(z[k].y);
+                    }
+                  } else if constexpr (OUT == QWT_OUT_BF16) {
 #pragma unroll
-                    for (int k = 0; k < 4; ++k)
-                      *reinterpret_cast<uint32_t*>(stage_at(q + 8 * k, b)) = pack_bf16x2(z[k].x, z[k].y);
+                    for (int k = 0; k < 4; ++k) ow[i * WPB + k] = pack_bf16x2(z[k].x, z[k].y);
                   } else {
                     // INT8: neighbouring lanes (c even / odd) swap halves so that each ends up with 4 consecutive
                     // codes of two rows: the even lane keeps rows q, q + 16, the odd lane rows q + 8, q + 24
@@ -985,6 +992,22 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const int b = (colb + 2 * (c & ~1)) ^ (odd ? 8 : 0);
                     *reinterpret_cast<uint32_t*>(stage_at(odd ? q + 8 : q, b)) = wa;
                     *reinterpret_cast<uint32_t*>(stage_at(odd ? q + 24 : q + 16, b)) = wb;
+                  }
+                }
+              }
+              if constexpr (C::kTmaStore) {
+                // the slot is written only now: the copy of the previous box has had this box's TMEM load and
+                // arithmetic to finish reading it
+                if (h == 0) slot_free();
+#pragma unroll
+                for (int i = 0; i < NB; ++i) {
+                  const int b = (h * LDC + 8 * i + 2 * c) * C::kEsz;
+#pragma unroll
+                  for (int k = 0; k < 4; ++k) {
+                    if constexpr (C::kEsz == 4)
+                      *reinterpret_cast<uint2*>(stage_at(q + 8 * k, b)) = make_uint2(ow[i * WPB + 2 * k], ow[i * WPB + 2 * k + 1]);
+                    else
+                      *reinterpret_cast<uint32_t*>(stage_at(q + 8 * k, b)) = ow[i * WPB + k];
                   }
                 }
               }
@@ -1198,7 +1221,7 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   pl.ws_status_off = off;
   off += 256;
   pl.ws_partial_off = off;      // (tag, row maximum) per strip row and 128-column unit
-  const int strip_units = (N + kUnitN - 1) / kUnitN;
+  const int strip_units = (N + unit_cols(out_mode) - 1) / unit_cols(out_mode);
   pl.gather_words = strip_units <= 16 ? strip_units : 0;
   if (out_mode == QWT_OUT_INT8_PER_TOKEN) {
     if (pl.gather_words > 0) {
@@ -1248,7 +1271,8 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   prm.num_kb = (K + kBK - 1) / kBK;
   prm.status = reinterpret_cast<uint32_t*>(ws + plan.ws_status_off);
   prm.partial = reinterpret_cast<unsigned long long*>(ws + plan.ws_partial_off);
-  prm.counter_target = (uint32_t)((N + kUnitN - 1) / kUnitN);   // units of a row strip that lie inside the matrix
+  // units of a row strip that lie inside the matrix
+  prm.counter_target = (uint32_t)((N + unit_cols(out_mode) - 1) / unit_cols(out_mode));
   prm.gather_words = plan.gather_words;
   prm.x_zero = x_zero;
   prm.x_rowsum = x_rowsum;
