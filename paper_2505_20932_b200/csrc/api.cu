@@ -350,7 +350,9 @@ qwt_status fused_calib_layout(int32_t M, int32_t N, int32_t K, int32_t wfmt, Fus
   L->red.chunk_rows = 128;
   L->red.partial_bytes = (size_t)L->red.chunks * 4 * L->red.cpad * sizeof(double);
   L->off_partial = 256;
-  L->total = L->off_partial + L->red.partial_bytes;
+  // the expanded int8 copy of packed weights (if the plan asks for one) goes behind the partials
+  L->plan.ws_w_off = (L->off_partial + L->red.partial_bytes + 255) / 256 * 256;
+  L->total = L->plan.ws_w_off + (L->plan.w4_expand ? (size_t)N * (size_t)K : 0);
   return QWT_OK;
 }
 }  // namespace

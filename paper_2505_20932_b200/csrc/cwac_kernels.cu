@@ -359,6 +359,26 @@ pack_int4_kernel(const int8_t* __restrict__ codes, int64_t n_bytes, uint8_t* __r
   packed[i] = (uint8_t)((lo & 0xF) | ((hi & 0xF) << 4));
 }
 
+// Packed int4 -> int8 codes (two's-complement nibbles, even element in the low half): 16 packed bytes per thread.
+__global__ void __launch_bounds__(256)
+unpack_int4_kernel(const uint4* __restrict__ packed, int64_t n_vec, uint4* __restrict__ codes) {
+  const int64_t i = (int64_t)blockIdx.x * blockDim.x + threadIdx.x;
+  if (i >= n_vec) return;
+  const uint4 w = __ldg(packed + i);
+  const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+  uint32_t out[8];
+#pragma unroll
+  for (int k = 0; k < 4; ++k) {
+    // sign extension of a nibble n: (n ^ 8) - 8, on four bytes at a time
+    const uint32_t lo = __vsub4((in[k] & 0x0F0F0F0Fu) ^ 0x08080808u, 0x08080808u);         // even elements
+    const uint32_t hi = __vsub4(((in[k] >> 4) & 0x0F0F0F0Fu) ^ 0x08080808u, 0x08080808u);  // odd elements
+    out[2 * k] = __byte_perm(lo, hi, 0x5140);
+    out[2 * k + 1] = __byte_perm(lo, hi, 0x7362);
+  }
+  codes[2 * i] = make_uint4(out[0], out[1], out[2], out[3]);
+  codes[2 * i + 1] = make_uint4(out[4], out[5], out[6], out[7]);
+}
+
 // ------------------------------------------------------------------------------------------------ host side
 
 CwacPlan cwac_plan(int64_t rows, int32_t channels, int /*sm_count*/) {
@@ -472,6 +492,15 @@ qwt_status launch_im2col_i8(const int8_t* X, int32_t Bn, int32_t H, int32_t W, i
 qwt_status launch_pack_int4(const int8_t* codes, int64_t rows, int32_t cols, uint8_t* packed, cudaStream_t st) {
   const int64_t n_bytes = rows * (int64_t)(cols / 2);
   pack_int4_kernel<<<(unsigned)((n_bytes + 255) / 256), 256, 0, st>>>(codes, n_bytes, packed);
+  QWT_LAUNCH_CHECK();
+  return QWT_OK;
+}
+
+// packed: [rows, cols / 2] with cols % 32 == 0, 16-byte aligned; codes: int8 [rows, cols], 16-byte aligned
+qwt_status launch_unpack_int4(const void* packed, int64_t rows, int32_t cols, int8_t* codes, cudaStream_t st) {
+  const int64_t n_vec = rows * (int64_t)(cols / 32);
+  unpack_int4_kernel<<<(unsigned)((n_vec + 255) / 256), 256, 0, st>>>(static_cast<const uint4*>(packed), n_vec,
+                                                                     reinterpret_cast<uint4*>(codes));
   QWT_LAUNCH_CHECK();
   return QWT_OK;
 }

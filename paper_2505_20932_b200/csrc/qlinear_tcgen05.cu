@@ -1184,6 +1184,16 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
                         QlinearPlan* plan) {
   QlinearPlan pl{};
   pl.tiles_m = (M + kBM - 1) / kBM;
+  // Packed int4 weights: with many rows the layer is compute-bound, and converting the W tile on chip for every
+  // CTA and k-block holds the tensor pipe at about half its int8 rate (4 converter warps per CTA).  The weights are
+  // then expanded once per call into the workspace (1.5 N K bytes of traffic) and the int8 kernel runs; with few
+  // rows (weight-bandwidth-bound) the packed tile is streamed and converted on chip.
+  {
+    const char* e = getenv("QWT_W4_EXPAND");
+    const bool many_rows = M >= 1024;
+    pl.w4_expand = wfmt == QWT_W_INT4_PACKED && (e != nullptr ? e[0] == '1' : many_rows);
+  }
+  if (pl.w4_expand) wfmt = QWT_W_INT8;        // everything below plans the int8 kernel
   // 256-wide tiles keep the tensor pipe ahead of shared-memory bandwidth and are used when the mainloop
   // dominates (long K); short-K layers are bound by the epilogue, which is organised around 128-wide tiles
   // (four accumulator buffers, so the INT8 row-maximum exchange can trail by two tiles).
@@ -1232,6 +1242,9 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   }
   pl.ws_z_off = off;
   if (out_mode == QWT_OUT_INT8_PER_TOKEN && !pl.fused_requant) off += (size_t)M * N * 4;
+  off = (off + 255) / 256 * 256;
+  pl.ws_w_off = off;
+  if (pl.w4_expand) off += (size_t)N * (size_t)K;
   pl.ws_total = off;
   *plan = pl;
   return QWT_OK;
@@ -1242,8 +1255,15 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
                           float* y_scale, void* workspace, const QlinearPlan& plan, cudaStream_t st,
                           const int32_t* x_zero, const int32_t* x_rowsum, const int32_t* w_terms,
                           const QlinearStatsArgs* stats) {
-  const bool w4 = wfmt == QWT_W_INT4_PACKED;
   uint8_t* ws = static_cast<uint8_t*>(workspace);
+  if (plan.w4_expand) {
+    int8_t* w8 = reinterpret_cast<int8_t*>(ws + plan.ws_w_off);
+    qwt_status su = launch_unpack_int4(W, N, K, w8, st);
+    if (su != QWT_OK) return su;
+    W = w8;
+    wfmt = QWT_W_INT8;
+  }
+  const bool w4 = wfmt == QWT_W_INT4_PACKED;
   CUtensorMap tmA, tmB;
   const bool okA = make_byte_map(&tmA, X, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
   const bool okB = w4 ? make_byte_map(&tmB, W, (uint64_t)N, (uint64_t)K / 2, kBK / 2, (uint32_t)plan.bn,

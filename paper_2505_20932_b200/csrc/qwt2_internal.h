@@ -65,6 +65,7 @@ qwt_status launch_quantize_rows(const float* X, int64_t rows, int32_t cols, int6
                                 float* scale, cudaStream_t st);
 qwt_status launch_im2col_i8(const int8_t* X, int32_t Bn, int32_t H, int32_t W, int32_t C, int32_t kh, int32_t kw,
                             int32_t stride, int32_t pad, int8_t* P, cudaStream_t st);
+qwt_status launch_unpack_int4(const void* packed, int64_t rows, int32_t cols, int8_t* codes, cudaStream_t st);
 qwt_status launch_pack_int4(const int8_t* codes, int64_t rows, int32_t cols, uint8_t* packed, cudaStream_t st);
 
 // ---- forward (qlinear_tcgen05.cu)
@@ -75,7 +76,9 @@ struct QlinearPlan {
   bool fused_requant;    // cross-CTA row-max protocol inside the GEMM kernel
   int gather_words;      // INT8 output: exchange words per row (one per 128-column unit; 0 = counter protocol)
   bool w_resident;       // grid is a multiple of tiles_n: a CTA's W tile can stay in shared memory
-  size_t ws_status_off, ws_partial_off, ws_z_off, ws_total;
+  bool w4_expand;        // packed int4 weights are expanded to int8 in the workspace first (many rows: the GEMM is
+                         // compute-bound and the int8 mainloop is twice as fast as the one that converts on chip)
+  size_t ws_status_off, ws_partial_off, ws_z_off, ws_w_off, ws_total;
 };
 qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
                         QlinearPlan* plan);

@@ -283,3 +283,17 @@ def test_convolution_through_the_patch_matrix(H, B, Bn, Hh, Ww, C, N, k, stride,
     fb = (0.01 * rng.standard_normal(N)).astype(np.float32)
     z, _ = H.gpu_forward(Ph, xs, Wq.reshape(N, K), fs, fb, B.QWT_OUT_FP32)
     assert_fp32_close(z, O.forward_folded(acc_ref, xs, fs, fb))
+
+
+@pytest.mark.parametrize("M,N,K,expand", [(300, 2304, 768, "1"), (2000, 384, 1536, "0"), (130, 272, 416, "1")])
+def test_w4_both_weight_paths(H, B, M, N, K, expand, monkeypatch):
+    """Packed weights are either converted on chip per tile or expanded once into the workspace (the default above
+    1024 rows); both paths give the same integers."""
+    monkeypatch.setenv("QWT_W4_EXPAND", expand)
+    Xq, Wq, Wp, xs, fs, fb = random_w4_layer(M, N, K, seed=M + N + K + 11)
+    acc, _ = H.gpu_forward(Xq, None, Wp, None, None, B.QWT_OUT_INT32_ACC, wfmt=B.QWT_W_INT4_PACKED, K=K)
+    assert np.array_equal(acc.astype(np.int64), O.int_matmul(Xq, Wq))
+    codes, ys = H.gpu_forward(Xq, xs, Wp, fs, fb, B.QWT_OUT_INT8_PER_TOKEN, wfmt=B.QWT_W_INT4_PACKED, K=K)
+    c_ref, ys_ref = O.requant_per_token(O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb))
+    assert np.allclose(ys, ys_ref, rtol=1e-5)
+    assert_codes_close(codes, c_ref)
