@@ -25,7 +25,7 @@
 // The epilogue of a tile therefore has two phases and the accumulators stay in TMEM between them:
 //   phase 1  z from the accumulators (written back to TMEM in their place) -> row maxima of the unit (combined
 //            over the four lanes that share a row) -> published to the other CTAs of the strip:
-//            as a tagged 8-byte word per row and unit (strips of at most 16 units), or by atomicMax on
+//            as a tagged 8-byte word per row and unit (strips of at most 32 units), or by atomicMax on
 //            rowmax[m] plus a strip counter and flag (wider layers);
 //   phase 2  once the maxima of every unit of the strip are there, the rows' scales follow (the unit at column
 //            0 writes y_scale); z is read back from TMEM, divided, rounded and stored as codes; only then is
@@ -57,6 +57,7 @@ constexpr int kBM = 128;           // rows of a CTA tile (= TMEM lanes)
 constexpr int kBK = 128;           // bytes of K per stage: one 128-byte swizzle row
 constexpr int kUmmaK = 32;         // K of one kind::i8 instruction
 constexpr int kTmemCols = 512;
+constexpr int kMaxGatherWords = 32;   // per-token INT8: strips of up to this many units exchange tagged words
 constexpr int kGroupWarps = 4;        // warps of an epilogue group (one per TMEM lane quadrant)
 constexpr int kGroups = 4;            // epilogue groups; a group works on one 128-column unit of a tile at a time
 // Columns of an epilogue unit: 128 in every mode (512 TMEM columns = 4 units in flight, one per group).  64-column
@@ -668,7 +669,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int my = q + 8 * c;             // row (inside the warp's 32) this lane publishes and fetches
         const int row = y0 + my;
         // Exchange of the row maxima between the CTAs of a row strip (all words start at zero):
-        //  - up to 16 units per strip: every unit stores (tag 1, its maximum) in an 8-byte word of its own per
+        //  - up to 32 units per strip: every unit stores (tag 1, its maximum) in an 8-byte word of its own per
         //    row -- a single aligned 8-byte access is indivisible, so no fence is needed -- and a thread polls
         //    the words of its row until all are tagged (one store, then loads that hit L2);
         //  - wider layers (their long mainloop hides the extra round trips): atomicMax into rowmax[m] (a
@@ -686,16 +687,22 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           uint32_t polls = 0;
           uint64_t t0 = 0;
           while (true) {
-            unsigned long long w[16];
-#pragma unroll
-            for (int v = 0; v < 16; ++v) w[v] = v < strip_units ? ptx::ld_relaxed_gpu_u64(slot + (size_t)v * kBM) : (1ull << 32);
             bool all = true;
             float m = 0.f;
+            // 16 words at a time, every batch in flight at once; narrow strips (the common case) take one batch
+            auto batch = [&](int v0) {
+              unsigned long long w[16];
 #pragma unroll
-            for (int v = 0; v < 16; ++v) {
-              all = all && (w[v] >> 32) != 0ull;
-              m = fmaxf(m, __uint_as_float((uint32_t)w[v]));
-            }
+              for (int v = 0; v < 16; ++v)
+                w[v] = v0 + v < strip_units ? ptx::ld_relaxed_gpu_u64(slot + (size_t)(v0 + v) * kBM) : (1ull << 32);
+#pragma unroll
+              for (int v = 0; v < 16; ++v) {
+                all = all && (w[v] >> 32) != 0ull;
+                m = fmaxf(m, __uint_as_float((uint32_t)w[v]));
+              }
+            };
+            batch(0);
+            if (strip_units > 16) batch(16);
             if (all) {
               amax_row = m;
               break;
@@ -1232,7 +1239,9 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   off += 256;
   pl.ws_partial_off = off;      // (tag, row maximum) per strip row and 128-column unit
   const int strip_units = (N + unit_cols(out_mode) - 1) / unit_cols(out_mode);
-  pl.gather_words = strip_units <= 16 ? strip_units : 0;
+  // tagged words for strips of up to 16 units, and up to 32 when K is short enough for the exchange to show; with a
+  // long mainloop the units of a strip finish far apart and the one-flag-per-strip protocol polls far less
+  pl.gather_words = (strip_units <= 16 || (strip_units <= kMaxGatherWords && K <= 4096)) ? strip_units : 0;
   if (out_mode == QWT_OUT_INT8_PER_TOKEN) {
     if (pl.gather_words > 0) {
       off += (size_t)pl.tiles_m * kBM * pl.gather_words * sizeof(unsigned long long);
