@@ -106,3 +106,41 @@ def test_config5_calibration_sampled_channels(B, C, bits):
     expect = 1.0 / (1.0 + (8.0 / (2 ** bits - 1)) ** 2 / 12.0)
     assert np.abs(a.cpu().numpy() - expect).max() < 6.0 / np.sqrt(R) * (1.2 if bits == 4 else 0.1) + 1e-4
     assert np.abs(b.cpu().numpy() / sig).max() < 6.0 / np.sqrt(R)
+
+
+def test_config2_fused_calibration_sampled_channels(B):
+    """Calibration inside the layer at config 2's calibration size (512 images x 197 tokens, the qkv projection):
+    the oracle recomputes the quantized layer for sampled channels and fits them against the same fp_out."""
+    M, N, K = 512 * 197, 1152, 384
+    g = torch.Generator(device=DEV)
+    g.manual_seed(11)
+    Xq = torch.randint(-127, 128, (M, K), generator=g, device=DEV, dtype=torch.int8)
+    Wq = torch.randint(-127, 128, (N, K), generator=g, device=DEV, dtype=torch.int8)
+    xs = torch.rand(M, generator=g, device=DEV) * 0.04 + 0.01
+    ws = torch.rand(N, generator=g, device=DEV) * 2e-4 + 1e-4
+    bias = torch.randn(N, generator=g, device=DEV) * 0.5 + 1.0
+    # a synthetic "full-precision" output: a per-channel affine image of the integer product plus noise
+    # (built from float arithmetic of the inputs only, never from the library's own q)
+    gain = 1.0 + 0.05 * torch.randn(N, generator=g, device=DEV)
+    fp = torch.empty((M, N), dtype=torch.float32, device=DEV)
+    for r0 in range(0, M, 16384):
+        r1 = min(M, r0 + 16384)
+        acc = Xq[r0:r1].float() @ Wq.float().t()                       # exact: |acc| < 2^24
+        fp[r0:r1] = (acc * xs[r0:r1, None] * ws[None, :] + bias[None, :]) * gain[None, :]
+        fp[r0:r1] += 0.02 * torch.randn((r1 - r0, N), generator=g, device=DEV)
+    a = torch.empty(N, dtype=torch.float32, device=DEV)
+    b = torch.empty(N, dtype=torch.float32, device=DEV)
+    nd = torch.full((1,), -1, dtype=torch.int32, device=DEV)
+    wsb = B.qwt_qlinear_cwac_calibrate_workspace_bytes(M, N, K, B.QWT_W_INT8)
+    wsp = torch.empty(wsb, dtype=torch.uint8, device=DEV)
+    B.qwt_qlinear_cwac_calibrate(Xq, xs, Wq, B.QWT_W_INT8, ws, bias, fp, N, M, N, K, None, a, b, nd, wsp, wsb)
+    B.qwt_qlinear_check_status(wsp)
+    assert int(nd.item()) == 0
+    ch = np.unique(np.concatenate([np.random.default_rng(5).integers(0, N, 24), [0, 127, 128, 255, 256, N - 1]]))
+    ct = torch.from_numpy(ch).to(DEV)
+    q = O.dequant(O.int_matmul(Xq.cpu().numpy(), Wq[ct].cpu().numpy()), xs.cpu().numpy(), ws[ct].cpu().numpy(),
+                  bias[ct].cpu().numpy())
+    fph = fp[:, ct].cpu().numpy()
+    a_ref, b_ref, _ = O.cwac_fit(fph, q)
+    assert_ab_close(a[ct].cpu().numpy(), b[ct].cpu().numpy(), a_ref, b_ref, np.maximum(np.abs(fph.mean(0)), fph.std(0)))
+    assert np.abs(a_ref - gain[ct].cpu().numpy()).max() < 0.01       # the planted per-channel gain is what the fit finds
