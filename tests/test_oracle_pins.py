@@ -189,6 +189,19 @@ def test_fit_hand_cases():
         assert nd == 0
 
 
+def test_apply_hand_case_and_fit_residual():
+    """alpha (.) y + beta per channel: a worked case, and the least-squares property that ties it to the fit
+    (after compensation the residual has zero mean and is uncorrelated with q in every channel)."""
+    y = np.array([[1.0, 2.0], [3.0, 4.0]])
+    assert np.array_equal(O.cwac_apply(y, np.array([2.0, 0.5]), np.array([1.0, -1.0])), np.array([[3.0, 0.0], [7.0, 1.0]]))
+    rng = np.random.default_rng(12)
+    q = rng.standard_normal((500, 7)) + rng.uniform(-2, 2, 7)
+    f = q * rng.uniform(0.5, 1.5, 7) + 0.3 * rng.standard_normal((500, 7)) + rng.uniform(-1, 1, 7)
+    a, b, _ = O.cwac_fit(f, q)
+    res = f - O.cwac_apply(q, a, b)
+    assert np.abs(res.mean(0)).max() < 1e-12 and np.abs((res * q).mean(0)).max() < 1e-12
+
+
 def test_fit_planted_recovery_and_identity():
     rng = np.random.default_rng(8)
     q = rng.standard_normal((50, 7)) * 3 + 1
