@@ -182,7 +182,11 @@ qwt_status qwt_qlinear_check_status(const void* workspace, void* stream, int32_t
 /* Forward with HOST activations: X, x_scale are host inputs, Y, y_scale host outputs (pinned memory
  * recommended); W, fscale, fbias stay DEVICE resident (they are model parameters).  `staging` is device
  * scratch >= qwt_qlinear_host_staging_bytes(...).  The call copies in, runs the same kernel, copies out
- * and waits for the stream, so the outputs are valid on return. */
+ * and waits for the stream, so the outputs are valid on return.  More than 4096 rows are cut into row chunks
+ * (exact: a row's scale needs that row only) that alternate over two helper streams of the library, ordered after
+ * the work already queued on `stream`, so that the copy-in of a chunk, the kernel of the one before and the
+ * copy-out of the one before that overlap; the streams and events are created on the thread's first such call
+ * on a device and kept. */
 size_t qwt_qlinear_host_staging_bytes(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode);
 qwt_status qwt_qlinear_cwac_forward_host(const int8_t* X /*HOST*/, const float* x_scale /*HOST*/, const void* W,
                                          int32_t wfmt, const float* fscale, const float* fbias, int32_t M,

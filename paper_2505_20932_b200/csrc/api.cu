@@ -423,25 +423,56 @@ qwt_status qwt_qlinear_check_status(const void* workspace, void* stream, int32_t
 }
 
 namespace {
+// Rows of a chunk of the host-buffer forward: inputs of chunk c + 1 travel to the device while chunk c is computed
+// and the outputs of chunk c - 1 travel back (a row's per-token scale needs that row only, so row chunks are exact).
+constexpr int32_t kHostChunkRows = 4096;
+
 struct HostFwdLayout {
-  size_t off_x, off_xs, off_y, off_ys, off_ws, total;
-  size_t x_bytes, y_bytes;
+  size_t off_x, off_xs, off_y, off_ys, off_ws[2], ws_bytes, total;
+  size_t esz;
+  int32_t chunk_rows, chunks;
 };
 HostFwdLayout host_fwd_layout(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode) {
   HostFwdLayout L{};
   auto up = [](size_t x) { return (x + 255) / 256 * 256; };
-  const size_t esz = (out_mode == QWT_OUT_INT8_PER_TOKEN || out_mode == QWT_OUT_INT8_STATIC)
-                         ? 1 : (out_mode == QWT_OUT_BF16 ? 2 : 4);
-  L.x_bytes = (size_t)M * K;
-  L.y_bytes = (size_t)M * N * esz;
+  L.esz = (out_mode == QWT_OUT_INT8_PER_TOKEN || out_mode == QWT_OUT_INT8_STATIC)
+              ? 1 : (out_mode == QWT_OUT_BF16 ? 2 : 4);
+  L.chunk_rows = M > kHostChunkRows ? kHostChunkRows : M;
+  L.chunks = (M + L.chunk_rows - 1) / L.chunk_rows;
   size_t off = 0;
-  L.off_x = off; off += up(L.x_bytes);
+  L.off_x = off; off += up((size_t)M * K);
   L.off_xs = off; off += up((size_t)M * 4);
-  L.off_y = off; off += up(L.y_bytes);
+  L.off_y = off; off += up((size_t)M * N * L.esz);
   L.off_ys = off; off += up((size_t)M * 4);
-  L.off_ws = off; off += up(qwt_qlinear_workspace_bytes(M, N, K, wfmt, out_mode));
+  L.ws_bytes = up(qwt_qlinear_workspace_bytes(L.chunk_rows, N, K, wfmt, out_mode));
+  L.off_ws[0] = off; off += L.ws_bytes;
+  L.off_ws[1] = off; off += L.chunks > 1 ? L.ws_bytes : 0;
   L.total = off;
   return L;
+}
+
+// Two helper streams and three events per host thread and device, created on first use and kept.
+struct HostPipe {
+  cudaStream_t s[2];
+  cudaEvent_t start, done[2];
+  bool ready;
+};
+qwt_status host_pipe(HostPipe** out) {
+  static thread_local HostPipe pipes[64] = {};
+  int dev = 0;
+  QWT_CUDA_TRY(cudaGetDevice(&dev));
+  if (dev < 0 || dev >= 64) return QWT_ERR_ARCH;
+  HostPipe& hp = pipes[dev];
+  if (!hp.ready) {
+    for (int i = 0; i < 2; ++i) {
+      QWT_CUDA_TRY(cudaStreamCreateWithFlags(&hp.s[i], cudaStreamNonBlocking));
+      QWT_CUDA_TRY(cudaEventCreateWithFlags(&hp.done[i], cudaEventDisableTiming));
+    }
+    QWT_CUDA_TRY(cudaEventCreateWithFlags(&hp.start, cudaEventDisableTiming));
+    hp.ready = true;
+  }
+  *out = &hp;
+  return QWT_OK;
 }
 }  // namespace
 
@@ -463,19 +494,46 @@ qwt_status qwt_qlinear_cwac_forward_host(const int8_t* X, const float* x_scale, 
   uint8_t* base = static_cast<uint8_t*>(staging);
   int8_t* d_x = reinterpret_cast<int8_t*>(base + L.off_x);
   float* d_xs = reinterpret_cast<float*>(base + L.off_xs);
-  void* d_y = base + L.off_y;
+  uint8_t* d_y = base + L.off_y;
   float* d_ys = reinterpret_cast<float*>(base + L.off_ys);
-  QWT_CUDA_TRY(cudaMemcpyAsync(d_x, X, L.x_bytes, cudaMemcpyHostToDevice, st));
-  if (x_scale != nullptr) QWT_CUDA_TRY(cudaMemcpyAsync(d_xs, x_scale, (size_t)M * 4, cudaMemcpyHostToDevice, st));
-  s = qwt_qlinear_cwac_forward(d_x, x_scale ? d_xs : nullptr, W, wfmt, fscale, fbias, M, N, K, out_mode, d_y,
-                               out_mode == QWT_OUT_INT8_PER_TOKEN ? d_ys : nullptr, base + L.off_ws,
-                               L.total - L.off_ws, st);
-  if (s != QWT_OK) return s;
-  QWT_CUDA_TRY(cudaMemcpyAsync(Y, d_y, L.y_bytes, cudaMemcpyDeviceToHost, st));
-  if (out_mode == QWT_OUT_INT8_PER_TOKEN)
-    QWT_CUDA_TRY(cudaMemcpyAsync(y_scale, d_ys, (size_t)M * 4, cudaMemcpyDeviceToHost, st));
+  const bool per_token = out_mode == QWT_OUT_INT8_PER_TOKEN;
+  // one chunk of rows [r0, r0 + rows): copy in, compute, copy out, all on stream cs
+  auto chunk = [&](int32_t r0, int32_t rows, void* ws, cudaStream_t cs) -> qwt_status {
+    QWT_CUDA_TRY(cudaMemcpyAsync(d_x + (size_t)r0 * K, X + (size_t)r0 * K, (size_t)rows * K, cudaMemcpyHostToDevice, cs));
+    if (x_scale != nullptr)
+      QWT_CUDA_TRY(cudaMemcpyAsync(d_xs + r0, x_scale + r0, (size_t)rows * 4, cudaMemcpyHostToDevice, cs));
+    const size_t y_off = (size_t)r0 * N * L.esz;
+    qwt_status r = qwt_qlinear_cwac_forward(d_x + (size_t)r0 * K, x_scale ? d_xs + r0 : nullptr, W, wfmt, fscale, fbias,
+                                            rows, N, K, out_mode, d_y + y_off, per_token ? d_ys + r0 : nullptr, ws,
+                                            L.ws_bytes, cs);
+    if (r != QWT_OK) return r;
+    QWT_CUDA_TRY(cudaMemcpyAsync(static_cast<uint8_t*>(Y) + y_off, d_y + y_off, (size_t)rows * N * L.esz,
+                                 cudaMemcpyDeviceToHost, cs));
+    if (per_token) QWT_CUDA_TRY(cudaMemcpyAsync(y_scale + r0, d_ys + r0, (size_t)rows * 4, cudaMemcpyDeviceToHost, cs));
+    return QWT_OK;
+  };
+  if (L.chunks == 1) {
+    if ((s = chunk(0, M, base + L.off_ws[0], st)) != QWT_OK) return s;
+    QWT_CUDA_TRY(cudaStreamSynchronize(st));
+    return QWT_OK;
+  }
+  // several chunks: they alternate over two helper streams that start after the work already queued on `stream`
+  HostPipe* hp = nullptr;
+  if ((s = host_pipe(&hp)) != QWT_OK) return s;
+  QWT_CUDA_TRY(cudaEventRecord(hp->start, st));
+  for (int i = 0; i < 2; ++i) QWT_CUDA_TRY(cudaStreamWaitEvent(hp->s[i], hp->start, 0));
+  qwt_status rc = QWT_OK;
+  for (int32_t c = 0; c < L.chunks && rc == QWT_OK; ++c) {
+    const int32_t r0 = c * L.chunk_rows;
+    const int32_t rows = M - r0 < L.chunk_rows ? M - r0 : L.chunk_rows;
+    rc = chunk(r0, rows, base + L.off_ws[c & 1], hp->s[c & 1]);
+  }
+  for (int i = 0; i < 2; ++i) {
+    QWT_CUDA_TRY(cudaEventRecord(hp->done[i], hp->s[i]));
+    QWT_CUDA_TRY(cudaStreamWaitEvent(st, hp->done[i], 0));
+  }
   QWT_CUDA_TRY(cudaStreamSynchronize(st));
-  return QWT_OK;
+  return rc;
 }
 
 // ------------------------------------------------------------------------------------------------ support

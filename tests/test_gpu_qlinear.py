@@ -168,6 +168,33 @@ def test_forward_from_host_memory(H, B):
     assert_codes_close(Y, c_ref)
 
 
+@pytest.mark.parametrize("mode", ["int8", "bf16"])
+def test_forward_from_host_memory_in_row_chunks(H, B, mode):
+    """More than 4096 rows: the host-buffer call pipelines row chunks over two streams; same bits as one device call."""
+    import torch
+    M, N, K = 9001, 272, 144
+    Xq, Wq, xs, fs, fb = random_layer(M, N, K, seed=8)
+    out_mode = B.QWT_OUT_INT8_PER_TOKEN if mode == "int8" else B.QWT_OUT_BF16
+    dW, dfs, dfb = H.dev(Wq), H.dev(fs), H.dev(fb)
+    hx = torch.from_numpy(Xq).pin_memory()
+    hxs = torch.from_numpy(xs).pin_memory()
+    hy = torch.zeros((M, N), dtype=torch.int8 if mode == "int8" else torch.bfloat16).pin_memory()
+    hys = torch.zeros(M, dtype=torch.float32).pin_memory()
+    sb = B.qwt_qlinear_host_staging_bytes(M, N, K, B.QWT_W_INT8, out_mode)
+    st = H.empty_bytes(sb)
+    st.fill_(0xFF)
+    for _ in range(2):          # the second call reuses the helper streams
+        B.qwt_qlinear_cwac_forward_host(hx.data_ptr(), hxs.data_ptr(), dW, B.QWT_W_INT8, dfs, dfb, M, N, K, out_mode,
+                                        hy.data_ptr(), hys.data_ptr() if mode == "int8" else None, st, sb)
+    ref, ys_ref = H.gpu_forward(Xq, xs, Wq, fs, fb, out_mode)
+    if mode == "int8":
+        assert np.array_equal(hy.numpy(), ref) and np.array_equal(hys.numpy(), ys_ref)
+        c_ref, _ = O.requant_per_token(O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb))
+        assert_codes_close(hy.numpy(), c_ref)
+    else:
+        assert np.array_equal(hy.view(torch.int16).numpy().view(np.uint16), ref)
+
+
 # ------------------------------------------------------------------ packed 4-bit weights (W4A8)
 
 def random_w4_layer(M, N, K, seed):
