@@ -1,5 +1,6 @@
 // extern "C" entry points of libqwt2: argument validation on the host, then kernel launches.
 #include <cuda_runtime.h>
+#include <stdlib.h>
 #include <stdint.h>
 #include <string.h>
 
@@ -500,8 +501,6 @@ qwt_status qwt_qlinear_cwac_forward_host(const int8_t* X, const float* x_scale, 
   // one chunk of rows [r0, r0 + rows): copy in, compute, copy out, all on stream cs
   auto chunk = [&](int32_t r0, int32_t rows, void* ws, cudaStream_t cs) -> qwt_status {
     QWT_CUDA_TRY(cudaMemcpyAsync(d_x + (size_t)r0 * K, X + (size_t)r0 * K, (size_t)rows * K, cudaMemcpyHostToDevice, cs));
-    if (x_scale != nullptr)
-      QWT_CUDA_TRY(cudaMemcpyAsync(d_xs + r0, x_scale + r0, (size_t)rows * 4, cudaMemcpyHostToDevice, cs));
     const size_t y_off = (size_t)r0 * N * L.esz;
     qwt_status r = qwt_qlinear_cwac_forward(d_x + (size_t)r0 * K, x_scale ? d_xs + r0 : nullptr, W, wfmt, fscale, fbias,
                                             rows, N, K, out_mode, d_y + y_off, per_token ? d_ys + r0 : nullptr, ws,
@@ -509,11 +508,13 @@ qwt_status qwt_qlinear_cwac_forward_host(const int8_t* X, const float* x_scale, 
     if (r != QWT_OK) return r;
     QWT_CUDA_TRY(cudaMemcpyAsync(static_cast<uint8_t*>(Y) + y_off, d_y + y_off, (size_t)rows * N * L.esz,
                                  cudaMemcpyDeviceToHost, cs));
-    if (per_token) QWT_CUDA_TRY(cudaMemcpyAsync(y_scale + r0, d_ys + r0, (size_t)rows * 4, cudaMemcpyDeviceToHost, cs));
     return QWT_OK;
   };
+  // the per-row scales travel once, whole: in before the first chunk, out after the last
+  if (x_scale != nullptr) QWT_CUDA_TRY(cudaMemcpyAsync(d_xs, x_scale, (size_t)M * 4, cudaMemcpyHostToDevice, st));
   if (L.chunks == 1) {
     if ((s = chunk(0, M, base + L.off_ws[0], st)) != QWT_OK) return s;
+    if (per_token) QWT_CUDA_TRY(cudaMemcpyAsync(y_scale, d_ys, (size_t)M * 4, cudaMemcpyDeviceToHost, st));
     QWT_CUDA_TRY(cudaStreamSynchronize(st));
     return QWT_OK;
   }
@@ -532,6 +533,8 @@ qwt_status qwt_qlinear_cwac_forward_host(const int8_t* X, const float* x_scale, 
     QWT_CUDA_TRY(cudaEventRecord(hp->done[i], hp->s[i]));
     QWT_CUDA_TRY(cudaStreamWaitEvent(st, hp->done[i], 0));
   }
+  if (per_token && rc == QWT_OK)
+    QWT_CUDA_TRY(cudaMemcpyAsync(y_scale, d_ys, (size_t)M * 4, cudaMemcpyDeviceToHost, st));
   QWT_CUDA_TRY(cudaStreamSynchronize(st));
   return rc;
 }
