@@ -451,7 +451,11 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       }
     };
-    if (C::kNeedSlice && lead && g < n_units) prefetch_params(g);
+    int pre_n0 = -1;                        // lead warp: first column of the unit the prefetch registers hold
+    if (C::kNeedSlice && lead && g < n_units) {
+      prefetch_params(g);
+      pre_n0 = unit_col0(g);
+    }
 
     // Writes the warp's box (32 rows x BOXB bytes, swizzled in its staging slot) to global memory: lanes are
     // re-dealt so that one store instruction covers whole box rows (BOXB contiguous bytes each).
@@ -492,6 +496,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     };
 
     int use = 0;                            // units this group has handled
+    int slice_n0 = -1;                      // first column of the unit whose parameters are in the group's slice
+    int reloads = 0;                        // times the slice has been (re)loaded
     for (int u = g; u < n_units; u += kGroups, ++use) {
       const int j = u / UPT;
       const int tile = (int)blockIdx.x + j * G;
@@ -541,8 +547,14 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
       }
-      if (C::kNeedSlice) {
+      // The slice is reloaded only when the unit's columns differ from those of the group's previous unit: with a
+      // resident W tile every tile of the CTA has the same columns, and the group's slice is loaded once per call.
+      const bool reload = C::kNeedSlice && n0 != slice_n0;
+      if (reload) {
+        slice_n0 = n0;
+        const uint32_t ppar = (uint32_t)(reloads++) & 1u;
         if (lead) {
+          if (pre_n0 != n0) prefetch_params(u);      // not fetched ahead (never the case with a regular tile walk)
           // the slice is free once the group's 4 warps have finished the unit that used it before
           if (!ptx::mbar_wait_bounded(&gdone[g], upar ^ 1u, cta_abort, tmo)) {
             give_up(kStWaitParam);
@@ -561,9 +573,12 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&pfull[g]);
-          if (u + kGroups < n_units) prefetch_params(u + kGroups);
+          if (u + kGroups < n_units && unit_col0(u + kGroups) != n0) {
+            prefetch_params(u + kGroups);
+            pre_n0 = unit_col0(u + kGroups);
+          }
         }
-        if (!ptx::mbar_wait_bounded(&pfull[g], upar, cta_abort, tmo)) {
+        if (!ptx::mbar_wait_bounded(&pfull[g], ppar, cta_abort, tmo)) {
           give_up(kStWaitParam);
           break;
         }
