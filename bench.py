@@ -37,9 +37,9 @@ FALLBACK_HBM_GBS = 6650.0
 FALLBACK_BF16_TFLOPS = 1590.0
 INT8_OVER_BF16 = 2.0      # nominal dense ratio (4.5 POPS int8 : 2.25 PFLOPS bf16)
 
-# DRAM bytes per algorithmic byte of cwac_stats_kernel, from the ncu capture summarised in
-# profiles/cwac_stats_kernel_cfg5_small.md (None until a capture exists).
-STATS_TRAFFIC_RATIO = 1.01
+# DRAM bytes per algorithmic byte of the statistics pass (cwac_stats_batch_kernel; cwac_stats_kernel runs the same
+# block function), from the ncu capture summarised in profiles/cwac_stats_batch_kernel_cfg2_small.md.
+STATS_TRAFFIC_RATIO = 1.005
 # same for the forward kernel on the config-2 layers, profiles/qlinear_cwac_kernel_cfg2_int8.md
 QLINEAR_TRAFFIC_RATIO = 0.48    # the outputs stay in L2 for the length of the kernel (config-2 capture)
 
@@ -181,9 +181,25 @@ def build_layer(B, torch, WL, spec, seed, device, calib_rows=None):
     return L
 
 
-def phase_a(B, layers, stream, side=None):
-    """Calibrate + fold every layer.  The layers are independent, so with a second stream (`side`) they alternate
-    between the two: the small solve / fold kernels of one layer then run under the next layer's statistics pass."""
+class CalibBatch:
+    """All layers' calibration problems (with their folds) for the batched entry point, and its workspace."""
+
+    def __init__(self, B, layers, device):
+        import torch
+        self.probs = B.calib_problems((L.fp_out, L.q_out, L.R, L.spec.N, L.spec.N, L.a, L.b, L.ws, L.bias, L.fs, L.fb)
+                                      for L in layers)
+        self.wsb = B.qwt_cwac_calibrate_batch_workspace_bytes(self.probs)
+        self.ws = torch.empty(max(self.wsb, 256), dtype=torch.uint8, device=device)
+        self.groups = (len(layers) + 47) // 48        # launches of the statistics kernel per call
+
+
+def phase_a(B, layers, stream, side=None, batch=None):
+    """Calibrate + fold every layer: one batched call (statistics of all layers in one launch, reduce + solve + fold
+    in a second), or layer by layer.  Layer by layer the independent layers alternate over two streams when `side` is
+    given: the small solve / fold kernels of one layer then run under the next layer's statistics pass."""
+    if batch is not None:
+        B.qwt_cwac_calibrate_batch(batch.probs, None, batch.ws, batch.wsb, stream)
+        return
     if side is not None:
         side.wait_stream(stream)
     for i, L in enumerate(layers):
@@ -361,8 +377,9 @@ def run_ours(args):
             dist.barrier()
         torch.cuda.synchronize()
 
+    batch = None if args.calibration == "per-layer" else CalibBatch(B, layers, device)
     for _ in range(args.warmup):
-        phase_a(B, layers, stream)
+        phase_a(B, layers, stream, batch=batch)
         phase_b(B, layers, stream)
     for L in layers:
         if L.fws_bytes:
@@ -383,7 +400,7 @@ def run_ours(args):
         with torch.cuda.stream(cap):
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=cap):
-                phase_a(B, layers, cap, side)
+                phase_a(B, layers, cap, side, batch=batch)
             graphs.append(g)
             g = torch.cuda.CUDAGraph()
             with torch.cuda.graph(g, stream=cap):
@@ -402,7 +419,7 @@ def run_ours(args):
     for k in range(args.steps):
         ev[k][0].record(stream)
         if graphs is None:
-            phase_a(B, layers, stream)
+            phase_a(B, layers, stream, batch=batch)
         else:
             graphs[0].replay()
         ev[k][1].record(stream)
@@ -498,14 +515,16 @@ def run_ours(args):
     # ---- rooflines
     int8_peak = peaks["bf16_tflops"] * INT8_OVER_BF16
     int8_peak_sus = peaks["bf16_tflops_sustained"] * INT8_OVER_BF16
-    n_cal_launch = len(layers) * args.steps
+    n_cal_launch = (len(layers) if batch is None else batch.groups) * args.steps
+    cal_per_launch = cal_bytes * args.steps / n_cal_launch
     cal_ach = cal_bytes * args.steps / t_a / 1e9           # per GPU
-    roof_cal = {"kernel": "cwac_stats_kernel", "bound": "hbm", "achieved": cal_ach, "peak": peaks["hbm_gbs"],
+    roof_cal = {"kernel": "cwac_stats_kernel" if batch is None else "cwac_stats_batch_kernel", "bound": "hbm", "achieved": cal_ach, "peak": peaks["hbm_gbs"],
                 "unit": "GB/s", "frac": cal_ach / peaks["hbm_gbs"], "peak_source": f"of {peaks['source']}",
-                "traffic": (None if STATS_TRAFFIC_RATIO is None else STATS_TRAFFIC_RATIO * cal_bytes / len(layers)),
-                "algorithmic_bytes_per_launch": cal_bytes / len(layers), "launches": n_cal_launch,
+                "traffic": (None if STATS_TRAFFIC_RATIO is None else STATS_TRAFFIC_RATIO * cal_per_launch),
+                "algorithmic_bytes_per_launch": cal_per_launch, "launches": n_cal_launch,
                 "avg_launch_ms": t_a / n_cal_launch * 1e3,
-                "note": "duration = phase A (stats + reduce/solve + fold kernels of every layer) / launches"}
+                "note": ("duration = phase A (stats + reduce/solve + fold kernels of every layer) / launches" if batch is None
+                         else "duration = phase A (one statistics launch for all layers + one reduce/solve/fold launch) / launches")}
     fwd_tops_gpu = fwd_ops * args.steps / t_b / 1e12
     t_min_compute = fwd_ops / (int8_peak * 1e12)
     t_min_hbm = fwd_bytes / (peaks["hbm_gbs"] * 1e9)
@@ -631,6 +650,9 @@ def main():
     ap.add_argument("--out", default="", choices=["", "int8", "bf16"], help="override the output stage")
     ap.add_argument("--seed", type=int, default=0)
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--calibration", default="batch", choices=["batch", "per-layer"],
+                    help="phase A through the batched entry point (one statistics launch for all layers) or one "
+                         "calibrate + fold call per layer")
     ap.add_argument("--forward-streams", type=int, default=2, choices=[1, 2, 3, 4],
                     help="streams the forward calls of phase B alternate over inside the graph")
     ap.add_argument("--no-library-int8", action="store_true", help="skip timing the library int8 matmul reference point")

@@ -98,6 +98,32 @@ qwt_status qwt_cwac_calibrate_host(const float* fp_out /*HOST*/, const float* q_
                                    int32_t* n_degenerate /*HOST, may be NULL*/,
                                    void* staging, size_t staging_bytes, void* stream);
 
+/* Calibration of several layers in one call (the layers of a model on one calibration set): one statistics launch
+ * and one reduce / solve launch for all of them, instead of two (three with the fold) per layer.  Every problem is
+ * cut and summed exactly as its own qwt_cwac_calibrate call would cut and sum it, so the results are bit for bit
+ * the same; what goes away is a launch, a ramp and a tail per layer.
+ *   problems : HOST array of `count` descriptors (read during the call only); the pointers inside are DEVICE
+ *              pointers with the meaning and alignment of qwt_cwac_calibrate / qwt_cwac_fold.  w_scale != NULL
+ *              asks for the fold of that layer as well: fscale = a * w_scale, fbias = a * bias + b (bias may be NULL).
+ *   n_degenerate : DEVICE int32, total over all problems, may be NULL
+ *   workspace    : device, 256-byte aligned, >= qwt_cwac_calibrate_batch_workspace_bytes(problems, count) */
+typedef struct qwt_calib_problem {
+  const float* fp_out;
+  const float* q_out;
+  int64_t rows;
+  int64_t ld;
+  int32_t channels;
+  float* a;
+  float* b;
+  const float* w_scale;
+  const float* bias;
+  float* fscale;
+  float* fbias;
+} qwt_calib_problem;
+size_t qwt_cwac_calibrate_batch_workspace_bytes(const qwt_calib_problem* problems /*HOST*/, int32_t count);
+qwt_status qwt_cwac_calibrate_batch(const qwt_calib_problem* problems /*HOST*/, int32_t count,
+                                    int32_t* n_degenerate, void* workspace, size_t workspace_bytes, void* stream);
+
 /* Calibration without any workspace argument (the paper has no counterpart: this is a packaging variant of
  * qwt_cwac_calibrate, same kernels, same results within the library's calibration tolerance).
  * For callers that cannot allocate device memory -- e.g. a plug-in confined to a host program's fixed

@@ -38,6 +38,8 @@ SIGNATURES = {
     "qwt_cwac_solve": (_i32, [_p, _i32, _p, _p, _p, _p]),
     "qwt_cwac_host_staging_bytes": (_sz, [_i64, _i32]),
     "qwt_cwac_calibrate_host": (_i32, [_p, _p, _i64, _i32, _i64, _p, _p, _p, _p, _sz, _p]),
+    "qwt_cwac_calibrate_batch_workspace_bytes": (_sz, [_p, _i32]),
+    "qwt_cwac_calibrate_batch": (_i32, [_p, _i32, _p, _p, _sz, _p]),
     "qwt_cwac_calibrate_noalloc": (_i32, [_p, _p, _i64, _i32, _i64, _p, _p, _p, _p]),
     "qwt_cwac_fold": (_i32, [_p, _p, _p, _p, _i32, _p, _p, _p]),
     "qwt_cwac_fold_static": (_i32, [_p, _p, _p, _p, _i32, C.c_float, C.c_float, _p, _p, _p]),
@@ -166,6 +168,36 @@ def qwt_cwac_calibrate_host(fp_out, q_out, rows, channels, ld, a, b, n_degenerat
                                     _ptr(n_degenerate), _ptr(staging), staging_bytes, _stream(stream))
     if check:
         _check(s, "qwt_cwac_calibrate_host")
+    return s
+
+
+class CalibProblem(C.Structure):
+    """Mirror of qwt_calib_problem."""
+    _fields_ = [("fp_out", _p), ("q_out", _p), ("rows", _i64), ("ld", _i64), ("channels", _i32), ("a", _p), ("b", _p),
+                ("w_scale", _p), ("bias", _p), ("fscale", _p), ("fbias", _p)]
+
+
+def calib_problems(items):
+    """items: iterable of (fp_out, q_out, rows, channels, ld, a, b[, w_scale, bias, fscale, fbias]) -> ctypes array."""
+    items = list(items)
+    arr = (CalibProblem * len(items))()
+    for dst, it in zip(arr, items):
+        it = tuple(it) + (None,) * (11 - len(it))
+        fp, q, rows, ch, ld, a, b, ws, bias, fs, fb = it
+        dst.fp_out, dst.q_out, dst.rows, dst.ld, dst.channels = _ptr(fp), _ptr(q), rows, ld, ch
+        dst.a, dst.b, dst.w_scale, dst.bias, dst.fscale, dst.fbias = _ptr(a), _ptr(b), _ptr(ws), _ptr(bias), _ptr(fs), _ptr(fb)
+    return arr
+
+
+def qwt_cwac_calibrate_batch_workspace_bytes(problems) -> int:
+    return int(lib.qwt_cwac_calibrate_batch_workspace_bytes(C.cast(problems, _p), len(problems)))
+
+
+def qwt_cwac_calibrate_batch(problems, n_degenerate, workspace, workspace_bytes, stream=None, check=True) -> int:
+    s = lib.qwt_cwac_calibrate_batch(C.cast(problems, _p), len(problems), _ptr(n_degenerate), _ptr(workspace),
+                                     workspace_bytes, _stream(stream))
+    if check:
+        _check(s, "qwt_cwac_calibrate_batch")
     return s
 
 

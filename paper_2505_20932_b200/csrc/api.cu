@@ -107,6 +107,37 @@ qwt_status qwt_cwac_calibrate(const float* fp_out, const float* q_out, int64_t r
   return launch_cwac_reduce(workspace, plan, channels, rows, nullptr, a, b, n_degenerate, as_stream(stream));
 }
 
+static_assert(sizeof(qwt_calib_problem) == sizeof(CalibBatchItem), "the ABI struct and the internal one are the same");
+
+static qwt_status check_batch(const qwt_calib_problem* p, int32_t count) {
+  if (p == nullptr) return QWT_ERR_NULL;
+  if (count < 1 || count > 4096) return QWT_ERR_SHAPE;
+  for (int32_t i = 0; i < count; ++i) {
+    qwt_status s = check_calib_args(p[i].fp_out, p[i].q_out, p[i].rows, p[i].channels, p[i].ld);
+    if (s != QWT_OK) return s;
+    if (p[i].a == nullptr || p[i].b == nullptr) return QWT_ERR_NULL;
+    if (p[i].w_scale != nullptr && (p[i].fscale == nullptr || p[i].fbias == nullptr)) return QWT_ERR_NULL;
+  }
+  return QWT_OK;
+}
+
+size_t qwt_cwac_calibrate_batch_workspace_bytes(const qwt_calib_problem* problems, int32_t count) {
+  if (check_batch(problems, count) != QWT_OK) return 0;
+  return cwac_batch_workspace_bytes(reinterpret_cast<const CalibBatchItem*>(problems), count);
+}
+
+qwt_status qwt_cwac_calibrate_batch(const qwt_calib_problem* problems, int32_t count, int32_t* n_degenerate,
+                                    void* workspace, size_t workspace_bytes, void* stream) {
+  qwt_status s = check_batch(problems, count);
+  if (s != QWT_OK) return s;
+  if (workspace == nullptr) return QWT_ERR_NULL;
+  const CalibBatchItem* items = reinterpret_cast<const CalibBatchItem*>(problems);
+  if (workspace_bytes < cwac_batch_workspace_bytes(items, count) || !aligned(workspace, 256)) return QWT_ERR_WORKSPACE;
+  DeviceInfo dev;
+  if ((s = current_device(&dev)) != QWT_OK) return s;
+  return launch_cwac_calibrate_batch(items, count, n_degenerate, workspace, as_stream(stream));
+}
+
 qwt_status qwt_cwac_stats_accumulate(const float* fp_out, const float* q_out, int64_t rows, int32_t channels,
                                      int64_t ld, double* stats, void* workspace, size_t workspace_bytes,
                                      void* stream) {

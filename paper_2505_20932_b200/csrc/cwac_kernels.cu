@@ -21,6 +21,38 @@ namespace qwt {
 // the shifted sums are turned back into raw sums in FP64 and written as one partial per (chunk, sum,
 // channel).  No atomics: a second kernel adds the partials in chunk order, so results are reproducible.
 // ------------------------------------------------------------------------------------------------
+// Descriptors of a batched launch (passed by value as kernel parameters).
+constexpr int kMaxBatch = 48;        // 48 descriptors of 80 bytes + the block offsets stay below the 4 KB of kernel parameters
+struct StatsProblem {
+  const float* fp_out;
+  const float* q_out;
+  double* partial;
+  int64_t rows, ld, chunk_rows;
+  int channels, cpad, slabs, pad_;
+};
+struct StatsBatch {
+  int count;
+  int block0[kMaxBatch + 1];
+  StatsProblem prob[kMaxBatch];
+};
+struct ReduceProblem {
+  const double* partial;
+  float* a;
+  float* b;
+  const float* w_scale;
+  const float* bias;
+  float* fscale;
+  float* fbias;
+  double n_rows;
+  int chunks, cpad, channels, pad_;
+};
+struct ReduceBatch {
+  int count;
+  int block0[kMaxBatch + 1];
+  ReduceProblem prob[kMaxBatch];
+};
+static_assert(sizeof(ReduceBatch) + sizeof(int*) <= 4096 && sizeof(StatsBatch) <= 4096, "kernel parameter space");
+
 constexpr int kStatsTX = 32;
 constexpr int kStatsTY = 8;
 constexpr int kStatsThreads = kStatsTX * kStatsTY;
@@ -32,13 +64,14 @@ __device__ __forceinline__ float4 ld_stream(const float* p) {
   return __ldcs(reinterpret_cast<const float4*>(p));
 }
 
-__global__ void __launch_bounds__(kStatsThreads)
-cwac_stats_kernel(const float* __restrict__ fp_out, const float* __restrict__ q_out, int64_t rows, int channels,
-                  int64_t ld, int64_t chunk_rows, double* __restrict__ partial, int cpad) {
+// One block's work: column slab `slab`, row chunk `chunk` of one (fp_out, q_out) pair.
+__device__ __forceinline__ void cwac_stats_block(const float* __restrict__ fp_out, const float* __restrict__ q_out,
+                                                 int64_t rows, int channels, int64_t ld, int64_t chunk_rows,
+                                                 double* __restrict__ partial, int cpad, int slab, int chunk) {
   const int tx = threadIdx.x & (kStatsTX - 1);
   const int ty = threadIdx.x / kStatsTX;
-  const int c0 = blockIdx.x * kSlabChannels + tx * 4;
-  const int64_t r0 = (int64_t)blockIdx.y * chunk_rows;
+  const int c0 = slab * kSlabChannels + tx * 4;
+  const int64_t r0 = (int64_t)chunk * chunk_rows;
   const int64_t r1 = (r0 + chunk_rows < rows) ? r0 + chunk_rows : rows;
   // c0 + 3 may pass `channels`, but ld % 4 == 0 and ld >= channels keep the 16-byte load inside the row
   const bool active = c0 < channels;
@@ -112,7 +145,7 @@ cwac_stats_kernel(const float* __restrict__ fp_out, const float* __restrict__ q_
   if (threadIdx.x < kSlabChannels) {
     const int ch = threadIdx.x;           // channel inside the slab
     const int ltx = ch >> 2, j = ch & 3;
-    const int c = blockIdx.x * kSlabChannels + ch;
+    const int c = slab * kSlabChannels + ch;
     double sd[4];
 #pragma unroll
     for (int s = 0; s < 4; ++s) {
@@ -128,12 +161,32 @@ cwac_stats_kernel(const float* __restrict__ fp_out, const float* __restrict__ q_
     const double Sf = sd[1] + nb * Kf;
     const double Sqf = sd[2] + Kf * sd[0] + Kq * sd[1] + nb * Kq * Kf;
     const double Sqq = sd[3] + 2.0 * Kq * sd[0] + nb * Kq * Kq;
-    double* out = partial + (size_t)blockIdx.y * 4 * cpad + c;
+    double* out = partial + (size_t)chunk * 4 * cpad + c;
     out[0 * (size_t)cpad] = Sq;
     out[1 * (size_t)cpad] = Sf;
     out[2 * (size_t)cpad] = Sqf;
     out[3 * (size_t)cpad] = Sqq;
   }
+}
+
+// (two blocks per SM: 256 threads x 128 registers each is the whole register file)
+__global__ void __launch_bounds__(kStatsThreads, 2)
+cwac_stats_kernel(const float* __restrict__ fp_out, const float* __restrict__ q_out, int64_t rows, int channels,
+                  int64_t ld, int64_t chunk_rows, double* __restrict__ partial, int cpad) {
+  cwac_stats_block(fp_out, q_out, rows, channels, ld, chunk_rows, partial, cpad, (int)blockIdx.x, (int)blockIdx.y);
+}
+
+// Several pairs in one launch (the layers of a model): block b belongs to the problem p with
+// block0[p] <= b < block0[p + 1] and does exactly what block (slab, chunk) of that problem's own launch would do,
+// so the results are bit for bit those of the single calls; what goes away is one launch, ramp and tail per layer.
+__global__ void __launch_bounds__(kStatsThreads, 2)
+cwac_stats_batch_kernel(const __grid_constant__ StatsBatch sb) {
+  int p = 0;
+  while (p + 1 < sb.count && (int)blockIdx.x >= sb.block0[p + 1]) ++p;
+  const StatsProblem pr = sb.prob[p];
+  const int local = (int)blockIdx.x - sb.block0[p];
+  cwac_stats_block(pr.fp_out, pr.q_out, pr.rows, pr.channels, pr.ld, pr.chunk_rows, pr.partial, pr.cpad,
+                   local % pr.slabs, local / pr.slabs);
 }
 
 // Closed form of Eq. 4-5 from the five sums of one channel.
@@ -160,13 +213,15 @@ __device__ __forceinline__ void cwac_solve_channel(double n, double Sq, double S
 // stats_io (may be NULL): running statistics to update.  a, b (may be NULL): solve after the reduction.
 constexpr int kRedTX = 32;
 constexpr int kRedTY = 32;
-__global__ void __launch_bounds__(kRedTX * kRedTY)
-cwac_reduce_kernel(const double* __restrict__ partial, int chunks, int cpad, int channels, double n_rows,
-                   double* __restrict__ stats_io, float* __restrict__ a, float* __restrict__ b,
-                   int* __restrict__ n_degenerate) {
+__device__ __forceinline__ void cwac_reduce_block(const double* __restrict__ partial, int chunks, int cpad,
+                                                  int channels, double n_rows, double* __restrict__ stats_io,
+                                                  float* __restrict__ a, float* __restrict__ b,
+                                                  int* __restrict__ n_degenerate, int block,
+                                                  const float* __restrict__ w_scale, const float* __restrict__ bias,
+                                                  float* __restrict__ fscale, float* __restrict__ fbias) {
   const int tx = threadIdx.x & (kRedTX - 1);
   const int ty = threadIdx.x / kRedTX;
-  const int c = blockIdx.x * kRedTX + tx;       // < cpad by construction of the grid
+  const int c = block * kRedTX + tx;            // < cpad by construction of the grid
   double s[4] = {0.0, 0.0, 0.0, 0.0};
   if (c < channels) {
     for (int k = ty; k < chunks; k += kRedTY) {
@@ -200,7 +255,31 @@ cwac_reduce_kernel(const double* __restrict__ partial, int chunks, int cpad, int
     int deg;
     cwac_solve_channel(n, s[0], s[1], s[2], s[3], &a[c], &b[c], &deg);
     if (deg && n_degenerate != nullptr) atomicAdd(n_degenerate, 1);
+    if (w_scale != nullptr) {     // Eq. 11 at once, the arithmetic of cwac_fold_kernel
+      const float ai = a[c], bi = b[c];
+      const float bs = bias ? bias[c] : 0.0f;
+      fscale[c] = ai * w_scale[c];
+      fbias[c] = fmaf(ai, bs, bi);
+    }
   }
+}
+
+__global__ void __launch_bounds__(kRedTX * kRedTY)
+cwac_reduce_kernel(const double* __restrict__ partial, int chunks, int cpad, int channels, double n_rows,
+                   double* __restrict__ stats_io, float* __restrict__ a, float* __restrict__ b,
+                   int* __restrict__ n_degenerate) {
+  cwac_reduce_block(partial, chunks, cpad, channels, n_rows, stats_io, a, b, n_degenerate, (int)blockIdx.x, nullptr,
+                    nullptr, nullptr, nullptr);
+}
+
+__global__ void __launch_bounds__(kRedTX * kRedTY)
+cwac_reduce_batch_kernel(const __grid_constant__ ReduceBatch rb, int* __restrict__ n_degenerate) {
+  int p = 0;
+#pragma unroll 1
+  while (p + 1 < rb.count && (int)blockIdx.x >= rb.block0[p + 1]) ++p;
+  const ReduceProblem pr = rb.prob[p];
+  cwac_reduce_block(pr.partial, pr.chunks, pr.cpad, pr.channels, pr.n_rows, nullptr, pr.a, pr.b, n_degenerate,
+                    (int)blockIdx.x - rb.block0[p], pr.w_scale, pr.bias, pr.fscale, pr.fbias);
 }
 
 __global__ void __launch_bounds__(128)
@@ -429,6 +508,50 @@ qwt_status launch_cwac_reduce(const void* workspace, const CwacPlan& plan, int32
                                                              plan.cpad, channels, (double)rows, stats_io, a, b,
                                                              n_degenerate);
   QWT_LAUNCH_CHECK();
+  return QWT_OK;
+}
+
+size_t cwac_batch_workspace_bytes(const CalibBatchItem* items, int32_t count) {
+  size_t total = 0;
+  for (int32_t i = 0; i < count; ++i)
+    total += (cwac_plan(items[i].rows, items[i].channels, 148).partial_bytes + 255) / 256 * 256;
+  return total;
+}
+
+// Statistics of all problems in one launch, reduction + solve (+ fold) of all problems in a second one; more than
+// kMaxBatch problems go in groups.
+qwt_status launch_cwac_calibrate_batch(const CalibBatchItem* items, int32_t count, int32_t* n_degenerate,
+                                       void* workspace, cudaStream_t st) {
+  if (n_degenerate != nullptr) QWT_CUDA_TRY(cudaMemsetAsync(n_degenerate, 0, sizeof(int32_t), st));
+  uint8_t* ws = static_cast<uint8_t*>(workspace);
+  size_t off = 0;
+  for (int32_t g0 = 0; g0 < count; g0 += kMaxBatch) {
+    const int n = count - g0 < kMaxBatch ? count - g0 : kMaxBatch;
+    StatsBatch sb{};
+    ReduceBatch rb{};
+    sb.count = rb.count = n;
+    int sblocks = 0, rblocks = 0;
+    for (int i = 0; i < n; ++i) {
+      const CalibBatchItem& it = items[g0 + i];
+      const CwacPlan plan = cwac_plan(it.rows, it.channels, 148);
+      double* partial = reinterpret_cast<double*>(ws + off);
+      off += (plan.partial_bytes + 255) / 256 * 256;
+      sb.block0[i] = sblocks;
+      sb.prob[i] = StatsProblem{it.fp_out, it.q_out, partial, it.rows, it.ld, plan.chunk_rows, it.channels, plan.cpad,
+                                plan.slabs, 0};
+      sblocks += plan.slabs * plan.chunks;
+      rb.block0[i] = rblocks;
+      rb.prob[i] = ReduceProblem{partial, it.a, it.b, it.w_scale, it.bias, it.fscale, it.fbias, (double)it.rows,
+                                 plan.chunks, plan.cpad, it.channels, 0};
+      rblocks += (it.channels + kRedTX - 1) / kRedTX;
+    }
+    sb.block0[n] = sblocks;
+    rb.block0[n] = rblocks;
+    cwac_stats_batch_kernel<<<sblocks, kStatsThreads, 0, st>>>(sb);
+    QWT_LAUNCH_CHECK();
+    cwac_reduce_batch_kernel<<<rblocks, kRedTX * kRedTY, 0, st>>>(rb, n_degenerate);
+    QWT_LAUNCH_CHECK();
+  }
   return QWT_OK;
 }
 

@@ -55,6 +55,21 @@ struct CwacPlan {
 CwacPlan cwac_plan(int64_t rows, int32_t channels, int sm_count);
 qwt_status launch_cwac_stats(const float* fp_out, const float* q_out, int64_t rows, int32_t channels, int64_t ld,
                              double* stats, void* workspace, const CwacPlan& plan, cudaStream_t st);
+struct CalibBatchItem {
+  const float* fp_out;
+  const float* q_out;
+  int64_t rows, ld;
+  int32_t channels;
+  float* a;
+  float* b;
+  const float* w_scale;   // non-NULL: fold as well (Eq. 11) into fscale / fbias
+  const float* bias;
+  float* fscale;
+  float* fbias;
+};
+size_t cwac_batch_workspace_bytes(const CalibBatchItem* items, int32_t count);
+qwt_status launch_cwac_calibrate_batch(const CalibBatchItem* items, int32_t count, int32_t* n_degenerate,
+                                       void* workspace, cudaStream_t st);
 qwt_status launch_cwac_solve(const double* stats, int32_t channels, float* a, float* b, int32_t* n_degenerate,
                              cudaStream_t st);
 qwt_status launch_cwac_fold(const float* w_scale, const float* bias, const float* a, const float* b, int32_t n,

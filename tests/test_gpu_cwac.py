@@ -139,3 +139,42 @@ def test_pack_int4_bit_exact(H):
     rng = np.random.default_rng(8)
     c = rng.integers(-7, 8, (37, 64)).astype(np.int8)
     assert np.array_equal(H.gpu_pack_int4(c), O.pack_int4(c))
+
+
+def test_batched_calibration_is_the_single_calls_bit_for_bit(H):
+    """Several layers in one call: same partition, same order, hence the same bits as one call per layer, with the
+    fold of Eq. 11 done on the way when asked for; more problems than one launch takes go in groups."""
+    import torch
+    from paper_2505_20932_b200 import binding as B
+    rng = np.random.default_rng(3)
+    shapes = [(6304, 384, 384), (1000, 768, 768), (129, 132, 136), (1, 4, 4), (3000, 1152, 1152)] * 9   # 45 problems
+    items, keep, single = [], [], []
+    for i, (rows, C, ld) in enumerate(shapes):
+        fp, q, _ = WL.host_calib_pair(rows, ld, 4 if i % 2 else 8, seed=100 + i)
+        dfp, dq = H.dev(fp), H.dev(q)
+        a, b = (torch.full((C,), 7.0, device=H.DEV) for _ in range(2))
+        fold = i % 3 != 0
+        ws_, bias = (H.dev(rng.uniform(1e-3, 2e-3, C).astype(np.float32)), H.dev(rng.standard_normal(C).astype(np.float32))) if fold else (None, None)
+        fs, fb = (torch.zeros(C, device=H.DEV), torch.zeros(C, device=H.DEV)) if fold else (None, None)
+        items.append((dfp, dq, rows, C, ld, a, b, ws_, bias if i % 2 else None, fs, fb))
+        keep.append((fp, q, C, a, b, ws_, bias if i % 2 else None, fs, fb))
+    probs = B.calib_problems(items)
+    wsb = B.qwt_cwac_calibrate_batch_workspace_bytes(probs)
+    ws = H.empty_bytes(wsb)
+    ws.fill_(0xFF)
+    nd = torch.full((1,), -1, dtype=torch.int32, device=H.DEV)
+    B.qwt_cwac_calibrate_batch(probs, nd, ws, wsb)
+    torch.cuda.synchronize()
+    nd_total = 0
+    for fp, q, C, a, b, ws_, bias, fs, fb in keep:
+        a1, b1, nd1 = H.gpu_calibrate(fp, q, channels=C)
+        nd_total += nd1
+        assert np.array_equal(a.cpu().numpy(), a1) and np.array_equal(b.cpu().numpy(), b1)
+        if ws_ is not None:
+            gfs, gfb = H.gpu_fold(ws_.cpu().numpy(), None if bias is None else bias.cpu().numpy(), a1, b1)
+            assert np.array_equal(fs.cpu().numpy(), gfs) and np.array_equal(fb.cpu().numpy(), gfb)
+    assert int(nd.item()) == nd_total
+    # and against the oracle, one of them
+    fp, q, C, a, b = keep[4][:5]
+    a_ref, b_ref, _ = O.cwac_fit(fp[:, :C], q[:, :C])
+    assert_ab_close(a.cpu().numpy(), b.cpu().numpy(), a_ref, b_ref, nat_scale(fp[:, :C]))
