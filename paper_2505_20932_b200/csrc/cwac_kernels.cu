@@ -322,7 +322,10 @@ cwac_fold_static_kernel(const float* __restrict__ w_scale, const float* __restri
   offset[i] = (int32_t)fmin(fmax(off, -2147483647.0), 2147483647.0);
 }
 
-// Eq. 1-2 with zero-point 0: one warp per row, two passes over the row (the second hits cache).
+// Eq. 1-2 with zero-point 0: one warp per row, two passes over the row (the second hits cache).  VEC: 16-byte
+// loads and 4-byte stores (cols and ld multiples of 4, 16-byte aligned X, 4-byte aligned Xq); same arithmetic
+// per element either way.
+template <bool VEC>
 __global__ void __launch_bounds__(256)
 quantize_rows_kernel(const float* __restrict__ X, int64_t rows, int cols, int64_t ld, float qmax,
                      int8_t* __restrict__ Xq, float* __restrict__ scale) {
@@ -331,18 +334,39 @@ quantize_rows_kernel(const float* __restrict__ X, int64_t rows, int cols, int64_
   if (r >= rows) return;
   const float* x = X + r * ld;
   float m = 0.f;
-  for (int c = lane; c < cols; c += 32) m = fmaxf(m, fabsf(x[c]));
+  if (VEC) {
+    const float4* x4 = reinterpret_cast<const float4*>(x);
+    for (int c = lane; c < cols / 4; c += 32) {
+      const float4 v = x4[c];
+      m = fmaxf(fmaxf(m, fmaxf(fabsf(v.x), fabsf(v.y))), fmaxf(fabsf(v.z), fabsf(v.w)));
+    }
+  } else {
+    for (int c = lane; c < cols; c += 32) m = fmaxf(m, fabsf(x[c]));
+  }
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
   const float s = __fdiv_rn(m, qmax);
   if (lane == 0) scale[r] = s;
   int8_t* q = Xq + r * (int64_t)cols;
-  if (s > 0.f) {
-    for (int c = lane; c < cols; c += 32) {
-      float v = rintf(__fdiv_rn(x[c], s));
-      v = fminf(fmaxf(v, -qmax), qmax);
-      q[c] = (int8_t)(int)v;
+  auto code = [&](float xv) -> int {
+    float v = rintf(__fdiv_rn(xv, s));
+    v = fminf(fmaxf(v, -qmax), qmax);
+    return (int)v;
+  };
+  if (VEC) {
+    const float4* x4 = reinterpret_cast<const float4*>(x);
+    uint32_t* q4 = reinterpret_cast<uint32_t*>(q);
+    for (int c = lane; c < cols / 4; c += 32) {
+      uint32_t w = 0u;
+      if (s > 0.f) {
+        const float4 v = x4[c];
+        w = (uint32_t)(code(v.x) & 0xff) | ((uint32_t)(code(v.y) & 0xff) << 8) | ((uint32_t)(code(v.z) & 0xff) << 16) |
+            ((uint32_t)(code(v.w) & 0xff) << 24);
+      }
+      q4[c] = w;
     }
+  } else if (s > 0.f) {
+    for (int c = lane; c < cols; c += 32) q[c] = (int8_t)code(x[c]);
   } else {
     for (int c = lane; c < cols; c += 32) q[c] = 0;
   }
@@ -582,7 +606,9 @@ qwt_status launch_quantize_rows(const float* X, int64_t rows, int32_t cols, int6
                                 float* scale, cudaStream_t st) {
   const int rows_per_block = 8;
   const int64_t blocks = (rows + rows_per_block - 1) / rows_per_block;
-  quantize_rows_kernel<<<(unsigned)blocks, rows_per_block * 32, 0, st>>>(X, rows, cols, ld, (float)qmax, Xq, scale);
+  const bool vec = (cols % 4) == 0 && (ld % 4) == 0 && aligned(X, 16) && aligned(Xq, 4);
+  if (vec) quantize_rows_kernel<true><<<(unsigned)blocks, rows_per_block * 32, 0, st>>>(X, rows, cols, ld, (float)qmax, Xq, scale);
+  else quantize_rows_kernel<false><<<(unsigned)blocks, rows_per_block * 32, 0, st>>>(X, rows, cols, ld, (float)qmax, Xq, scale);
   QWT_LAUNCH_CHECK();
   return QWT_OK;
 }

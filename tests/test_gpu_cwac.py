@@ -124,7 +124,8 @@ def test_fold_matches_oracle(H):
         assert np.allclose(fb, fb_ref, rtol=1e-6, atol=1e-9)
 
 
-@pytest.mark.parametrize("rows,cols,qmax", [(788, 384, 127), (1536, 384, 127), (64, 768, 7), (3, 16, 127), (33, 1000, 7)])
+@pytest.mark.parametrize("rows,cols,qmax", [(788, 384, 127), (1536, 384, 127), (64, 768, 7), (3, 16, 127), (33, 1000, 7),
+                                            (5, 18, 127), (33, 1001, 7)])      # the last two: no 16-byte row pieces
 def test_row_quantizer_bit_exact(H, rows, cols, qmax):
     X = WL.host_activations("sparse_outlier", rows, cols, seed=rows, tag="q")
     if rows > 2:
