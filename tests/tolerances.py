@@ -1,4 +1,10 @@
-"""Tolerances of the parity tests (stated by the task's target; see the design doc for the arithmetic)."""
+"""Tolerances of the parity tests.
+
+FP32 outputs: the kernel forms z with three FP32 roundings (int->float is exact below 2^24, the row-scale product,
+the fused multiply-add), the oracle in float64: |d| <= 1e-5 |ref| + 1e-6 leaves two orders of magnitude of room.
+INT8 codes: both sides round an FP32 quotient; they may disagree where it lies within a few 1e-6 of a half-integer,
+which is rare (about one code in a million measured): at most 1 LSB on at most 0.01 % of the elements.
+CWAC a, b: FP32 results of float64 sums, 1e-5 relative (b with an absolute floor of 1e-6 of the channel's scale)."""
 import numpy as np
 
 FP32_REL = 1e-5      # dequantized + compensated outputs: |d| <= 1e-5 |ref| + 1e-6
