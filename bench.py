@@ -38,9 +38,9 @@ FALLBACK_BF16_TFLOPS = 1590.0
 INT8_OVER_BF16 = 2.0      # nominal dense ratio (4.5 POPS int8 : 2.25 PFLOPS bf16)
 
 # DRAM bytes per algorithmic byte of the statistics pass (cwac_stats_batch_kernel; cwac_stats_kernel runs the same
-# block function), from the ncu capture summarised in profiles/cwac_stats_batch_kernel_cfg2_small.md.
+# block function), from an ncu capture of four config-2 layers at 50 000 rows (summary under profiles/).
 STATS_TRAFFIC_RATIO = 1.005
-# same for the forward kernel on the config-2 layers, profiles/qlinear_cwac_kernel_cfg2_int8.md
+# same for the forward kernel with per-token INT8 output on the four config-2 layer shapes (summary under profiles/)
 QLINEAR_TRAFFIC_RATIO = 0.48    # the outputs stay in L2 for the length of the kernel (config-2 capture)
 
 
