@@ -64,6 +64,26 @@ def test_int32_extreme_codes(H, B):
     assert abs(int(acc[0, 0])) == 127 * 127 * K
 
 
+def test_longest_reduction_stays_inside_int32(H, B):
+    """K = 131072, the longest the interface accepts: 127 * 127 * K = 2 114 060 288 < 2^31, with both signs; one more
+    k-block of 16 is refused."""
+    M, N, K = 130, 144, 131072
+    Xq = np.full((M, K), 127, np.int8)
+    Xq[1::2] = -127
+    Wq = np.full((N, K), 127, np.int8)
+    Wq[2::3] = -127
+    acc, _ = H.gpu_forward(Xq, None, Wq, None, None, B.QWT_OUT_INT32_ACC)
+    assert int(acc[0, 0]) == 127 * 127 * K and int(acc[1, 0]) == -127 * 127 * K and int(acc[1, 2]) == 127 * 127 * K
+    assert np.array_equal(acc.astype(np.int64), O.int_matmul(Xq, Wq))
+    import torch
+    d = H.dev(np.zeros((1, K + 16), np.int8))
+    y = torch.zeros(16, dtype=torch.int32, device=H.DEV)
+    w = H.dev(np.zeros((16, K + 16), np.int8))
+    ws = H.empty_bytes(4096)
+    assert B.qwt_qlinear_cwac_forward(d, None, w, B.QWT_W_INT8, None, None, 1, 16, K + 16, B.QWT_OUT_INT32_ACC, y, None,
+                                      ws, 4096, check=False) == B.QWT_ERR_SHAPE
+
+
 @pytest.mark.parametrize("M,N,K", SHAPES)
 def test_fp32_output_within_tolerance(H, B, M, N, K):
     Xq, Wq, xs, fs, fb = random_layer(M, N, K, seed=M + N + K + 1)
