@@ -249,7 +249,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   // Without the INT8 exchange nothing else in the workspace is used: the first CTA clears the status word
   // (a wait can only give up seconds later).
-  if (!C::kInt8Out && blockIdx.x == 0 && threadIdx.x == 0) *p.status = 0u;
+  if ((!C::kInt8Out || p.counter_target <= 1u) && blockIdx.x == 0 && threadIdx.x == 0) *p.status = 0u;
 
   auto give_up = [&](uint32_t code) {
     *cta_abort = 1;
@@ -695,7 +695,9 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         unsigned long long* slot = p.partial + ((size_t)tm * words) * kBM + qd * 32 + my;
         float amax_row = 0.f;
         int good = 1;
-        if (words > 0) {
+        if (strip_units == 1) {
+          amax_row = amax_mine;      // the unit is the whole row: nothing to exchange (and nothing was cleared)
+        } else if (words > 0) {
           ptx::st_relaxed_gpu_u64(slot + (size_t)(n0 / kUnitN) * kBM,
                                   (1ull << 32) | (unsigned long long)__float_as_uint(amax_mine));
           // all words of the row are requested together (one L2 round trip when they are all there)
@@ -1131,7 +1133,7 @@ qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams p
     QWT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  if (C::kInt8Out) {
+  if (C::kInt8Out && prm.counter_target > 1u) {
     // the row-maximum exchange needs every CTA of the grid resident
     void* args[] = {(void*)&tmA, (void*)&tmB, (void*)&tmY, (void*)&prm};
     QWT_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, smem_bytes, st));
@@ -1300,7 +1302,9 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   }
   // per-token INT8 output: the status word and the exchanged row maxima start at zero.  The other output
   // modes use only the status word, which their kernel clears itself (one launch less per call).
-  if (out_mode == QWT_OUT_INT8_PER_TOKEN && plan.fused_requant) QWT_CUDA_TRY(cudaMemsetAsync(ws, 0, plan.ws_z_off, st));
+  // (a layer of at most one unit per strip, N <= 128, exchanges nothing: its kernel clears the status word itself)
+  const bool exchanges = out_mode == QWT_OUT_INT8_PER_TOKEN && plan.fused_requant && N > unit_cols(out_mode);
+  if (exchanges) QWT_CUDA_TRY(cudaMemsetAsync(ws, 0, plan.ws_z_off, st));
 
   QlParams prm{};
   prm.x_scale = x_scale;
