@@ -26,7 +26,8 @@
 //   phase 1  z from the accumulators (written back to TMEM in their place) -> row maxima of the unit (combined
 //            over the four lanes that share a row) -> published to the other CTAs of the strip:
 //            as a tagged 8-byte word per row and unit (strips of at most 32 units), or by atomicMax on
-//            rowmax[m] plus a strip counter and flag (wider layers);
+//            rowmax[m] plus a strip counter and flag (wider layers); a row that lies inside one tile is settled
+//            inside the CTA (one unit: nothing to do; two units: through shared memory);
 //   phase 2  once the maxima of every unit of the strip are there, the rows' scales follow (the unit at column
 //            0 writes y_scale); z is read back from TMEM, divided, rounded and stored as codes; only then is
 //            the TMEM buffer released.
@@ -95,6 +96,7 @@ struct QlParams {
   const int* x_zero;             // [M] Z_x per token
   const int* x_rowsum;           // [M] rsx[m] = sum_k x_q[m, k]
   const int* w_terms;            // [2 N]: -Z_W[n], then K Z_W[n] - sum_k W_q[n, k]
+  int local_pair;                // per-token INT8: a strip is one 256-wide tile of two units, exchanged inside the CTA
   // calibration statistics instead of an output matrix (Section 3.3, Eq. 4-5)
   const float* F;                // [M, ldf] full-precision output of the same layer on the same rows
   long long ldf;
@@ -132,8 +134,11 @@ struct Cfg {
   // per group and unit: fscale | fbias, and with asymmetric codes also the two integer column terms of Eq. 7
   static constexpr int kParamArrays = ASYM ? 4 : 2;
   static constexpr int kParamBytes = kGroups * kParamArrays * kUnitN * 4;
+  // per-token INT8 with the whole row inside one tile: the tile's two units exchange their row maxima here
+  // ([2 pairs of groups][2 buffers][2 units][128 rows] floats)
+  static constexpr int kPairBytes = kInt8Out ? 2 * 2 * 2 * kBM * 4 : 0;
   static constexpr int kBarBytes = 512;
-  static constexpr int kFixedBytes = kStagingBytes + kParamBytes + kBarBytes;
+  static constexpr int kFixedBytes = kStagingBytes + kParamBytes + kPairBytes + kBarBytes;
   static constexpr int kMaxStages = 12;
   // full[S], empty[S], conv[S], tfull[A], tempty[A], pfull[4], pub[4], ready[4], gdone[4], drain, wfull
   static constexpr int kNumBars = 3 * kMaxStages + 2 * kAcc + 4 * kGroups + 2;
@@ -193,7 +198,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   uint8_t* sP = sB + (resident ? 0 : stages * C::kBBytes);             // [stages][BN x 64 B] packed int4 (W4 only)
   uint8_t* sStage = smem + C::ring_bytes(stages, p.res_kb);
   float* sParam = reinterpret_cast<float*>(sStage + C::kStagingBytes);      // [group][fscale 128 | fbias 128]
-  uint8_t* sBars = sStage + C::kStagingBytes + C::kParamBytes;
+  float* sPair = reinterpret_cast<float*>(sStage + C::kStagingBytes + C::kParamBytes);
+  uint8_t* sBars = sStage + C::kStagingBytes + C::kParamBytes + C::kPairBytes;
   uint64_t* full = reinterpret_cast<uint64_t*>(sBars);
   uint64_t* empty = full + kMaxStages;
   uint64_t* conv = empty + kMaxStages;   // W4 only: the stage's W tile has been expanded to int8
@@ -226,7 +232,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     for (int i = 0; i < kGroups; ++i) {
       ptx::mbar_init(&pfull[i], 1);
-      ptx::mbar_init(&pub[i], kGroupWarps);
+      // (in-CTA exchange of a tile's two units: pub[g & ~1] counts the warps of both groups)
+      ptx::mbar_init(&pub[i], p.local_pair ? 2 * kGroupWarps : kGroupWarps);
       ptx::mbar_init(&ready[i], 1);
       ptx::mbar_init(&gdone[i], kGroupWarps);
     }
@@ -249,7 +256,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   // Without the INT8 exchange nothing else in the workspace is used: the first CTA clears the status word
   // (a wait can only give up seconds later).
-  if ((!C::kInt8Out || p.counter_target <= 1u) && blockIdx.x == 0 && threadIdx.x == 0) *p.status = 0u;
+  if ((!C::kInt8Out || p.counter_target <= 1u || p.local_pair) && blockIdx.x == 0 && threadIdx.x == 0) *p.status = 0u;
 
   auto give_up = [&](uint32_t code) {
     *cta_abort = 1;
@@ -697,6 +704,17 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int good = 1;
         if (strip_units == 1) {
           amax_row = amax_mine;      // the unit is the whole row: nothing to exchange (and nothing was cleared)
+        } else if (p.local_pair) {
+          // the row is this tile's two units, handled by the groups g and g ^ 1: through shared memory (two
+          // buffers: the pair's next tile comes two tiles later, when everybody has long read this one)
+          const uint32_t xp = (uint32_t)(j >> 1) & 1u;
+          float* const pbuf = sPair + ((uint32_t)(g >> 1) * 2 + xp) * 2 * kBM;      // [unit of the tile][row]
+          float* mine = pbuf + (uint32_t)(u % UPT) * kBM + qd * 32 + my;
+          *mine = amax_mine;
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&pub[g & ~1]);
+          if (!ptx::mbar_wait_bounded(&pub[g & ~1], xp, cta_abort, tmo)) good = 0;
+          else amax_row = fmaxf(amax_mine, pbuf[(uint32_t)((u % UPT) ^ 1) * kBM + qd * 32 + my]);
         } else if (words > 0) {
           ptx::st_relaxed_gpu_u64(slot + (size_t)(n0 / kUnitN) * kBM,
                                   (1ull << 32) | (unsigned long long)__float_as_uint(amax_mine));
@@ -1133,7 +1151,7 @@ qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams p
     QWT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  if (C::kInt8Out && prm.counter_target > 1u) {
+  if (C::kInt8Out && prm.counter_target > 1u && !prm.local_pair) {
     // the row-maximum exchange needs every CTA of the grid resident
     void* args[] = {(void*)&tmA, (void*)&tmB, (void*)&tmY, (void*)&prm};
     QWT_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, smem_bytes, st));
@@ -1303,7 +1321,10 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   // per-token INT8 output: the status word and the exchanged row maxima start at zero.  The other output
   // modes use only the status word, which their kernel clears itself (one launch less per call).
   // (a layer of at most one unit per strip, N <= 128, exchanges nothing: its kernel clears the status word itself)
-  const bool exchanges = out_mode == QWT_OUT_INT8_PER_TOKEN && plan.fused_requant && N > unit_cols(out_mode);
+  const bool local_pair = out_mode == QWT_OUT_INT8_PER_TOKEN && plan.fused_requant && plan.tiles_n == 1 &&
+                          plan.bn == 256 && N > unit_cols(out_mode);
+  const bool exchanges = out_mode == QWT_OUT_INT8_PER_TOKEN && plan.fused_requant && N > unit_cols(out_mode) &&
+                         !local_pair;
   if (exchanges) QWT_CUDA_TRY(cudaMemsetAsync(ws, 0, plan.ws_z_off, st));
 
   QlParams prm{};
@@ -1322,6 +1343,7 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   // units of a row strip that lie inside the matrix
   prm.counter_target = (uint32_t)((N + unit_cols(out_mode) - 1) / unit_cols(out_mode));
   prm.gather_words = plan.gather_words;
+  prm.local_pair = local_pair ? 1 : 0;
   prm.x_zero = x_zero;
   prm.x_rowsum = x_rowsum;
   prm.w_terms = w_terms;

@@ -129,6 +129,17 @@ def test_zero_rows_and_zero_scale(H, B):
     assert_codes_close(codes, c_ref)
 
 
+@pytest.mark.parametrize("M,N,K", [(94757, 208, 64), (25088, 256, 128), (19000, 144, 48)])
+def test_whole_row_inside_one_tile(H, B, M, N, K):
+    """128 < N <= 256 with many rows: a row strip is one 256-wide tile, its two units exchange their row maxima
+    inside the CTA (several tiles per CTA, so the exchange buffers and barrier phases alternate)."""
+    Xq, Wq, xs, fs, fb = random_layer(M, N, K, seed=M + N)
+    codes, ys = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_INT8_PER_TOKEN)
+    c_ref, ys_ref = O.requant_per_token(O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb))
+    assert np.allclose(ys, ys_ref, rtol=1e-5)
+    assert_codes_close(codes, c_ref)
+
+
 def test_config1_layer_end_to_end(H, B):
     """Config 1: quantize -> calibrate CWAC on 32 images -> fold -> fused forward, every stage against the oracle."""
     spec = WL.config_layers(1)[0]
