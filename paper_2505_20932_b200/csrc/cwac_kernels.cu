@@ -277,9 +277,9 @@ cwac_reduce_batch_kernel(const __grid_constant__ ReduceBatch rb, int* __restrict
   int p = 0;
 #pragma unroll 1
   while (p + 1 < rb.count && (int)blockIdx.x >= rb.block0[p + 1]) ++p;
-  const ReduceProblem pr = rb.prob[p];
-  cwac_reduce_block(pr.partial, pr.chunks, pr.cpad, pr.channels, pr.n_rows, nullptr, pr.a, pr.b, n_degenerate,
-                    (int)blockIdx.x - rb.block0[p], pr.w_scale, pr.bias, pr.fscale, pr.fbias);
+  const ReduceProblem* pr = rb.prob + p;
+  cwac_reduce_block(pr->partial, pr->chunks, pr->cpad, pr->channels, pr->n_rows, nullptr, pr->a, pr->b, n_degenerate,
+                    (int)blockIdx.x - rb.block0[p], pr->w_scale, pr->bias, pr->fscale, pr->fbias);
 }
 
 __global__ void __launch_bounds__(128)
