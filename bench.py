@@ -124,7 +124,7 @@ def _quant_rows(B, torch, X, qmax):
     return q, s
 
 
-def build_layer(B, torch, WL, spec, seed, device, calib_rows=None):
+def build_layer(B, torch, WL, spec, seed, device, calib_rows=None, keep_calib_inputs=False):
     L = Layer()
     L.spec = spec
     M, K, N = spec.M, spec.K, spec.N
@@ -162,6 +162,8 @@ def build_layer(B, torch, WL, spec, seed, device, calib_rows=None):
         L.fp_out += torch.randn((R, N), generator=g, device=device) * (0.01 * sd)[None, :]
     else:
         L.fp_out = torch.addmm(L.bias, Xc, W.t())
+    # the quantized calibration inputs of the first layers are kept for the in-layer calibration figure
+    L.Xcq, L.xcs = (Xcq, xcs) if keep_calib_inputs else (None, None)
     del Xc, Xcq, xcs, W
     L.a = torch.empty(N, dtype=torch.float32, device=device)
     L.b = torch.empty(N, dtype=torch.float32, device=device)
@@ -366,7 +368,8 @@ def run_ours(args):
         import dataclasses
         specs = [dataclasses.replace(sp, out=args.out) for sp in specs]
     layers = [build_layer(B, torch, WL, sp, args.seed + 1000 * rank + i, device,
-                          calib_rows=(min(sp.calib_rows, args.calib_rows) if args.calib_rows else None))
+                          calib_rows=(min(sp.calib_rows, args.calib_rows) if args.calib_rows else None),
+                          keep_calib_inputs=(rank == 0 and i < 4))
               for i, sp in enumerate(specs)]
     torch.cuda.synchronize()
     stream = torch.cuda.current_stream()
@@ -489,6 +492,33 @@ def run_ours(args):
                "what": "phase B through qwt_qlinear_cwac_forward_host: pinned host X/x_scale in, host Y/y_scale out, per layer"}
         del staging, host
 
+    # ---- calibration inside the layer (the statistics accumulated in the layer's own epilogue, the quantized output
+    # never stored) on the first four layers: an extra figure outside the timed region, checked against phase A's fit
+    in_layer = None
+    if rank == 0:
+        us, moved, worst = 0.0, 0, 0.0
+        for L in layers[:4]:
+            s = L.spec
+            wsb = B.qwt_qlinear_cwac_calibrate_workspace_bytes(L.R, s.N, s.K, L.wfmt)
+            ws = torch.empty(wsb, dtype=torch.uint8, device=device)
+            a2, b2 = torch.empty_like(L.a), torch.empty_like(L.b)
+            call = lambda: B.qwt_qlinear_cwac_calibrate(L.Xcq, L.xcs, L.W, L.wfmt, L.ws, L.bias, L.fp_out, s.N, L.R, s.N, s.K,
+                                                        None, a2, b2, None, ws, wsb, stream)
+            call()
+            q0, q1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            q0.record(stream)
+            for _ in range(3):
+                call()
+            q1.record(stream)
+            torch.cuda.synchronize()
+            B.qwt_qlinear_check_status(ws)
+            us += q0.elapsed_time(q1) * 1e3 / 3
+            moved += 4 * L.R * s.N + L.R * s.K + s.N * (s.K if s.w_bits == 8 else s.K // 2)
+            worst = max(worst, float(((a2 - L.a).abs() / L.a.abs().clamp_min(1e-6)).max()))
+            del ws, L.Xcq, L.xcs
+        in_layer = {"value": moved / us / 1e3, "unit": "GB/s", "us": us, "layers": min(4, len(layers)),
+                    "bytes": "4 R N (fp_out) + R K (codes) + weights", "max_rel_diff_of_a_vs_phase_A": worst}
+
     # ---- an on-box INT8 reference point: the library's plain int8 x int8 -> int32 matmul (no epilogue) at 8192^3,
     # timed outside the timed region.  Context for the "% INT8 peak" figures, not part of the path.
     lib_int8_tops = None
@@ -573,7 +603,8 @@ def run_ours(args):
                         "min_time_ms": max(t_min_compute, t_min_hbm) * 1e3,
                         "frac_of_roofline": max(t_min_compute, t_min_hbm) / (t_b / args.steps)},
             "roofline": dominant, "rooflines": [roof_cal, roof_fwd],
-            "cpu_baseline": cpu, "e2e": e2e, "gpu_launches": int(launches), "clocks": clocks,
+            "cpu_baseline": cpu, "e2e": e2e, "calibration_in_layer": in_layer, "gpu_launches": int(launches),
+            "clocks": clocks,
         }
         print(json.dumps(line))
     if world > 1:
