@@ -27,7 +27,8 @@
 //            over the four lanes that share a row) -> published to the other CTAs of the strip:
 //            as a tagged 8-byte word per row and unit (strips of at most 32 units), or by atomicMax on
 //            rowmax[m] plus a strip counter and flag (wider layers); a row that lies inside one tile is settled
-//            inside the CTA (one unit: nothing to do; two units: through shared memory);
+//            inside the CTA (one unit: nothing to do; two units: through shared memory), and so is a row of
+//            exactly two tiles when the CTA takes whole strips (own strips);
 //   phase 2  once the maxima of every unit of the strip are there, the rows' scales follow (the unit at column
 //            0 writes y_scale); z is read back from TMEM, divided, rounded and stored as codes; only then is
 //            the TMEM buffer released.
@@ -97,6 +98,7 @@ struct QlParams {
   const int* x_rowsum;           // [M] rsx[m] = sum_k x_q[m, k]
   const int* w_terms;            // [2 N]: -Z_W[n], then K Z_W[n] - sum_k W_q[n, k]
   int local_pair;                // per-token INT8: a strip is one 256-wide tile of two units, exchanged inside the CTA
+  int own_strips;                // per-token INT8: a strip is two 256-wide tiles, both taken by the same CTA
   // calibration statistics instead of an output matrix (Section 3.3, Eq. 4-5)
   const float* F;                // [M, ldf] full-precision output of the same layer on the same rows
   long long ldf;
@@ -218,7 +220,15 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int lane = threadIdx.x & 31;
   const uint64_t tmo = p.timeout_ns;
   const int G = (int)gridDim.x;
-  const int n_local = (p.num_tiles - (int)blockIdx.x + G - 1) / G;    // tiles of this CTA
+  // Tiles of this CTA, in the order it takes them.  Default: b, b + G, b + 2G, ...  With own strips (per-token INT8
+  // whose rows span exactly two column tiles): the strips b, b + G, ... and both column tiles of each in turn, so
+  // that a row's maxima never leave the CTA.
+  const int tiles_m = p.num_tiles / p.tiles_n;
+  const int n_local = p.own_strips ? ((int)blockIdx.x < tiles_m ? ((tiles_m - (int)blockIdx.x + G - 1) / G) * p.tiles_n : 0)
+                                   : (p.num_tiles - (int)blockIdx.x + G - 1) / G;
+  auto tile_of = [&](int j) {
+    return p.own_strips ? ((int)blockIdx.x + (j / p.tiles_n) * G) * p.tiles_n + j % p.tiles_n : (int)blockIdx.x + j * G;
+  };
 
   if (threadIdx.x == 0) {
     for (int i = 0; i < stages; ++i) {
@@ -233,7 +243,9 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     for (int i = 0; i < kGroups; ++i) {
       ptx::mbar_init(&pfull[i], 1);
       // (in-CTA exchange of a tile's two units: pub[g & ~1] counts the warps of both groups)
-      ptx::mbar_init(&pub[i], p.local_pair ? 2 * kGroupWarps : kGroupWarps);
+      // (own strips: pub[0] counts the warps of all the strip's units)
+      ptx::mbar_init(&pub[i], p.own_strips ? kGroupWarps * (int)p.counter_target
+                                           : (p.local_pair ? 2 * kGroupWarps : kGroupWarps));
       ptx::mbar_init(&ready[i], 1);
       ptx::mbar_init(&gdone[i], kGroupWarps);
     }
@@ -256,7 +268,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   // Without the INT8 exchange nothing else in the workspace is used: the first CTA clears the status word
   // (a wait can only give up seconds later).
-  if ((!C::kInt8Out || p.counter_target <= 1u || p.local_pair) && blockIdx.x == 0 && threadIdx.x == 0) *p.status = 0u;
+  if ((!C::kInt8Out || p.counter_target <= 1u || p.local_pair || p.own_strips) && blockIdx.x == 0 && threadIdx.x == 0)
+    *p.status = 0u;
 
   auto give_up = [&](uint32_t code) {
     *cta_abort = 1;
@@ -276,7 +289,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
       uint32_t issued = 0, s = 0, ph = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += G) {
+      for (int jt = 0; ok && jt < n_local; ++jt) {
+        const int tile = tile_of(jt);
         const int m0 = (tile / p.tiles_n) * kBM;
         const int n0 = (tile % p.tiles_n) * BN;
         for (int kb = 0; kb < p.num_kb; ++kb, ++issued) {
@@ -328,7 +342,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         give_up(kStWaitFull);
         ok = false;
       }
-      for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += G, ++it) {
+      for (int jt = 0; ok && jt < n_local; ++jt, ++it) {
         const uint32_t buf = it % kAcc;
         if (!ptx::mbar_wait_bounded(&tempty[buf], ((it / kAcc) & 1u) ^ 1u, cta_abort, tmo)) {
           give_up(kStWaitTmemEmpty);
@@ -375,7 +389,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int ct = threadIdx.x - C::kConvWarp0 * 32;       // 0..127
     uint32_t s = 0, ph = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; ok && tile < p.num_tiles; tile += G) {
+    for (int jt = 0; ok && jt < n_local; ++jt) {
       for (int kb = 0; kb < p.num_kb; ++kb) {
         if (!ptx::mbar_wait_bounded(&full[s], ph, cta_abort, tmo)) {
           give_up(kStWaitFull);
@@ -436,7 +450,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     float pre_fs[kUnitN / 32], pre_fb[kUnitN / 32];
 
     auto unit_col0 = [&](int u) {           // first column of unit u in the output matrix
-      const int tile = (int)blockIdx.x + (u / UPT) * G;
+      const int tile = tile_of(u / UPT);
       return (tile % p.tiles_n) * BN + (u % UPT) * kUnitN;
     };
     auto prefetch_params = [&](int u) {
@@ -507,7 +521,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     int reloads = 0;                        // times the slice has been (re)loaded
     for (int u = g; u < n_units; u += kGroups, ++use) {
       const int j = u / UPT;
-      const int tile = (int)blockIdx.x + j * G;
+      const int tile = tile_of(j);
       const int tm = tile / p.tiles_n;
       const int n0 = unit_col0(u);
       const uint32_t buf = j % kAcc, tpar = (j / kAcc) & 1u, upar = use & 1u;
@@ -704,6 +718,20 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         int good = 1;
         if (strip_units == 1) {
           amax_row = amax_mine;      // the unit is the whole row: nothing to exchange (and nothing was cleared)
+        } else if (p.own_strips) {
+          // the row is this CTA's two tiles of the strip: all its units (up to 4, one per group) meet in shared
+          // memory (two buffers by the strip's ordinal: a group can be one strip ahead of the readers of the last)
+          const uint32_t xp = (uint32_t)(j / p.tiles_n) & 1u;
+          float* const sbuf = sPair + xp * 4 * kBM;                                   // [unit of the strip][row]
+          sbuf[(uint32_t)((tile % p.tiles_n) * UPT + u % UPT) * kBM + qd * 32 + my] = amax_mine;
+          __syncwarp();
+          if (lane == 0) ptx::mbar_arrive(&pub[0]);
+          if (!ptx::mbar_wait_bounded(&pub[0], xp, cta_abort, tmo)) {
+            good = 0;
+          } else {
+            amax_row = amax_mine;
+            for (int v = 0; v < strip_units; ++v) amax_row = fmaxf(amax_row, sbuf[v * kBM + qd * 32 + my]);
+          }
         } else if (p.local_pair) {
           // the row is this tile's two units, handled by the groups g and g ^ 1: through shared memory (two
           // buffers: the pair's next tile comes two tiles later, when everybody has long read this one)
@@ -1151,7 +1179,7 @@ qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams p
     QWT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  if (C::kInt8Out && prm.counter_target > 1u && !prm.local_pair) {
+  if (C::kInt8Out && prm.counter_target > 1u && !prm.local_pair && !prm.own_strips) {
     // the row-maximum exchange needs every CTA of the grid resident
     void* args[] = {(void*)&tmA, (void*)&tmB, (void*)&tmY, (void*)&prm};
     QWT_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, smem_bytes, st));
@@ -1268,6 +1296,19 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   pl.w_resident = !w4 && w_tile_bytes <= 96 * 1024 && pl.tiles_n <= sms && tiles > sms &&
                   !(nores != nullptr && nores[0] == '1');
   if (pl.w_resident) pl.grid = (sms / pl.tiles_n) * pl.tiles_n;
+  // Per-token INT8 whose rows span exactly two 256-wide tiles, with at least half a grid of strips: a CTA takes
+  // whole strips (both tiles, one after the other in its two accumulator buffers), so that the row maxima are
+  // settled inside the CTA: no workspace clearing, no cooperative launch, no L2 round trips.
+  {
+    const char* e = getenv("QWT_OWN_STRIPS");
+    const bool want = e != nullptr ? e[0] == '1' : true;
+    pl.own_strips = want && out_mode == QWT_OUT_INT8_PER_TOKEN && pl.tiles_n == 2 && pl.bn == 256 && !w4 &&
+                    pl.tiles_m >= sms / 2;
+    if (pl.own_strips) {
+      pl.w_resident = false;
+      pl.grid = pl.tiles_m < sms ? pl.tiles_m : sms;
+    }
+  }
   pl.fused_requant = (out_mode == QWT_OUT_INT8_PER_TOKEN) && (pl.tiles_n <= pl.grid);
   size_t off = 0;
   pl.ws_status_off = off;
@@ -1324,7 +1365,7 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   const bool local_pair = out_mode == QWT_OUT_INT8_PER_TOKEN && plan.fused_requant && plan.tiles_n == 1 &&
                           plan.bn == 256 && N > unit_cols(out_mode);
   const bool exchanges = out_mode == QWT_OUT_INT8_PER_TOKEN && plan.fused_requant && N > unit_cols(out_mode) &&
-                         !local_pair;
+                         !local_pair && !plan.own_strips;
   if (exchanges) QWT_CUDA_TRY(cudaMemsetAsync(ws, 0, plan.ws_z_off, st));
 
   QlParams prm{};
@@ -1344,6 +1385,7 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   prm.counter_target = (uint32_t)((N + unit_cols(out_mode) - 1) / unit_cols(out_mode));
   prm.gather_words = plan.gather_words;
   prm.local_pair = local_pair ? 1 : 0;
+  prm.own_strips = plan.own_strips ? 1 : 0;
   prm.x_zero = x_zero;
   prm.x_rowsum = x_rowsum;
   prm.w_terms = w_terms;

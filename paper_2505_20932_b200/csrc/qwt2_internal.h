@@ -91,6 +91,7 @@ struct QlinearPlan {
   bool fused_requant;    // cross-CTA row-max protocol inside the GEMM kernel
   int gather_words;      // INT8 output: exchange words per row (one per 128-column unit; 0 = counter protocol)
   bool w_resident;       // grid is a multiple of tiles_n: a CTA's W tile can stay in shared memory
+  bool own_strips;       // per-token INT8 with two column tiles per strip: a CTA takes whole strips
   bool w4_expand;        // packed int4 weights are expanded to int8 in the workspace first (many rows: the GEMM is
                          // compute-bound and the int8 mainloop is twice as fast as the one that converts on chip)
   size_t ws_status_off, ws_partial_off, ws_z_off, ws_w_off, ws_total;

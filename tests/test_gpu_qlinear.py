@@ -140,6 +140,19 @@ def test_whole_row_inside_one_tile(H, B, M, N, K):
     assert_codes_close(codes, c_ref)
 
 
+@pytest.mark.parametrize("M,N,K,own", [(10000, 400, 272, "1"), (10000, 400, 272, "0"), (40000, 512, 64, "1"), (9500, 272, 1040, "1")])
+def test_rows_spanning_two_tiles(H, B, M, N, K, own, monkeypatch):
+    """256 < N <= 512 with at least half a grid of strips: a CTA takes whole strips and settles the row maxima inside
+    itself (several strips per CTA: both exchange buffers and barrier phases); switched off, the same layer goes
+    through the exchange between CTAs.  Same results either way."""
+    monkeypatch.setenv("QWT_OWN_STRIPS", own)
+    Xq, Wq, xs, fs, fb = random_layer(M, N, K, seed=M + N + K)
+    codes, ys = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_INT8_PER_TOKEN)
+    c_ref, ys_ref = O.requant_per_token(O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb))
+    assert np.allclose(ys, ys_ref, rtol=1e-5)
+    assert_codes_close(codes, c_ref)
+
+
 def test_config1_layer_end_to_end(H, B):
     """Config 1: quantize -> calibrate CWAC on 32 images -> fold -> fused forward, every stage against the oracle."""
     spec = WL.config_layers(1)[0]
