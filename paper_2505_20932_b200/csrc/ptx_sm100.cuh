@@ -169,6 +169,13 @@ __device__ __forceinline__ void tmem_ld_32x32b_x32(uint32_t taddr, uint32_t (&r)
                : "memory");
 }
 
+// max(m, |x|, |y|) in one three-input instruction
+__device__ __forceinline__ float max3_abs(float m, float x, float y) {
+  float r;
+  asm("{\n\t.reg .f32 ax, ay;\n\tabs.f32 ax, %2;\n\tabs.f32 ay, %3;\n\tmax.f32 %0, %1, ax, ay;\n\t}" : "=f"(r) : "f"(m), "f"(x), "f"(y));
+  return r;
+}
+
 // Registers -> TMEM, same fragment layout as tmem_ld_16x256b_x4 (32 columns x 16 lanes).
 __device__ __forceinline__ void tmem_st_16x256b_x4(uint32_t taddr, const uint32_t (&r)[16]) {
   asm volatile("tcgen05.st.sync.aligned.16x256b.x4.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16};" ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])

@@ -680,7 +680,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             if (ASYM) asym_fix(a0 + 4 * i, a1 + 4 * i, h * 32 + 8 * i);
             z_block(a0 + 4 * i, a1 + 4 * i, h * 32 + 8 * i, z);
 #pragma unroll
-            for (int k = 0; k < 4; ++k) amax[k] = fmaxf(amax[k], fmaxf(fabsf(z[k].x), fabsf(z[k].y)));
+            for (int k = 0; k < 4; ++k) amax[k] = ptx::max3_abs(amax[k], z[k].x, z[k].y);
             // z replaces the accumulators in TMEM: phase 2 reads it back instead of recomputing it
             a0[4 * i] = __float_as_uint(z[0].x);
             a0[4 * i + 1] = __float_as_uint(z[0].y);
