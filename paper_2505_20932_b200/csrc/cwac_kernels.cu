@@ -238,7 +238,7 @@ __device__ __forceinline__ void cwac_reduce_block(const double* __restrict__ par
 #pragma unroll
   for (int i = 0; i < 4; ++i) {
     double t = 0.0;
-#pragma unroll
+#pragma unroll 4      // (fully unrolled, the 128 loads of the four sums are hoisted and spill)
     for (int y = 0; y < kRedTY; ++y) t += red[y][i][tx];
     s[i] = t;
   }
