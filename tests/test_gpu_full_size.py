@@ -8,7 +8,7 @@ import torch
 
 from oracle import qwt_oracle as O
 from paper_2505_20932_b200 import workload as WL
-from tolerances import assert_ab_close, assert_codes_close
+from tolerances import assert_ab_close, assert_bf16_close, assert_codes_close
 
 pytestmark = pytest.mark.gpu
 DEV = "cuda"
@@ -82,8 +82,7 @@ def test_config3_layer_sampled_rows_w4_bf16(B):
     z = O.forward_folded(O.int_matmul(Xq[rt].cpu().numpy(), Wq.cpu().numpy()), xs[rt].cpu().numpy(), fs.cpu().numpy(),
                          fb.cpu().numpy())
     bits = Y[rt].view(torch.int16).cpu().numpy().view(np.uint16)
-    d = np.abs(bits.astype(np.int32) - O.to_bf16_bits(z).astype(np.int32))
-    assert d.max() <= 1 and np.count_nonzero(d) <= max(1, int(1e-4 * d.size))
+    assert_bf16_close(bits, z, O.to_bf16_bits, O.bf16_bits_to_f32)
 
 
 @pytest.mark.parametrize("C,bits", [(768, 4), (3072, 8)])

@@ -4,7 +4,7 @@ import pytest
 
 from oracle import qwt_oracle as O
 from paper_2505_20932_b200 import workload as WL
-from tolerances import assert_codes_close, assert_fp32_close
+from tolerances import assert_bf16_close, assert_codes_close, assert_fp32_close
 
 pytestmark = pytest.mark.gpu
 
@@ -111,10 +111,7 @@ def test_bf16_output(H, B, M, N, K):
     Xq, Wq, xs, fs, fb = random_layer(M, N, K, seed=M + N + K + 3)
     bits, _ = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_BF16)
     z_ref = O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb)
-    ref_bits = O.to_bf16_bits(z_ref)
-    d = np.abs(bits.astype(np.int32) - ref_bits.astype(np.int32))
-    assert d.max() <= 1                                   # at most one bfloat16 ulp ...
-    assert np.count_nonzero(d) <= max(1, int(1e-4 * d.size))     # ... on at most 0.01 % of the elements
+    assert_bf16_close(bits, z_ref, O.to_bf16_bits, O.bf16_bits_to_f32)     # <= 1 bf16 ulp on <= 0.01 % of the elements
 
 
 def test_zero_rows_and_zero_scale(H, B):
@@ -283,8 +280,7 @@ def test_w4_bf16_fp32_and_int8_outputs(H, B, M, N, K):
     assert_fp32_close(z, z_ref)
     if N % 8 == 0:
         bits, _ = H.gpu_forward(Xq, xs, Wp, fs, fb, B.QWT_OUT_BF16, wfmt=B.QWT_W_INT4_PACKED, K=K)
-        d = np.abs(bits.astype(np.int32) - O.to_bf16_bits(z_ref).astype(np.int32))
-        assert d.max() <= 1 and np.count_nonzero(d) <= max(1, int(1e-4 * d.size))
+        assert_bf16_close(bits, z_ref, O.to_bf16_bits, O.bf16_bits_to_f32)
     codes, ys = H.gpu_forward(Xq, xs, Wp, fs, fb, B.QWT_OUT_INT8_PER_TOKEN, wfmt=B.QWT_W_INT4_PACKED, K=K)
     c_ref, ys_ref = O.requant_per_token(z_ref)
     assert np.allclose(ys, ys_ref, rtol=1e-5)
@@ -304,8 +300,7 @@ def test_w4_quantize_pack_forward_chain(H, B):
     fs, fb = fs.astype(np.float32), fb.astype(np.float32)
     bits, _ = H.gpu_forward(Xq, xs, O.pack_int4(Wq), fs, fb, B.QWT_OUT_BF16, wfmt=B.QWT_W_INT4_PACKED, K=spec.K)
     z_ref = O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb)
-    dd = np.abs(bits.astype(np.int32) - O.to_bf16_bits(z_ref).astype(np.int32))
-    assert dd.max() <= 1 and np.count_nonzero(dd) <= max(1, int(1e-4 * dd.size))
+    assert_bf16_close(bits, z_ref, O.to_bf16_bits, O.bf16_bits_to_f32)
 
 
 # ------------------------------------------------------------------ CNN-shaped layers (1x1 convolutions)

@@ -4,6 +4,10 @@ FP32 outputs: the kernel forms z with three FP32 roundings (int->float is exact 
 the fused multiply-add), the oracle in float64: |d| <= 1e-5 |ref| + 1e-6 leaves two orders of magnitude of room.
 INT8 codes: both sides round an FP32 quotient; they may disagree where it lies within a few 1e-6 of a half-integer,
 which is rare (about one code in a million measured): at most 1 LSB on at most 0.01 % of the elements.
+BF16 outputs: the bits of bf16_rne(float32(z_oracle)), except that the kernel rounds ITS FP32 z, which may sit on the
+other side of a bf16 rounding boundary: at most one bf16 ulp on at most 0.01 % of the elements.  Where z nearly
+cancels (|z| below 1e-4, i.e. a hundred times the FP32 absolute tolerance) an FP32 error of 1e-9 already moves several
+bf16 ulps of that tiny number; those elements are held to the FP32 tolerance instead.
 CWAC a, b: FP32 results of float64 sums, 1e-5 relative (b with an absolute floor of 1e-6 of the channel's scale)."""
 import numpy as np
 
@@ -39,3 +43,22 @@ def assert_ab_close(a, b, a_ref, b_ref, scale_b):
     db = np.abs(b - b_ref)
     lim = AB_REL * np.abs(b_ref) + 1e-6 * np.asarray(scale_b) + 1e-7
     assert np.all(db <= lim), f"b: worst excess {np.max(db - lim):.3e}"
+
+
+BF16_TINY = 1e-4     # |z| below this: compared as values (the FP32 tolerance), not as bf16 bit patterns
+
+
+def assert_bf16_close(bits, z_ref, to_bf16_bits, bf16_bits_to_f32, what="bf16"):
+    """bits: uint16 patterns from the kernel; z_ref: float64 oracle values; the two converters are the oracle's."""
+    z_ref = np.asarray(z_ref, dtype=np.float64)
+    bits = np.asarray(bits).astype(np.uint16)
+    ref_bits = to_bf16_bits(z_ref)
+    d = np.abs(bits.astype(np.int32) - ref_bits.astype(np.int32))
+    tiny = np.abs(z_ref) < BF16_TINY
+    big = ~tiny
+    assert d[big].max(initial=0) <= 1, f"{what}: {d[big].max()} bf16 ulps off"
+    assert np.count_nonzero(d[big]) <= max(1, int(1e-4 * d.size)), f"{what}: {np.count_nonzero(d[big])} elements differ"
+    if tiny.any():
+        got = bf16_bits_to_f32(bits[tiny]).astype(np.float64)
+        err = np.abs(got - z_ref[tiny])
+        assert np.all(err <= 2.0 ** -8 * np.abs(z_ref[tiny]) + FP32_ABS), f"{what}: tiny element off by {err.max():.3e}"
