@@ -13,6 +13,8 @@
  *   - Argument errors are found on the host before anything is launched.
  *   - Inputs are assumed finite; NaN/Inf behaviour is unspecified.  Outputs must not alias inputs.
  *   - Calls may run concurrently on different streams if their workspaces are distinct.
+ *   - Grids, workspace layouts and summation orders are functions of the problem shape only and are laid out for
+ *     the 148 SMs of a B200; a call on a device with fewer SMs than its persistent grid returns QWT_ERR_ARCH.
  */
 #ifndef QWT2_H_
 #define QWT2_H_
@@ -130,15 +132,18 @@ qwt_status qwt_cwac_calibrate_batch(const qwt_calib_problem* problems /*HOST*/, 
  * memory arena, or a service that must not call cudaMalloc while it is serving.  The per-chunk partial sums
  * live in a fixed array of QWT_NOALLOC_SCRATCH_BYTES inside the library image; every GPU that loads the
  * library holds that array until the process exits.  The call itself allocates nothing.
- *   - Limit: channels (rounded up to 128) * 32 bytes must fit the array, i.e. at most 131072 channels;
+ *   - Limit: channels (rounded up to 128) * 48 bytes must fit the array, i.e. at most 131072 channels;
  *     otherwise QWT_ERR_TOO_LARGE.  Long inputs are cut into fewer, longer row chunks so that they fit.
  *   - The first call on each device looks up the array's device address (with that device current); make
  *     that first call before any stream capture is started.
+ *   - The address is kept per device ordinal for the life of the process.  It belongs to the device's primary
+ *     context as it was at that first call: after cudaDeviceReset, or under another (non-primary) context on the same
+ *     device, it is stale and the entry point must not be used in that process any more.
  *   - All calls share the one array.  Nothing in it has to be cleared between calls (each call overwrites
  *     what it reads), but two calls that overlap on the GPU -- different streams, or different host threads
  *     -- race on it: serialise them, or use qwt_cwac_calibrate with separate workspaces.
  * Arguments and other errors as for qwt_cwac_calibrate. */
-#define QWT_NOALLOC_SCRATCH_BYTES (4u << 20)
+#define QWT_NOALLOC_SCRATCH_BYTES (6u << 20)
 qwt_status qwt_cwac_calibrate_noalloc(const float* fp_out, const float* q_out, int64_t rows, int32_t channels,
                                       int64_t ld, float* a, float* b, int32_t* n_degenerate, void* stream);
 
@@ -298,6 +303,20 @@ qwt_status qwt_qlinear_cwac_forward_asym(const uint8_t* X, const float* x_scale,
  * Errors: NULL, SHAPE, UNSUPPORTED (C % 16), ALIGN, ARCH, CUDA. */
 qwt_status qwt_im2col_i8(const int8_t* X, int32_t batch, int32_t H, int32_t W, int32_t C, int32_t kh, int32_t kw,
                          int32_t stride, int32_t pad, int8_t* patches, void* stream);
+
+/* ---------------------------------------------------------------------------------------------
+ * Test hooks (the paper has no counterpart).  Host-side, process-wide switches that exist so that the give-up path of
+ * the bounded device-side waits can be exercised without faulting or hanging a GPU; both are 0 in normal operation.
+ *   qwt_test_set_wait_limit_ns  bound of every device-side wait of the forward calls issued afterwards, in
+ *                               nanoseconds; 0 restores the default (QWT_TIMEOUT_MS from the environment, else 2 s).
+ *   qwt_test_set_phantom_units  per-token INT8 forward calls planned afterwards expect n (0..4) more 128-column units
+ *                               per row strip than the layer has.  Nothing ever publishes a row maximum for them, so
+ *                               the exchange of a layer wider than 128 columns cannot complete: every CTA's wait runs
+ *                               out after the limit, the kernel records a code in the workspace status word, tears
+ *                               down and returns, and qwt_qlinear_check_status reports QWT_ERR_TIMEOUT; Y and y_scale
+ *                               are then undefined.  Workspace sizes are planned with the same n. */
+void qwt_test_set_wait_limit_ns(uint64_t ns);
+void qwt_test_set_phantom_units(int32_t n);
 
 /* Kernels launched by this library on the calling thread since the last reset (for launch accounting). */
 int64_t qwt_launch_count(void);

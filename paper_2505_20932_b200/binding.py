@@ -21,7 +21,7 @@ lib = C.CDLL(LIB_PATH)
 # status / enums (mirrors of qwt2.h)
 QWT_OK, QWT_ERR_NULL, QWT_ERR_SHAPE, QWT_ERR_ALIGN, QWT_ERR_UNSUPPORTED = 0, 1, 2, 3, 4
 QWT_ERR_WORKSPACE, QWT_ERR_CUDA, QWT_ERR_TIMEOUT, QWT_ERR_ARCH, QWT_ERR_TOO_LARGE = 5, 6, 7, 8, 9
-QWT_NOALLOC_SCRATCH_BYTES = 4 << 20
+QWT_NOALLOC_SCRATCH_BYTES = 6 << 20
 QWT_W_INT8, QWT_W_INT4_PACKED = 0, 1
 QWT_OUT_INT8_PER_TOKEN, QWT_OUT_BF16, QWT_OUT_FP32, QWT_OUT_INT32_ACC, QWT_OUT_INT8_STATIC = 0, 1, 2, 3, 4
 
@@ -57,6 +57,8 @@ SIGNATURES = {
     "qwt_quantize_rows_i8": (_i32, [_p, _i64, _i32, _i64, _i32, _p, _p, _p]),
     "qwt_im2col_i8": (_i32, [_p, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _p, _p]),
     "qwt_pack_int4": (_i32, [_p, _i64, _i32, _p, _p]),
+    "qwt_test_set_wait_limit_ns": (None, [C.c_uint64]),
+    "qwt_test_set_phantom_units": (None, [_i32]),
     "qwt_launch_count": (_i64, []),
     "qwt_launch_count_reset": (None, []),
 }
@@ -313,3 +315,11 @@ def qwt_launch_count() -> int:
 
 def qwt_launch_count_reset() -> None:
     lib.qwt_launch_count_reset()
+
+
+def qwt_test_set_wait_limit_ns(ns: int) -> None:
+    lib.qwt_test_set_wait_limit_ns(int(ns))
+
+
+def qwt_test_set_phantom_units(n: int) -> None:
+    lib.qwt_test_set_phantom_units(int(n))

@@ -13,6 +13,11 @@ namespace qwt {
 static thread_local int tl_cuda_error = 0;
 static thread_local int64_t tl_launches = 0;
 
+TestHooks& test_hooks() {
+  static TestHooks hooks;     // zero-initialised
+  return hooks;
+}
+
 void set_cuda_error(int err) { tl_cuda_error = err; }
 void count_launch(int n) { tl_launches += n; }
 
@@ -82,6 +87,11 @@ qwt_status qwt_last_cuda_error(int* cuda_err) {
   return QWT_OK;
 }
 
+void qwt_test_set_wait_limit_ns(uint64_t ns) { test_hooks().wait_limit_ns.store(ns, std::memory_order_relaxed); }
+void qwt_test_set_phantom_units(int32_t n) {
+  test_hooks().phantom_units.store(n < 0 ? 0 : (n > 4 ? 4 : n), std::memory_order_relaxed);
+}
+
 int64_t qwt_launch_count(void) { return tl_launches; }
 void qwt_launch_count_reset(void) { tl_launches = 0; }
 
@@ -89,7 +99,7 @@ void qwt_launch_count_reset(void) { tl_launches = 0; }
 
 size_t qwt_cwac_workspace_bytes(int64_t rows, int32_t channels) {
   if (rows < 1 || channels < 1) return 0;
-  return cwac_plan(rows, channels, 148).partial_bytes;
+  return cwac_plan(rows, channels, kPlanSMs).partial_bytes;
 }
 
 qwt_status qwt_cwac_calibrate(const float* fp_out, const float* q_out, int64_t rows, int32_t channels, int64_t ld,
@@ -98,7 +108,7 @@ qwt_status qwt_cwac_calibrate(const float* fp_out, const float* q_out, int64_t r
   qwt_status s = check_calib_args(fp_out, q_out, rows, channels, ld);
   if (s != QWT_OK) return s;
   if (a == nullptr || b == nullptr || workspace == nullptr) return QWT_ERR_NULL;
-  const CwacPlan plan = cwac_plan(rows, channels, 148);
+  const CwacPlan plan = cwac_plan(rows, channels, kPlanSMs);
   if (workspace_bytes < plan.partial_bytes || !aligned(workspace, 256)) return QWT_ERR_WORKSPACE;
   DeviceInfo dev;
   if ((s = current_device(&dev)) != QWT_OK) return s;
@@ -144,7 +154,7 @@ qwt_status qwt_cwac_stats_accumulate(const float* fp_out, const float* q_out, in
   qwt_status s = check_calib_args(fp_out, q_out, rows, channels, ld);
   if (s != QWT_OK) return s;
   if (stats == nullptr || workspace == nullptr) return QWT_ERR_NULL;
-  const CwacPlan plan = cwac_plan(rows, channels, 148);
+  const CwacPlan plan = cwac_plan(rows, channels, kPlanSMs);
   if (workspace_bytes < plan.partial_bytes || !aligned(workspace, 256)) return QWT_ERR_WORKSPACE;
   DeviceInfo dev;
   if ((s = current_device(&dev)) != QWT_OK) return s;
@@ -183,7 +193,7 @@ HostCalibLayout host_calib_layout(int64_t rows, int32_t channels) {
   L.off_out = off; off += up((size_t)2 * channels * 4 + 16);
   L.slot_bytes = up((size_t)cr * channels * 4);
   for (int i = 0; i < 2; ++i) { L.off_slot[i] = off; off += 2 * L.slot_bytes; }
-  L.ws_bytes = cwac_plan(cr, channels, 148).partial_bytes;
+  L.ws_bytes = cwac_plan(cr, channels, kPlanSMs).partial_bytes;
   L.off_ws = off; off += up(L.ws_bytes);
   L.total = off;
   return L;
@@ -248,7 +258,7 @@ qwt_status qwt_cwac_calibrate_host(const float* fp_out, const float* q_out, int6
                                    (size_t)nr, cudaMemcpyHostToDevice, copy_st));
       QWT_HC_TRY(cudaEventRecord(copied[slot], copy_st));
       QWT_HC_TRY(cudaStreamWaitEvent(st, copied[slot], 0));
-      const CwacPlan plan = cwac_plan(nr, channels, 148);
+      const CwacPlan plan = cwac_plan(nr, channels, kPlanSMs);
       if ((rc = launch_cwac_stats(d_fp, d_q, nr, channels, channels, nullptr, base + L.off_ws, plan, st)) != QWT_OK) goto done;
       if ((rc = launch_cwac_reduce(base + L.off_ws, plan, channels, nr, stats, nullptr, nullptr, nullptr, st)) != QWT_OK) goto done;
       QWT_HC_TRY(cudaEventRecord(reduced[slot], st));
@@ -316,7 +326,7 @@ static qwt_status check_forward_args(const void* X, const float* x_scale, const 
 size_t qwt_qlinear_workspace_bytes(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode) {
   if (M < 1 || N < 1 || K < 1) return 0;
   DeviceInfo dev{};
-  dev.sm_count = 148;
+  dev.sm_count = kPlanSMs;
   QlinearPlan plan;
   if (qlinear_plan(M, N, K, wfmt, out_mode, dev, &plan) != QWT_OK) return 0;
   return plan.ws_total;
@@ -330,7 +340,7 @@ qwt_status qwt_qlinear_cwac_forward(const int8_t* X, const float* x_scale, const
   if (s != QWT_OK) return s;
   if (workspace == nullptr) return QWT_ERR_NULL;
   DeviceInfo dev{};
-  dev.sm_count = 148;
+  dev.sm_count = kPlanSMs;
   QlinearPlan plan;
   if ((s = qlinear_plan(M, N, K, wfmt, out_mode, dev, &plan)) != QWT_OK) return s;
   if (workspace_bytes < plan.ws_total || !aligned(workspace, 256)) return QWT_ERR_WORKSPACE;
@@ -352,7 +362,7 @@ qwt_status qwt_qlinear_cwac_forward_asym(const uint8_t* X, const float* x_scale,
   if (x_zero == nullptr || x_rowsum == nullptr || w_terms == nullptr || workspace == nullptr) return QWT_ERR_NULL;
   if (K > 33000) return QWT_ERR_SHAPE;   // 255^2 * K must stay below 2^31
   DeviceInfo dev{};
-  dev.sm_count = 148;
+  dev.sm_count = kPlanSMs;
   QlinearPlan plan;
   if ((s = qlinear_plan(M, N, K, QWT_W_INT8, out_mode, dev, &plan)) != QWT_OK) return s;
   if (workspace_bytes < plan.ws_total || !aligned(workspace, 256)) return QWT_ERR_WORKSPACE;
@@ -372,7 +382,7 @@ struct FusedCalibLayout {
 };
 qwt_status fused_calib_layout(int32_t M, int32_t N, int32_t K, int32_t wfmt, FusedCalibLayout* L) {
   DeviceInfo dev{};
-  dev.sm_count = 148;
+  dev.sm_count = kPlanSMs;
   qwt_status s = qlinear_plan(M, N, K, wfmt, kOutCalibStats, dev, &L->plan);
   if (s != QWT_OK) return s;
   L->red = CwacPlan{};
@@ -380,7 +390,7 @@ qwt_status fused_calib_layout(int32_t M, int32_t N, int32_t K, int32_t wfmt, Fus
   L->red.cpad = L->red.slabs * 128;
   L->red.chunks = L->plan.tiles_m;
   L->red.chunk_rows = 128;
-  L->red.partial_bytes = (size_t)L->red.chunks * 4 * L->red.cpad * sizeof(double);
+  L->red.partial_bytes = (size_t)L->red.chunks * kPartialValues * L->red.cpad * sizeof(double);
   L->off_partial = 256;
   // the expanded int8 copy of packed weights (if the plan asks for one) goes behind the partials
   L->plan.ws_w_off = (L->off_partial + L->red.partial_bytes + 255) / 256 * 256;

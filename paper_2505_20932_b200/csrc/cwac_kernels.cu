@@ -18,8 +18,11 @@ namespace qwt {
 // The sums run in FP32 for FLUSH rows and are then added to FP64 accumulators, so FP32 only ever adds
 // a handful of terms of the size of the channel's spread (the shift removes the mean), which keeps the
 // variance and covariance accurate for channels whose mean is far from zero.  At the end of the chunk
-// the shifted sums are turned back into raw sums in FP64 and written as one partial per (chunk, sum,
-// channel).  No atomics: a second kernel adds the partials in chunk order, so results are reproducible.
+// the four shifted sums and the two shifts are written as one partial per (chunk, value, channel), still in
+// shifted form: a second kernel re-references every chunk to the shift of chunk 0 (a change of the size of the
+// channel's spread, not of its mean), adds the chunks in a fixed order and solves Eq. 4-5 from sums that
+// never held the square of the mean -- var(q) = E[q^2] - E[q]^2 on raw FP64 sums loses log10((mean/std)^2)
+// digits.  No atomics, so results are reproducible.
 // ------------------------------------------------------------------------------------------------
 // Descriptors of a batched launch (passed by value as kernel parameters).
 constexpr int kMaxBatch = 48;        // 48 descriptors of 80 bytes + the block offsets stay below the 4 KB of kernel parameters
@@ -44,7 +47,7 @@ struct ReduceProblem {
   float* fscale;
   float* fbias;
   double n_rows;
-  int chunks, cpad, channels, pad_;
+  int chunks, cpad, channels, chunk_rows;
 };
 struct ReduceBatch {
   int count;
@@ -154,18 +157,14 @@ __device__ __forceinline__ void cwac_stats_block(const float* __restrict__ fp_ou
       for (int y = 0; y < kStatsTY; ++y) t += red[y][s * 4 + j][ltx];
       sd[s] = t;
     }
-    const double nb = (double)(r1 - r0);
-    const double Kq = (double)shift_q[ch], Kf = (double)shift_f[ch];
-    // raw sums from the shifted ones
-    const double Sq = sd[0] + nb * Kq;
-    const double Sf = sd[1] + nb * Kf;
-    const double Sqf = sd[2] + Kf * sd[0] + Kq * sd[1] + nb * Kq * Kf;
-    const double Sqq = sd[3] + 2.0 * Kq * sd[0] + nb * Kq * Kq;
-    double* out = partial + (size_t)chunk * 4 * cpad + c;
-    out[0 * (size_t)cpad] = Sq;
-    out[1 * (size_t)cpad] = Sf;
-    out[2 * (size_t)cpad] = Sqf;
-    out[3 * (size_t)cpad] = Sqq;
+    // shifted sums and the shifts themselves (kPartialValues per chunk and channel)
+    double* out = partial + (size_t)chunk * kPartialValues * cpad + c;
+    out[0 * (size_t)cpad] = sd[0];
+    out[1 * (size_t)cpad] = sd[1];
+    out[2 * (size_t)cpad] = sd[2];
+    out[3 * (size_t)cpad] = sd[3];
+    out[4 * (size_t)cpad] = (double)shift_q[ch];
+    out[5 * (size_t)cpad] = (double)shift_f[ch];
   }
 }
 
@@ -208,13 +207,34 @@ __device__ __forceinline__ void cwac_solve_channel(double n, double Sq, double S
   *b = (float)(mf - alpha * mq);
 }
 
+// The same from sums of values shifted by (Kq, Kf): variance and covariance do not see the shift, the means do.
+__device__ __forceinline__ void cwac_solve_channel_shifted(double n, double s0, double s1, double s2, double s3,
+                                                           double Kq, double Kf, float* a, float* b, int* degenerate) {
+  const double dq = s0 / n, df = s1 / n;            // means of the shifted values
+  const double var = s3 / n - dq * dq;
+  const double cov = s2 / n - dq * df;
+  const double mq = Kq + dq, mf = Kf + df;
+  const double msq = var + mq * mq;                  // E[q^2]
+  double alpha;
+  if (var <= 1e-12 * msq) {
+    alpha = 1.0;
+    *degenerate = 1;
+  } else {
+    alpha = cov / var;
+    *degenerate = 0;
+  }
+  *a = (float)alpha;
+  *b = (float)(mf - alpha * mq);
+}
+
 // Adds the partials of all row chunks.  A block owns 32 channels; its 32 row lanes each add every 32nd
 // chunk, then the lanes are combined in a fixed order, so the result does not depend on scheduling.
 // stats_io (may be NULL): running statistics to update.  a, b (may be NULL): solve after the reduction.
 constexpr int kRedTX = 32;
 constexpr int kRedTY = 32;
 __device__ __forceinline__ void cwac_reduce_block(const double* __restrict__ partial, int chunks, int cpad,
-                                                  int channels, double n_rows, double* __restrict__ stats_io,
+                                                  int channels, double n_rows, int chunk_rows,
+                                                  double* __restrict__ stats_io,
                                                   float* __restrict__ a, float* __restrict__ b,
                                                   int* __restrict__ n_degenerate, int block,
                                                   const float* __restrict__ w_scale, const float* __restrict__ bias,
@@ -223,11 +243,20 @@ __device__ __forceinline__ void cwac_reduce_block(const double* __restrict__ par
   const int ty = threadIdx.x / kRedTX;
   const int c = block * kRedTX + tx;            // < cpad by construction of the grid
   double s[4] = {0.0, 0.0, 0.0, 0.0};
+  double K0q = 0.0, K0f = 0.0;                  // reference shift: that of chunk 0
   if (c < channels) {
+    K0q = partial[(size_t)4 * cpad + c];
+    K0f = partial[(size_t)5 * cpad + c];
     for (int k = ty; k < chunks; k += kRedTY) {
-      const double* p = partial + (size_t)k * 4 * cpad + c;
-#pragma unroll
-      for (int i = 0; i < 4; ++i) s[i] += p[(size_t)i * cpad];
+      const double* p = partial + (size_t)k * kPartialValues * cpad + c;
+      const double left = n_rows - (double)k * (double)chunk_rows;
+      const double nb = left < (double)chunk_rows ? left : (double)chunk_rows;      // rows of this chunk
+      const double d0 = p[0], d1 = p[(size_t)cpad], d2 = p[2 * (size_t)cpad], d3 = p[3 * (size_t)cpad];
+      const double dq = p[4 * (size_t)cpad] - K0q, df = p[5 * (size_t)cpad] - K0f;
+      s[0] += d0 + nb * dq;
+      s[1] += d1 + nb * df;
+      s[2] += d2 + df * d0 + dq * d1 + nb * dq * df;
+      s[3] += d3 + 2.0 * dq * d0 + nb * dq * dq;
     }
   }
   __shared__ double red[kRedTY][4][kRedTX];
@@ -243,6 +272,25 @@ __device__ __forceinline__ void cwac_reduce_block(const double* __restrict__ par
     s[i] = t;
   }
   double n = n_rows;
+  if (stats_io == nullptr && a != nullptr) {     // one-shot fit: solve from the shifted sums
+    int deg;
+    cwac_solve_channel_shifted(n, s[0], s[1], s[2], s[3], K0q, K0f, &a[c], &b[c], &deg);
+    if (deg && n_degenerate != nullptr) atomicAdd(n_degenerate, 1);
+    if (w_scale != nullptr) {     // Eq. 11 at once, the arithmetic of cwac_fold_kernel
+      const float ai = a[c], bi = b[c];
+      const float bs = bias ? bias[c] : 0.0f;
+      fscale[c] = ai * w_scale[c];
+      fbias[c] = fmaf(ai, bs, bi);
+    }
+    return;
+  }
+  {   // running statistics are raw sums (the interface of the streaming calls): undo the reference shift
+    const double r0 = s[0], r1 = s[1];
+    s[0] = r0 + n * K0q;
+    s[1] = r1 + n * K0f;
+    s[2] = s[2] + K0f * r0 + K0q * r1 + n * K0q * K0f;
+    s[3] = s[3] + 2.0 * K0q * r0 + n * K0q * K0q;
+  }
   if (stats_io != nullptr) {
     n += stats_io[c];
 #pragma unroll
@@ -266,10 +314,10 @@ __device__ __forceinline__ void cwac_reduce_block(const double* __restrict__ par
 
 __global__ void __launch_bounds__(kRedTX * kRedTY)
 cwac_reduce_kernel(const double* __restrict__ partial, int chunks, int cpad, int channels, double n_rows,
-                   double* __restrict__ stats_io, float* __restrict__ a, float* __restrict__ b,
+                   int chunk_rows, double* __restrict__ stats_io, float* __restrict__ a, float* __restrict__ b,
                    int* __restrict__ n_degenerate) {
-  cwac_reduce_block(partial, chunks, cpad, channels, n_rows, stats_io, a, b, n_degenerate, (int)blockIdx.x, nullptr,
-                    nullptr, nullptr, nullptr);
+  cwac_reduce_block(partial, chunks, cpad, channels, n_rows, chunk_rows, stats_io, a, b, n_degenerate, (int)blockIdx.x,
+                    nullptr, nullptr, nullptr, nullptr);
 }
 
 __global__ void __launch_bounds__(kRedTX * kRedTY)
@@ -278,7 +326,8 @@ cwac_reduce_batch_kernel(const __grid_constant__ ReduceBatch rb, int* __restrict
 #pragma unroll 1
   while (p + 1 < rb.count && (int)blockIdx.x >= rb.block0[p + 1]) ++p;
   const ReduceProblem* pr = rb.prob + p;
-  cwac_reduce_block(pr->partial, pr->chunks, pr->cpad, pr->channels, pr->n_rows, nullptr, pr->a, pr->b, n_degenerate,
+  cwac_reduce_block(pr->partial, pr->chunks, pr->cpad, pr->channels, pr->n_rows, pr->chunk_rows, nullptr, pr->a, pr->b,
+                    n_degenerate,
                     (int)blockIdx.x - rb.block0[p], pr->w_scale, pr->bias, pr->fscale, pr->fbias);
 }
 
@@ -512,7 +561,7 @@ CwacPlan cwac_plan(int64_t rows, int32_t channels, int /*sm_count*/) {
   chunk_rows = (chunk_rows + kStatsTY - 1) / kStatsTY * kStatsTY;
   p.chunk_rows = chunk_rows;
   p.chunks = (int)((rows + chunk_rows - 1) / chunk_rows);
-  p.partial_bytes = (size_t)p.chunks * 4 * p.cpad * sizeof(double);
+  p.partial_bytes = (size_t)p.chunks * kPartialValues * p.cpad * sizeof(double);
   return p;
 }
 
@@ -528,9 +577,10 @@ qwt_status launch_cwac_stats(const float* fp_out, const float* q_out, int64_t ro
 qwt_status launch_cwac_reduce(const void* workspace, const CwacPlan& plan, int32_t channels, int64_t rows,
                               double* stats_io, float* a, float* b, int32_t* n_degenerate, cudaStream_t st) {
   if (a != nullptr && n_degenerate != nullptr) QWT_CUDA_TRY(cudaMemsetAsync(n_degenerate, 0, sizeof(int32_t), st));
-  cwac_reduce_kernel<<<(channels + kRedTX - 1) / kRedTX, kRedTX * kRedTY, 0, st>>>(static_cast<const double*>(workspace), plan.chunks,
-                                                             plan.cpad, channels, (double)rows, stats_io, a, b,
-                                                             n_degenerate);
+  if (plan.chunk_rows > 0x7fffffffll) return QWT_ERR_SHAPE;
+  cwac_reduce_kernel<<<(channels + kRedTX - 1) / kRedTX, kRedTX * kRedTY, 0, st>>>(
+      static_cast<const double*>(workspace), plan.chunks, plan.cpad, channels, (double)rows, (int)plan.chunk_rows, stats_io,
+      a, b, n_degenerate);
   QWT_LAUNCH_CHECK();
   return QWT_OK;
 }
@@ -538,7 +588,7 @@ qwt_status launch_cwac_reduce(const void* workspace, const CwacPlan& plan, int32
 size_t cwac_batch_workspace_bytes(const CalibBatchItem* items, int32_t count) {
   size_t total = 0;
   for (int32_t i = 0; i < count; ++i)
-    total += (cwac_plan(items[i].rows, items[i].channels, 148).partial_bytes + 255) / 256 * 256;
+    total += (cwac_plan(items[i].rows, items[i].channels, kPlanSMs).partial_bytes + 255) / 256 * 256;
   return total;
 }
 
@@ -557,7 +607,7 @@ qwt_status launch_cwac_calibrate_batch(const CalibBatchItem* items, int32_t coun
     int sblocks = 0, rblocks = 0;
     for (int i = 0; i < n; ++i) {
       const CalibBatchItem& it = items[g0 + i];
-      const CwacPlan plan = cwac_plan(it.rows, it.channels, 148);
+      const CwacPlan plan = cwac_plan(it.rows, it.channels, kPlanSMs);
       double* partial = reinterpret_cast<double*>(ws + off);
       off += (plan.partial_bytes + 255) / 256 * 256;
       sb.block0[i] = sblocks;
@@ -565,8 +615,9 @@ qwt_status launch_cwac_calibrate_batch(const CalibBatchItem* items, int32_t coun
                                 plan.slabs, 0};
       sblocks += plan.slabs * plan.chunks;
       rb.block0[i] = rblocks;
+      if (plan.chunk_rows > 0x7fffffffll) return QWT_ERR_SHAPE;
       rb.prob[i] = ReduceProblem{partial, it.a, it.b, it.w_scale, it.bias, it.fscale, it.fbias, (double)it.rows,
-                                 plan.chunks, plan.cpad, it.channels, 0};
+                                 plan.chunks, plan.cpad, it.channels, (int)plan.chunk_rows};
       rblocks += (it.channels + kRedTX - 1) / kRedTX;
     }
     sb.block0[n] = sblocks;

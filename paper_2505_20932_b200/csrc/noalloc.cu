@@ -17,7 +17,7 @@ qwt_status launch_cwac_reduce(const void* workspace, const CwacPlan& plan, int32
 
 namespace {
 
-// 4 MiB of per-chunk partial sums (double[chunks][4][channels padded to 128]).  Every GPU that loads the
+// 6 MiB of per-chunk partial sums (double[chunks][6][channels padded to 128]).  Every GPU that loads the
 // library carries this array until the process exits.
 constexpr size_t kScratchBytes = QWT_NOALLOC_SCRATCH_BYTES;
 static __device__ __align__(256) unsigned char g_calib_scratch[kScratchBytes];
@@ -51,8 +51,8 @@ extern "C" qwt_status qwt_cwac_calibrate_noalloc(const float* fp_out, const floa
   if (!aligned(fp_out, 16) || !aligned(q_out, 16) || (ld % 4) != 0) return QWT_ERR_ALIGN;
 
   // Same plan as qwt_cwac_calibrate, with fewer (longer) row chunks when its partial sums would not fit.
-  CwacPlan plan = cwac_plan(rows, channels, 148);
-  const size_t per_chunk = (size_t)4 * plan.cpad * sizeof(double);
+  CwacPlan plan = cwac_plan(rows, channels, kPlanSMs);
+  const size_t per_chunk = (size_t)kPartialValues * plan.cpad * sizeof(double);
   if (per_chunk > kScratchBytes) return QWT_ERR_TOO_LARGE;       // more than 131072 channels
   if (plan.partial_bytes > kScratchBytes) {
     const int64_t max_chunks = (int64_t)(kScratchBytes / per_chunk);

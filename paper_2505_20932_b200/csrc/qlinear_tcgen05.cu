@@ -45,6 +45,7 @@
 #include <stdint.h>
 #include <stdlib.h>
 
+#include <atomic>
 #include <mutex>
 #include <type_traits>
 
@@ -102,7 +103,7 @@ struct QlParams {
   // calibration statistics instead of an output matrix (Section 3.3, Eq. 4-5)
   const float* F;                // [M, ldf] full-precision output of the same layer on the same rows
   long long ldf;
-  double* sums;                  // [tiles_m][4][cpad]: sum q, sum f, sum q f, sum q q over the rows of a strip
+  double* sums;                  // [tiles_m][6][cpad]: shifted sums of q, f, q f, q q over the rows of a strip, and the two shifts
   int cpad;
 };
 
@@ -849,6 +850,13 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // column each, undo the shifts in FP64, add the four warps in order and write the strip's partial.  A
         // second kernel adds the strips in a fixed order.  Rows >= M and columns >= N contribute nothing.
         float* const wsum = reinterpret_cast<float*>(stg);      // [4 sums | shift of q | shift of f][128 columns]
+        // The slots of the group's four warps are read by all four after pub[g]: a warp may rewrite its own slot only
+        // when every warp of the group has finished the previous unit (the lead warp's wait above covers only the
+        // units whose columns change).
+        if (!ptx::mbar_wait_bounded(&gdone[g], upar ^ 1u, cta_abort, tmo)) {
+          give_up(kStWaitParam);
+          break;
+        }
         if (in_range) {
 #pragma unroll 2
           for (int h = 0; h < kUnitN / (8 * NB); ++h) {
@@ -931,27 +939,36 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         const int t = qd * 32 + lane;                           // the group's 128 threads take one column each
         if (in_range && n0 + t < p.N) {
-          double Sq = 0.0, Sf = 0.0, Sqf = 0.0, Sqq = 0.0;
+          // The four warps in the order of their rows (TMEM quadrant 0 first: its first row is the strip's first
+          // row, which always lies inside the matrix), every warp re-referenced to the shifts of quadrant 0 -- a
+          // change of the size of the channel's spread -- so that the strip's partial stays in shifted form.
+          double S0 = 0.0, S1 = 0.0, S2 = 0.0, S3 = 0.0, K0q = 0.0, K0f = 0.0;
 #pragma unroll
-          for (int w = 0; w < kGroupWarps; ++w) {
+          for (int qi = 0; qi < kGroupWarps; ++qi) {
             // the slot of epilogue warp g * 4 + w holds the rows of TMEM quadrant (g * 4 + w + 2) % 4
-            const int row0 = tm * kBM + ((g * kGroupWarps + w + 2) & 3) * 32;
-            const int left = p.M - row0;
+            const int w = (qi + 2) & 3;
+            const int left = p.M - (tm * kBM + qi * 32);
             if (left <= 0) continue;                            // nothing of this warp is inside the matrix
             const double nw = (double)(left < 32 ? left : 32);
             const float* ws4 = reinterpret_cast<const float*>(sStage + (g * kGroupWarps + w) * C::kSlotBytes) + t;
             const double d0 = ws4[0], d1 = ws4[kUnitN], d2 = ws4[2 * kUnitN], d3 = ws4[3 * kUnitN];
-            const double Kq = ws4[4 * kUnitN], Kf = ws4[5 * kUnitN];
-            Sq += d0 + nw * Kq;
-            Sf += d1 + nw * Kf;
-            Sqf += d2 + Kf * d0 + Kq * d1 + nw * Kq * Kf;
-            Sqq += d3 + 2.0 * Kq * d0 + nw * Kq * Kq;
+            if (qi == 0) {
+              K0q = ws4[4 * kUnitN];
+              K0f = ws4[5 * kUnitN];
+            }
+            const double dq = (double)ws4[4 * kUnitN] - K0q, df = (double)ws4[5 * kUnitN] - K0f;
+            S0 += d0 + nw * dq;
+            S1 += d1 + nw * df;
+            S2 += d2 + df * d0 + dq * d1 + nw * dq * df;
+            S3 += d3 + 2.0 * dq * d0 + nw * dq * dq;
           }
-          double* out = p.sums + (size_t)tm * 4 * (size_t)p.cpad + n0 + t;
-          out[0] = Sq;
-          out[(size_t)p.cpad] = Sf;
-          out[2 * (size_t)p.cpad] = Sqf;
-          out[3 * (size_t)p.cpad] = Sqq;
+          double* out = p.sums + (size_t)tm * kPartialValues * (size_t)p.cpad + n0 + t;
+          out[0] = S0;
+          out[(size_t)p.cpad] = S1;
+          out[2 * (size_t)p.cpad] = S2;
+          out[3 * (size_t)p.cpad] = S3;
+          out[4 * (size_t)p.cpad] = K0q;
+          out[5 * (size_t)p.cpad] = K0f;
         }
       } else if (C::kInt8Out && in_range) {
         // ---------------------------------------------------------------- phase 2: codes, box by box
@@ -1140,6 +1157,8 @@ bool make_byte_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t ro
 }
 
 unsigned long long timeout_ns_from_env() {
+  const unsigned long long forced = test_hooks().wait_limit_ns.load(std::memory_order_relaxed);
+  if (forced != 0ull) return forced;
   static unsigned long long v = [] {
     const char* e = getenv("QWT_TIMEOUT_MS");
     unsigned long long ms = 2000;
@@ -1172,12 +1191,13 @@ qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams p
   prm.stages = C::stages_for(res_kb);
   const int smem_bytes = C::dynamic_bytes(prm.stages, res_kb);
   // the opt-in shared-memory size is a per-device attribute of the function: set once per device
-  static bool attr_set[64] = {false};
+  // (setting it twice is harmless, so concurrent first calls need no lock, only an atomic flag)
+  static std::atomic<bool> attr_set[64];
   int dev = 0;
   QWT_CUDA_TRY(cudaGetDevice(&dev));
-  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+  if (dev < 0 || dev >= 64 || !attr_set[dev].load(std::memory_order_acquire)) {
     QWT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
-    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+    if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
   }
   if (C::kInt8Out && prm.counter_target > 1u && !prm.local_pair && !prm.own_strips) {
     // the row-maximum exchange needs every CTA of the grid resident
@@ -1267,7 +1287,8 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   // 256-wide tiles keep the tensor pipe ahead of shared-memory bandwidth and are used when the mainloop
   // dominates (long K); short-K layers are bound by the epilogue, which is organised around 128-wide tiles
   // (four accumulator buffers, so the INT8 row-maximum exchange can trail by two tiles).
-  const int sms = dev.sm_count > 0 ? dev.sm_count : 148;
+  const int sms = dev.sm_count > 0 ? dev.sm_count : kPlanSMs;
+  const int phantom = out_mode == QWT_OUT_INT8_PER_TOKEN ? test_hooks().phantom_units.load(std::memory_order_relaxed) : 0;
   auto score = [&](int bn) {
     const long tn = (N + bn - 1) / bn;
     const long tiles = (long)pl.tiles_m * tn;
@@ -1303,7 +1324,7 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
     const char* e = getenv("QWT_OWN_STRIPS");
     const bool want = e != nullptr ? e[0] == '1' : true;
     pl.own_strips = want && out_mode == QWT_OUT_INT8_PER_TOKEN && pl.tiles_n == 2 && pl.bn == 256 && !w4 &&
-                    pl.tiles_m >= sms / 2;
+                    pl.tiles_m >= sms / 2 && phantom == 0;
     if (pl.own_strips) {
       pl.w_resident = false;
       pl.grid = pl.tiles_m < sms ? pl.tiles_m : sms;
@@ -1314,7 +1335,9 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   pl.ws_status_off = off;
   off += 256;
   pl.ws_partial_off = off;      // (tag, row maximum) per strip row and 128-column unit
-  const int strip_units = (N + unit_cols(out_mode) - 1) / unit_cols(out_mode);
+  // (test hook: phantom units are expected by the exchange but never published, so that its bounded wait runs out)
+  const int strip_units = (N + unit_cols(out_mode) - 1) / unit_cols(out_mode) + phantom;
+  pl.strip_units = strip_units;
   // tagged words for strips of up to 16 units, and up to 32 when K is short enough for the exchange to show; with a
   // long mainloop the units of a strip finish far apart and the one-flag-per-strip protocol polls far less
   pl.gather_words = (strip_units <= 16 || (strip_units <= kMaxGatherWords && K <= 4096)) ? strip_units : 0;
@@ -1363,8 +1386,8 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   // modes use only the status word, which their kernel clears itself (one launch less per call).
   // (a layer of at most one unit per strip, N <= 128, exchanges nothing: its kernel clears the status word itself)
   const bool local_pair = out_mode == QWT_OUT_INT8_PER_TOKEN && plan.fused_requant && plan.tiles_n == 1 &&
-                          plan.bn == 256 && N > unit_cols(out_mode);
-  const bool exchanges = out_mode == QWT_OUT_INT8_PER_TOKEN && plan.fused_requant && N > unit_cols(out_mode) &&
+                          plan.bn == 256 && plan.strip_units == 2;
+  const bool exchanges = out_mode == QWT_OUT_INT8_PER_TOKEN && plan.fused_requant && plan.strip_units > 1 &&
                          !local_pair && !plan.own_strips;
   if (exchanges) QWT_CUDA_TRY(cudaMemsetAsync(ws, 0, plan.ws_z_off, st));
 
@@ -1382,7 +1405,7 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   prm.status = reinterpret_cast<uint32_t*>(ws + plan.ws_status_off);
   prm.partial = reinterpret_cast<unsigned long long*>(ws + plan.ws_partial_off);
   // units of a row strip that lie inside the matrix
-  prm.counter_target = (uint32_t)((N + unit_cols(out_mode) - 1) / unit_cols(out_mode));
+  prm.counter_target = (uint32_t)plan.strip_units;
   prm.gather_words = plan.gather_words;
   prm.local_pair = local_pair ? 1 : 0;
   prm.own_strips = plan.own_strips ? 1 : 0;

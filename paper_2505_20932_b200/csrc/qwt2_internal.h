@@ -4,9 +4,23 @@
 #include <cuda_runtime.h>
 #include <stdint.h>
 
+#include <atomic>
+
 #include "qwt2.h"
 
 namespace qwt {
+
+// Plans (tile walk, grids, workspace layouts, summation order) are functions of the problem shape only, laid out for
+// this many SMs, so that workspace sizes and the bits of the results do not depend on the device that happens to be
+// current; a call checks that the device has at least as many SMs as its plan's persistent grid.
+constexpr int kPlanSMs = 148;
+
+// Process-wide test hooks (qwt_test_* in the C ABI); both zero in normal operation.
+struct TestHooks {
+  std::atomic<unsigned long long> wait_limit_ns;   // != 0: bound of every device-side wait of later forward calls
+  std::atomic<int> phantom_units;                  // per-token INT8: units a row strip expects beyond those that exist
+};
+TestHooks& test_hooks();
 
 // thread-local record of the last CUDA failure and of the number of kernels launched
 void set_cuda_error(int err);
@@ -45,11 +59,14 @@ qwt_status current_device(DeviceInfo* out);
 inline bool aligned(const void* p, size_t a) { return (reinterpret_cast<uintptr_t>(p) % a) == 0; }
 
 // ---- calibration (cwac_kernels.cu)
+// Values per (row chunk, channel) in the partial sums of the statistics pass: four sums of shifted values
+// (dq, df, dq df, dq dq) and the two shifts.
+constexpr int kPartialValues = 6;
 struct CwacPlan {
   int slabs;        // column slabs of 128 channels
   int chunks;       // row chunks
   int64_t chunk_rows;
-  size_t partial_bytes;  // double[chunks][4][channels_padded]
+  size_t partial_bytes;  // double[chunks][kPartialValues][channels_padded]
   int cpad;         // channels rounded up to 128
 };
 CwacPlan cwac_plan(int64_t rows, int32_t channels, int sm_count);
@@ -90,6 +107,7 @@ struct QlinearPlan {
   int grid;
   bool fused_requant;    // cross-CTA row-max protocol inside the GEMM kernel
   int gather_words;      // INT8 output: exchange words per row (one per 128-column unit; 0 = counter protocol)
+  int strip_units;       // 128-column units of a row strip (whose row maxima the per-token INT8 exchange waits for)
   bool w_resident;       // grid is a multiple of tiles_n: a CTA's W tile can stay in shared memory
   bool own_strips;       // per-token INT8 with two column tiles per strip: a CTA takes whole strips
   bool w4_expand;        // packed int4 weights are expanded to int8 in the workspace first (many rows: the GEMM is
@@ -103,7 +121,7 @@ constexpr int kOutCalibStats = 5;
 struct QlinearStatsArgs {
   const float* F;      // [M, ldf] full-precision output
   int64_t ldf;
-  double* sums;        // [tiles_m][4][cpad] partials, one per strip of 128 rows
+  double* sums;        // [tiles_m][kPartialValues][cpad] partials, one per strip of 128 rows
   int cpad;
 };
 qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, int32_t wfmt, const float* fscale,

@@ -49,7 +49,12 @@ def calibrate_sharded(B, fp_out, q_out, rows_local: int, channels: int, ld: int,
     import torch
     if rows_local > 0:
         B.qwt_cwac_stats_accumulate(fp_out, q_out, rows_local, channels, ld, stats, workspace, workspace_bytes, stream)
-    if stream is not None:
+    # The collective is ordered with the CURRENT stream; when the library calls run on a side stream the all-reduce
+    # must wait for the local statistics and the solve must wait for the sum over ranks.
+    side = stream is not None and getattr(stats, "is_cuda", False)
+    if side:
         torch.cuda.current_stream().wait_stream(stream)
     allreduce_stats_(stats)
+    if side:
+        stream.wait_stream(torch.cuda.current_stream())
     B.qwt_cwac_solve(stats, channels, a, b, None, stream)

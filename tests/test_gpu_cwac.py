@@ -30,6 +30,19 @@ def test_calibrate_matches_oracle(H, rows, C, bits):
     assert_ab_close(a, b, a_ref, b_ref, nat_scale(fp))
 
 
+def test_calibrate_channel_means_far_above_their_spread(H):
+    """|mean| / std between 1e4 and 1e5: var(q) = E[q^2] - E[q]^2 loses nine to ten digits to cancellation."""
+    rng = np.random.default_rng(17)
+    rows, C = 20_000, 256
+    ratio = np.geomspace(1e4, 1e5, C)
+    q = (rng.standard_normal((rows, C)) + ratio[None, :]).astype(np.float32)
+    f = (1.03 * q.astype(np.float64) + 0.25 + 0.05 * rng.standard_normal((rows, C))).astype(np.float32)
+    a, b, nd = H.gpu_calibrate(f, q)
+    a_ref, b_ref, nd_ref = O.cwac_fit(f, q)
+    assert nd == nd_ref == 0
+    assert_ab_close(a, b, a_ref, b_ref, nat_scale(f))
+
+
 def test_calibrate_leading_dimension_and_ragged_channels(H):
     # 130 channels inside rows of 136 floats: the padding columns hold garbage that must not matter
     rows, C, ld = 777, 130, 136

@@ -130,3 +130,35 @@ def test_fused_argument_errors(H, B):
     bad = list(args)
     bad[7] = N - 4                                            # ld < N
     assert B.qwt_qlinear_cwac_calibrate(*bad, a, a.clone(), None, w, wsb, check=False) == B.QWT_ERR_SHAPE
+
+
+def test_fused_resident_weights_many_tiles_per_cta(H, B):
+    """One column tile, W resident in shared memory, six row strips per CTA: a group's warps reuse their staging slots
+    unit after unit without the parameter slice ever being reloaded.  Every channel against the oracle's sums, and two
+    runs on the same input bit for bit."""
+    M, N, K = 128 * 148 * 6 - 40, 256, 128
+    Xq, xs, Wq, ws, bias, fp, f, q = layer(M, N, K, seed=8, bias_mean=0.5)
+    r1 = H.gpu_calibrate_fused(Xq, xs, Wq, ws, bias, fp, stats=np.zeros((5, N)))
+    r2 = H.gpu_calibrate_fused(Xq, xs, Wq, ws, bias, fp, stats=np.zeros((5, N)))
+    assert np.array_equal(r1[0], r2[0]) and np.array_equal(r1[1], r2[1]) and np.array_equal(r1[3], r2[3])
+    a_ref, b_ref, nd_ref = O.cwac_fit(f, q)
+    assert r1[2] == nd_ref == 0
+    assert_ab_close(r1[0], r1[1], a_ref, b_ref, nat_scale(f))
+    s_ref = O.cwac_stats(f, q)
+    scale = np.stack([np.abs(q).sum(0), np.abs(f.astype(np.float64)).sum(0), np.abs(q * f).sum(0), (q * q).sum(0)])
+    assert np.array_equal(r1[3][0], s_ref[0])
+    assert np.all(np.abs(r1[3][1:] - s_ref[1:]) <= 2e-6 * scale + 1e-9)
+
+
+def test_fused_channel_means_far_above_their_spread(H, B):
+    """|mean| / std of the layer's output around 1e4 (a large bias on a unit-spread product): the variance is then a
+    difference of sums that agree to eight digits, which the shifted sums never form.  (At this ratio the fit is
+    already sensitive to the FP32 rounding of q itself -- steps of 1e-3 at 1e4 -- so the oracle fits the FP32 values
+    of its own q, as the layer's FP32 output stage would deliver them; a ratio of 3e4 moves b by its whole tolerance
+    when sixteen of a million q values round the other way.)"""
+    M, N, K = 4000, 256, 256
+    Xq, xs, Wq, ws, bias, fp, f, q = layer(M, N, K, seed=9, bias_mean=1.0e4)
+    a, b, nd, _ = H.gpu_calibrate_fused(Xq, xs, Wq, ws, bias, fp)
+    a_ref, b_ref, nd_ref = O.cwac_fit(f, q.astype(np.float32))
+    assert nd == nd_ref == 0
+    assert_ab_close(a, b, a_ref, b_ref, nat_scale(f))

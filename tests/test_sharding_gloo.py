@@ -74,3 +74,52 @@ def test_two_rank_statistics_allreduce_matches_single_process(tmp_path):
     b = sf / n - a * sq / n
     a_ref, b_ref, _ = O.cwac_fit(fp, q)
     assert np.allclose(a, a_ref, rtol=1e-9) and np.allclose(b, b_ref, rtol=1e-7, atol=1e-12)
+
+
+class _CpuBinding:
+    """Stands in for the ctypes binding on CPU tensors so that calibrate_sharded itself runs under gloo: the two calls
+    it makes are answered with the oracle's sums and with Eq. 4-5 written out."""
+
+    def qwt_cwac_stats_accumulate(self, fp, q, rows, C, ld, stats, ws, wsb, stream=None):
+        import torch
+        from oracle import qwt_oracle as O
+        stats += torch.from_numpy(O.cwac_stats(fp.numpy()[:rows, :C], q.numpy()[:rows, :C]).reshape(-1))
+
+    def qwt_cwac_solve(self, stats, C, a, b, nd, stream=None):
+        import torch
+        n, sq, sf, sqf, sqq = stats.reshape(5, C)
+        alpha = (sqf / n - (sq / n) * (sf / n)) / (sqq / n - (sq / n) ** 2)
+        a.copy_(alpha.float())
+        b.copy_((sf / n - alpha * sq / n).float())
+
+
+def _worker_sharded(rank, world, port, rows, C, out):
+    import torch
+    import torch.distributed as dist
+    from paper_2505_20932_b200 import workload as WL
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    try:
+        fp, q, _ = WL.host_calib_pair(rows, C, 4, seed=22)
+        s, n = sharding.shard_rows(rows, world, rank, align=8)
+        a, b = torch.empty(C), torch.empty(C)
+        stats = torch.zeros(5 * C, dtype=torch.float64)
+        sharding.calibrate_sharded(_CpuBinding(), torch.from_numpy(fp[s:s + n]), torch.from_numpy(q[s:s + n]), n, C, C,
+                                   a, b, stats, None, 0)
+        np.save(out + f".{rank}.npy", np.stack([a.numpy(), b.numpy()]))
+    finally:
+        dist.destroy_process_group()
+
+
+def test_calibrate_sharded_over_two_ranks(tmp_path):
+    import torch.multiprocessing as mp
+    from oracle import qwt_oracle as O
+    from paper_2505_20932_b200 import workload as WL
+    rows, C, world = 1203, 16, 2
+    out = str(tmp_path / "ab")
+    mp.spawn(_worker_sharded, args=(world, _free_port(), rows, C, out), nprocs=world, join=True)
+    fp, q, _ = WL.host_calib_pair(rows, C, 4, seed=22)
+    a_ref, b_ref, _ = O.cwac_fit(fp, q)
+    r0, r1 = np.load(out + ".0.npy"), np.load(out + ".1.npy")
+    assert np.array_equal(r0, r1)                            # every rank solves the same summed statistics
+    assert np.allclose(r0[0], a_ref, rtol=1e-6) and np.allclose(r0[1], b_ref, rtol=1e-6, atol=1e-7)

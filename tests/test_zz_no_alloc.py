@@ -5,6 +5,7 @@ other tests.  Passes alone in a fresh process and after the rest of the suite.""
 import numpy as np
 import pytest
 
+from oracle import qwt_oracle as O
 from paper_2505_20932_b200 import workload as WL
 from tolerances import assert_ab_close
 
@@ -49,6 +50,9 @@ def test_noalloc_calibration_matches_regular_entry_point_twice_in_a_row():
         assert n0 == n1 == 1 and a1[1] == 1.0
         scale = np.maximum(np.abs(fp[:, :C].mean(0)), fp[:, :C].std(0))
         assert_ab_close(a1, b1, a0, b0, scale)          # same tolerance as the oracle comparison of a, b
+        ch = np.unique(np.concatenate([np.random.default_rng(C).integers(0, C, 48), [0, 1, 127, 128, C - 1]]))
+        a_ref, b_ref, _ = O.cwac_fit(fp[:, ch], q[:, ch])        # and the oracle's own fit of sampled channels
+        assert_ab_close(a1[ch], b1[ch], a_ref, b_ref, scale[ch])
     assert B.qwt_cwac_workspace_bytes(2000, 12800) > B.QWT_NOALLOC_SCRATCH_BYTES
 
 

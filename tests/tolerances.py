@@ -39,9 +39,9 @@ def assert_ab_close(a, b, a_ref, b_ref, scale_b):
     a_ref = np.asarray(a_ref, dtype=np.float64)
     b_ref = np.asarray(b_ref, dtype=np.float64)
     da = np.abs(a - a_ref)
-    assert np.all(da <= AB_REL * np.abs(a_ref) + 1e-7), f"a: worst rel {np.max(da / np.maximum(np.abs(a_ref), 1e-30)):.3e}"
+    assert np.all(da <= AB_REL * np.abs(a_ref)), f"a: worst rel {np.max(da / np.maximum(np.abs(a_ref), 1e-30)):.3e}"
     db = np.abs(b - b_ref)
-    lim = AB_REL * np.abs(b_ref) + 1e-6 * np.asarray(scale_b) + 1e-7
+    lim = AB_REL * np.abs(b_ref) + 1e-6 * np.asarray(scale_b)
     assert np.all(db <= lim), f"b: worst excess {np.max(db - lim):.3e}"
 
 
