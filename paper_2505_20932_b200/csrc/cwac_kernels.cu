@@ -87,9 +87,11 @@ __device__ __forceinline__ void cwac_stats_block(const float* __restrict__ fp_ou
     kf[0] = b.x; kf[1] = b.y; kf[2] = b.z; kf[3] = b.w;
   }
 
-  double acc[16];
+  // FP64 accumulators: one private slot per thread and sum in shared memory (the same array the block reduction
+  // reads at the end), touched once per kFlushRows rows; in registers they would cost 32 of the thread's 128
+  __shared__ double red[kStatsTY][16][kStatsTX];
 #pragma unroll
-  for (int i = 0; i < 16; ++i) acc[i] = 0.0;
+  for (int i = 0; i < 16; ++i) red[ty][i][tx] = 0.0;
 
   if (active) {
     const float* qp = q_out + c0;
@@ -128,15 +130,12 @@ __device__ __forceinline__ void cwac_stats_block(const float* __restrict__ fp_ou
         }
       }
 #pragma unroll
-      for (int i = 0; i < 16; ++i) acc[i] += (double)s[i];
+      for (int i = 0; i < 16; ++i) red[ty][i][tx] += (double)s[i];
     }
   }
 
   // block reduction over the 8 row lanes, in a fixed order
-  __shared__ double red[kStatsTY][16][kStatsTX];
   __shared__ float shift_q[kSlabChannels], shift_f[kSlabChannels];
-#pragma unroll
-  for (int i = 0; i < 16; ++i) red[ty][i][tx] = acc[i];
   if (ty == 0) {
 #pragma unroll
     for (int j = 0; j < 4; ++j) {
