@@ -84,6 +84,9 @@ struct QlParams {
   float* y_scale;
   int M, N, K;
   int tiles_n, num_tiles, num_kb;
+  // the CTA's tile walk without divisions: CTA b has nl_mul * (nl_base + (b < nl_rem)) tiles; from one tile to the next
+  // the (row strip, column tile) pair moves by (step_q, step_r) with carry (default walk: b, b + G, ...)
+  int nl_base, nl_rem, nl_mul, step_q, step_r;
   int stages;           // depth of the operand ring in shared memory
   int res_kb;           // > 0: the CTA's W tile (all res_kb k-blocks) stays resident, the ring holds X only
   uint32_t* status;
@@ -184,6 +187,50 @@ __device__ __forceinline__ float2 z_pair(uint32_t a0, uint32_t a1, float2 xs2, f
   return __ffma2_rn(__fmul2_rn(a, xs2), make_float2(f0, f1), make_float2(b0, b1));
 }
 
+// The tiles of one CTA in the order it takes them, as (row strip, column tile), advanced without divisions.
+// Default: tiles b, b + G, b + 2G, ... of the strip-major numbering.  Own strips: the strips b, b + G, ... and every
+// column tile of each in turn.
+struct TileWalk {
+  int tm, tn;        // current tile
+  int ord;           // own strips: ordinal of the current strip among this CTA's strips
+  int tiles_n, step_q, step_r, G;
+  bool own;
+  __device__ __forceinline__ void init(const QlParams& p, int b, int G_) {
+    tiles_n = p.tiles_n;
+    step_q = p.step_q;
+    step_r = p.step_r;
+    G = G_;
+    own = p.own_strips != 0;
+    ord = 0;
+    if (own) {
+      tm = b;
+      tn = 0;
+    } else {
+      tm = b / tiles_n;            // the only division of the walk
+      tn = b - tm * tiles_n;
+    }
+  }
+  __device__ __forceinline__ void advance() {
+    if (own) {
+      if (++tn == tiles_n) {
+        tn = 0;
+        tm += G;
+        ++ord;
+      }
+    } else {
+      tn += step_r;
+      tm += step_q;
+      if (tn >= tiles_n) {
+        tn -= tiles_n;
+        ++tm;
+      }
+    }
+  }
+  __device__ __forceinline__ void advance(int n) {
+    for (int i = 0; i < n; ++i) advance();
+  }
+};
+
 template <int BN, int OUT, bool W4, bool WIDE, bool ASYM>
 __global__ void __launch_bounds__((Cfg<BN, OUT, W4, WIDE, ASYM>::kThreads), 1)
 qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
@@ -224,39 +271,30 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   // Tiles of this CTA, in the order it takes them.  Default: b, b + G, b + 2G, ...  With own strips (per-token INT8
   // whose rows span exactly two column tiles): the strips b, b + G, ... and both column tiles of each in turn, so
   // that a row's maxima never leave the CTA.
-  const int tiles_m = p.num_tiles / p.tiles_n;
-  const int n_local = p.own_strips ? ((int)blockIdx.x < tiles_m ? ((tiles_m - (int)blockIdx.x + G - 1) / G) * p.tiles_n : 0)
-                                   : (p.num_tiles - (int)blockIdx.x + G - 1) / G;
-  auto tile_of = [&](int j) {
-    return p.own_strips ? ((int)blockIdx.x + (j / p.tiles_n) * G) * p.tiles_n + j % p.tiles_n : (int)blockIdx.x + j * G;
-  };
+  const int n_local = p.nl_mul * (p.nl_base + ((int)blockIdx.x < p.nl_rem ? 1 : 0));
 
-  if (threadIdx.x == 0) {
-    for (int i = 0; i < stages; ++i) {
-      ptx::mbar_init(&full[i], 1);
-      ptx::mbar_init(&empty[i], 1);
-      ptx::mbar_init(&conv[i], kNumConvWarps);
+  if (warp == 0) {
+    // the barriers lie one after the other in shared memory; the lanes of warp 0 initialise them side by side
+    // (one thread doing all of them costs the CTA most of a microsecond before its first load)
+    if (lane == 0) {
+      ptx::prefetch_tensormap(&tmA);
+      ptx::prefetch_tensormap(&tmB);
+      if (C::kTmaStore) ptx::prefetch_tensormap(&tmY);
+      *cta_abort = 0;
     }
-    for (int i = 0; i < kAcc; ++i) {
-      ptx::mbar_init(&tfull[i], 1);
-      ptx::mbar_init(&tempty[i], kGroupWarps * C::kUPT);
+    for (int i = lane; i < C::kNumBars; i += 32) {
+      uint32_t count = 1;                                            // full, empty, tfull, pfull, ready, drain, wfull
+      if (i >= 2 * kMaxStages && i < 3 * kMaxStages) count = kNumConvWarps;                       // conv
+      else if (i >= 3 * kMaxStages + kAcc && i < 3 * kMaxStages + 2 * kAcc) count = kGroupWarps * C::kUPT;   // tempty
+      else if (i >= 3 * kMaxStages + 2 * kAcc + kGroups && i < 3 * kMaxStages + 2 * kAcc + 2 * kGroups)
+        // pub (in-CTA exchange of a tile's two units: pub[g & ~1] counts the warps of both groups; own strips:
+        // pub[0] counts the warps of all the strip's units)
+        count = p.own_strips ? kGroupWarps * p.counter_target : (p.local_pair ? 2 * kGroupWarps : kGroupWarps);
+      else if (i >= 3 * kMaxStages + 2 * kAcc + 3 * kGroups && i < 3 * kMaxStages + 2 * kAcc + 4 * kGroups)
+        count = kGroupWarps;                                                                       // gdone
+      ptx::mbar_init(&full[i], count);
     }
-    for (int i = 0; i < kGroups; ++i) {
-      ptx::mbar_init(&pfull[i], 1);
-      // (in-CTA exchange of a tile's two units: pub[g & ~1] counts the warps of both groups)
-      // (own strips: pub[0] counts the warps of all the strip's units)
-      ptx::mbar_init(&pub[i], p.own_strips ? kGroupWarps * (int)p.counter_target
-                                           : (p.local_pair ? 2 * kGroupWarps : kGroupWarps));
-      ptx::mbar_init(&ready[i], 1);
-      ptx::mbar_init(&gdone[i], kGroupWarps);
-    }
-    ptx::mbar_init(drain, 1);
-    ptx::mbar_init(wfull, 1);
-    *cta_abort = 0;
     ptx::fence_mbar_init();
-    ptx::prefetch_tensormap(&tmA);
-    ptx::prefetch_tensormap(&tmB);
-    if (C::kTmaStore) ptx::prefetch_tensormap(&tmY);
   }
   if (warp == 1) {
     ptx::tmem_alloc(tmem_slot, kTmemCols);
@@ -284,16 +322,17 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // With a grid that is a multiple of tiles_n every tile of this CTA has the same column tile: its W
         // tile is loaded once and the ring below streams X only (half the bytes per tile through the SM's
         // load port, which is what bounds short-K layers).
-        const int n0 = ((int)blockIdx.x % p.tiles_n) * BN;
+        const int n0 = ((int)blockIdx.x % p.tiles_n) * BN;      // (one modulo per call)
         ptx::mbar_arrive_expect_tx(wfull, (uint32_t)(p.res_kb * C::kBBytes));
         for (int kb = 0; kb < p.res_kb; ++kb) ptx::tma_load_2d(sWres + kb * C::kBBytes, &tmB, kb * kBK, n0, wfull);
       }
       uint32_t issued = 0, s = 0, ph = 0;
       bool ok = true;
-      for (int jt = 0; ok && jt < n_local; ++jt) {
-        const int tile = tile_of(jt);
-        const int m0 = (tile / p.tiles_n) * kBM;
-        const int n0 = (tile % p.tiles_n) * BN;
+      TileWalk walk;
+      walk.init(p, (int)blockIdx.x, G);
+      for (int jt = 0; ok && jt < n_local; ++jt, walk.advance()) {
+        const int m0 = walk.tm * kBM;
+        const int n0 = walk.tn * BN;
         for (int kb = 0; kb < p.num_kb; ++kb, ++issued) {
           if (!ptx::mbar_wait_bounded(&empty[s], ph ^ 1u, cta_abort, tmo)) {
             give_up(kStWaitEmpty);
@@ -450,12 +489,18 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const int n_units = n_local * UPT;
     float pre_fs[kUnitN / 32], pre_fb[kUnitN / 32];
 
-    auto unit_col0 = [&](int u) {           // first column of unit u in the output matrix
-      const int tile = tile_of(u / UPT);
-      return (tile % p.tiles_n) * BN + (u % UPT) * kUnitN;
+    // the group's walk over its units g, g + 4, ...: `walk` stands on the tile of the current unit, `next` on the
+    // tile of the group's next unit (for the parameter prefetch)
+    constexpr int kTileStep = kGroups / UPT;                 // tiles between two units of a group
+    TileWalk walk, next;
+    walk.init(p, (int)blockIdx.x, G);
+    walk.advance(g / UPT);
+    next = walk;
+    next.advance(kTileStep);
+    auto col0_at = [&](const TileWalk& w, int u) {           // first column of unit u (whose tile w stands on)
+      return w.tn * BN + (u % UPT) * kUnitN;
     };
-    auto prefetch_params = [&](int u) {
-      const int n0 = unit_col0(u);
+    auto prefetch_params = [&](int n0) {
 #pragma unroll
       for (int i = 0; i < kUnitN / 32; ++i) {
         const int c = n0 + i * 32 + lane;
@@ -475,8 +520,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     };
     int pre_n0 = -1;                        // lead warp: first column of the unit the prefetch registers hold
     if (C::kNeedSlice && lead && g < n_units) {
-      prefetch_params(g);
-      pre_n0 = unit_col0(g);
+      pre_n0 = col0_at(walk, g);
+      prefetch_params(pre_n0);
     }
 
     // Writes the warp's box (32 rows x BOXB bytes, swizzled in its staging slot) to global memory: lanes are
@@ -520,11 +565,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     int use = 0;                            // units this group has handled
     int slice_n0 = -1;                      // first column of the unit whose parameters are in the group's slice
     int reloads = 0;                        // times the slice has been (re)loaded
-    for (int u = g; u < n_units; u += kGroups, ++use) {
+    for (int u = g; u < n_units; u += kGroups, ++use, walk = next, next.advance(kTileStep)) {
       const int j = u / UPT;
-      const int tile = tile_of(j);
-      const int tm = tile / p.tiles_n;
-      const int n0 = unit_col0(u);
+      const int tm = walk.tm;
+      const int n0 = col0_at(walk, u);
       const uint32_t buf = j % kAcc, tpar = (j / kAcc) & 1u, upar = use & 1u;
       const int y0 = tm * kBM + qd * 32;
       const uint32_t taddr = taddr_q + buf * BN + (uint32_t)(u % UPT) * kUnitN;   // the unit's columns in TMEM
@@ -576,7 +620,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         slice_n0 = n0;
         const uint32_t ppar = (uint32_t)(reloads++) & 1u;
         if (lead) {
-          if (pre_n0 != n0) prefetch_params(u);      // not fetched ahead (never the case with a regular tile walk)
+          if (pre_n0 != n0) prefetch_params(n0);     // not fetched ahead (never the case with a regular tile walk)
           // the slice is free once the group's 4 warps have finished the unit that used it before
           if (!ptx::mbar_wait_bounded(&gdone[g], upar ^ 1u, cta_abort, tmo)) {
             give_up(kStWaitParam);
@@ -595,9 +639,9 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&pfull[g]);
-          if (u + kGroups < n_units && unit_col0(u + kGroups) != n0) {
-            prefetch_params(u + kGroups);
-            pre_n0 = unit_col0(u + kGroups);
+          if (u + kGroups < n_units && col0_at(next, u + kGroups) != n0) {
+            pre_n0 = col0_at(next, u + kGroups);
+            prefetch_params(pre_n0);
           }
         }
         if (!ptx::mbar_wait_bounded(&pfull[g], ppar, cta_abort, tmo)) {
@@ -722,9 +766,9 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         } else if (p.own_strips) {
           // the row is this CTA's two tiles of the strip: all its units (up to 4, one per group) meet in shared
           // memory (two buffers by the strip's ordinal: a group can be one strip ahead of the readers of the last)
-          const uint32_t xp = (uint32_t)(j / p.tiles_n) & 1u;
+          const uint32_t xp = (uint32_t)walk.ord & 1u;
           float* const sbuf = sPair + xp * 4 * kBM;                                   // [unit of the strip][row]
-          sbuf[(uint32_t)((tile % p.tiles_n) * UPT + u % UPT) * kBM + qd * 32 + my] = amax_mine;
+          sbuf[(uint32_t)(walk.tn * UPT + u % UPT) * kBM + qd * 32 + my] = amax_mine;
           __syncwarp();
           if (lane == 0) ptx::mbar_arrive(&pub[0]);
           if (!ptx::mbar_wait_bounded(&pub[0], xp, cta_abort, tmo)) {
@@ -1402,6 +1446,18 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   prm.tiles_n = plan.tiles_n;
   prm.num_tiles = plan.tiles_m * plan.tiles_n;
   prm.num_kb = (K + kBK - 1) / kBK;
+  if (plan.own_strips) {       // strips b, b + G, ...: every CTA takes tiles_n tiles of each of its strips
+    prm.nl_base = plan.tiles_m / plan.grid;
+    prm.nl_rem = plan.tiles_m % plan.grid;
+    prm.nl_mul = plan.tiles_n;
+    prm.step_q = prm.step_r = 0;
+  } else {                     // tiles b, b + G, ...
+    prm.nl_base = prm.num_tiles / plan.grid;
+    prm.nl_rem = prm.num_tiles % plan.grid;
+    prm.nl_mul = 1;
+    prm.step_q = plan.grid / plan.tiles_n;
+    prm.step_r = plan.grid % plan.tiles_n;
+  }
   prm.status = reinterpret_cast<uint32_t*>(ws + plan.ws_status_off);
   prm.partial = reinterpret_cast<unsigned long long*>(ws + plan.ws_partial_off);
   // units of a row strip that lie inside the matrix
