@@ -111,8 +111,11 @@ struct QlParams {
 };
 
 // Compile-time geometry of one instantiation.
-template <int BN, int OUT, bool W4, bool WIDE, bool ASYM = false>
+template <int BN, int OUT, bool W4, bool WIDE, bool ASYM = false, bool PAIR = false>
 struct Cfg {
+  // PAIR: two CTAs of a cluster work on two row strips of the same column tile; the even CTA issues MMAs of
+  // M = 256 (tcgen05 cta_group::2) that take the A tile and half of the W tile from each CTA's shared memory
+  static_assert(!PAIR || (!W4 && !ASYM && OUT != kOutCalibStats && BN == 256), "CTA pairs: int8 weights, 256-wide tiles");
   static constexpr bool kInt8Out = OUT == QWT_OUT_INT8_PER_TOKEN;     // dynamic per-token scale: two-phase epilogue
   static constexpr bool kStatic8 = OUT == QWT_OUT_INT8_STATIC;       // Eq. 10 as printed: static multiplier + offset
   static constexpr bool kCodes = kInt8Out || kStatic8;               // one byte per output element
@@ -134,7 +137,8 @@ struct Cfg {
   static constexpr int kBC = kBoxBytes / kEsz;                       // columns per box
   static constexpr int kSlotBytes = 32 * kBoxBytes;
   static constexpr int kStagingBytes = kEpiWarps * kSlotBytes;
-  static constexpr int kBBytes = BN * kBK;                           // expanded (int8) W tile of one stage
+  static constexpr int kBRows = PAIR ? BN / 2 : BN;                   // rows of the W tile this CTA loads
+  static constexpr int kBBytes = kBRows * kBK;                       // expanded (int8) W tile of one stage
   static constexpr int kPBytes = W4 ? BN * (kBK / 2) : 0;            // packed (int4) W tile of one stage
   static constexpr int kStageBytes = kABytes + kBBytes + kPBytes;
   // per group and unit: fscale | fbias, and with asymmetric codes also the two integer column terms of Eq. 7
@@ -231,11 +235,11 @@ struct TileWalk {
   }
 };
 
-template <int BN, int OUT, bool W4, bool WIDE, bool ASYM>
-__global__ void __launch_bounds__((Cfg<BN, OUT, W4, WIDE, ASYM>::kThreads), 1)
+template <int BN, int OUT, bool W4, bool WIDE, bool ASYM, bool PAIR>
+__global__ void __launch_bounds__((Cfg<BN, OUT, W4, WIDE, ASYM, PAIR>::kThreads), 1)
 qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmY, const QlParams p) {
-  using C = Cfg<BN, OUT, W4, WIDE, ASYM>;
+  using C = Cfg<BN, OUT, W4, WIDE, ASYM, PAIR>;
   constexpr int kAcc = C::kAcc;
   constexpr int kMaxStages = C::kMaxStages;
   const int stages = p.stages;
@@ -267,11 +271,15 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   const int warp = threadIdx.x >> 5;
   const int lane = threadIdx.x & 31;
   const uint64_t tmo = p.timeout_ns;
-  const int G = (int)gridDim.x;
+  // CTA pairs: the pair is the unit of the tile walk; this CTA's row strip is 2 * (the walk's strip) + its rank
+  const uint32_t rank = PAIR ? ptx::cluster_ctarank() : 0u;
+  const int G = PAIR ? (int)(gridDim.x >> 1) : (int)gridDim.x;
+  const int walker = PAIR ? (int)(blockIdx.x >> 1) : (int)blockIdx.x;      // index of this CTA (pair) in the walk
+  auto strip_of = [&](int walk_tm) { return PAIR ? 2 * walk_tm + (int)rank : walk_tm; };
   // Tiles of this CTA, in the order it takes them.  Default: b, b + G, b + 2G, ...  With own strips (per-token INT8
   // whose rows span exactly two column tiles): the strips b, b + G, ... and both column tiles of each in turn, so
   // that a row's maxima never leave the CTA.
-  const int n_local = p.nl_mul * (p.nl_base + ((int)blockIdx.x < p.nl_rem ? 1 : 0));
+  const int n_local = p.nl_mul * (p.nl_base + (walker < p.nl_rem ? 1 : 0));
 
   if (warp == 0) {
     // the barriers lie one after the other in shared memory; the lanes of warp 0 initialise them side by side
@@ -285,7 +293,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     for (int i = lane; i < C::kNumBars; i += 32) {
       uint32_t count = 1;                                            // full, empty, tfull, pfull, ready, drain, wfull
       if (i >= 2 * kMaxStages && i < 3 * kMaxStages) count = kNumConvWarps;                       // conv
-      else if (i >= 3 * kMaxStages + kAcc && i < 3 * kMaxStages + 2 * kAcc) count = kGroupWarps * C::kUPT;   // tempty
+      else if (i >= 3 * kMaxStages + kAcc && i < 3 * kMaxStages + 2 * kAcc)
+        count = kGroupWarps * C::kUPT * (PAIR ? 2 : 1);              // tempty (pairs: the warps of both CTAs)
       else if (i >= 3 * kMaxStages + 2 * kAcc + kGroups && i < 3 * kMaxStages + 2 * kAcc + 2 * kGroups)
         // pub (in-CTA exchange of a tile's two units: pub[g & ~1] counts the warps of both groups; own strips:
         // pub[0] counts the warps of all the strip's units)
@@ -297,11 +306,20 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     ptx::fence_mbar_init();
   }
   if (warp == 1) {
-    ptx::tmem_alloc(tmem_slot, kTmemCols);
-    ptx::tmem_relinquish();
+    if (PAIR) {
+      ptx::tmem_alloc_pair(tmem_slot, kTmemCols);
+      ptx::tmem_relinquish_pair();
+    } else {
+      ptx::tmem_alloc(tmem_slot, kTmemCols);
+      ptx::tmem_relinquish();
+    }
   }
   ptx::tc_fence_before();
   __syncthreads();
+  if (PAIR) {       // the peer's barriers must exist before anything of this CTA signals them
+    ptx::cluster_arrive();
+    ptx::cluster_wait();
+  }
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
 
@@ -312,6 +330,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
   auto give_up = [&](uint32_t code) {
     *cta_abort = 1;
+    if (PAIR) ptx::st_shared_cluster_u32(ptx::mapa_shared(ptx::smem_u32(const_cast<int*>(cta_abort)), rank ^ 1u), 1u);
     atomicCAS(p.status, 0u, code);
   };
 
@@ -329,9 +348,9 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       uint32_t issued = 0, s = 0, ph = 0;
       bool ok = true;
       TileWalk walk;
-      walk.init(p, (int)blockIdx.x, G);
+      walk.init(p, walker, G);
       for (int jt = 0; ok && jt < n_local; ++jt, walk.advance()) {
-        const int m0 = walk.tm * kBM;
+        const int m0 = strip_of(walk.tm) * kBM;
         const int n0 = walk.tn * BN;
         for (int kb = 0; kb < p.num_kb; ++kb, ++issued) {
           if (!ptx::mbar_wait_bounded(&empty[s], ph ^ 1u, cta_abort, tmo)) {
@@ -339,7 +358,13 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             ok = false;
             break;
           }
-          if (resident) {
+          if (PAIR) {
+            // both CTAs' loads of the stage are counted on the even CTA's barrier, where the MMAs are issued
+            const uint32_t lead_full = ptx::mapa_shared(ptx::smem_u32(&full[s]), 0u);
+            if (rank == 0u) ptx::mbar_arrive_expect_tx(&full[s], 2u * (kABytes + C::kBBytes));
+            ptx::tma_load_2d_pair(sA + s * kABytes, &tmA, kb * kBK, m0, lead_full);
+            ptx::tma_load_2d_pair(sB + s * C::kBBytes, &tmB, kb * kBK, n0 + (int)rank * C::kBRows, lead_full);
+          } else if (resident) {
             ptx::mbar_arrive_expect_tx(&full[s], kABytes);
             ptx::tma_load_2d(sA + s * kABytes, &tmA, kb * kBK, m0, &full[s]);
           } else {
@@ -354,8 +379,9 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
       }
-      if (*cta_abort != 0) {
-        // let copies still in flight land before the CTA's shared memory is released
+      if (*cta_abort != 0 && rank == 0u) {
+        // let copies still in flight land before the CTA's shared memory is released (pairs: the even CTA's
+        // barriers count the loads of both, and the odd CTA stays until the pair's final synchronisation)
         const uint32_t back = issued < (uint32_t)stages ? issued : (uint32_t)stages;
         for (uint32_t j = 0; j < back; ++j) {
           // walk back over the last `back` issues: stage and phase of issue number issued - 1 - j
@@ -373,8 +399,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
   } else if (warp == 1) {
     // ------------------------------------------------------------------ MMA issuer
-    if (lane == 0) {
-      constexpr uint32_t idesc = ASYM ? ptx::make_idesc_u8(kBM, BN) : ptx::make_idesc_i8(kBM, BN);
+    if (lane == 0 && rank == 0u) {
+      constexpr uint32_t idesc = ASYM ? ptx::make_idesc_u8(kBM, BN) : ptx::make_idesc_i8(PAIR ? 2 * kBM : kBM, BN);
       const uint32_t a_base = ptx::smem_u32(sA), b_base = ptx::smem_u32(sB), w_base = ptx::smem_u32(sWres);
       uint32_t s = 0, ph = 0, it = 0;
       bool ok = true;
@@ -402,19 +428,25 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
           for (int k = 0; k < kBK / kUmmaK; ++k) {
             // next 32 bytes of K inside the swizzled 128-byte row: start address + 32 B (>> 4 = 2)
-            ptx::mma_i8_ss(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            if (PAIR) ptx::mma_i8_ss_pair(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+            else ptx::mma_i8_ss(d_tmem, a_desc + 2 * k, b_desc + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
           }
-          ptx::tc_commit(&empty[s]);
+          if (PAIR) ptx::tc_commit_pair_mc(&empty[s], 3);     // the stage is free in both CTAs
+          else ptx::tc_commit(&empty[s]);
           if (++s == (uint32_t)stages) {
             s = 0;
             ph ^= 1u;
           }
         }
-        if (ok) ptx::tc_commit(&tfull[buf]);
+        if (ok) {
+          if (PAIR) ptx::tc_commit_pair_mc(&tfull[buf], 3);   // the accumulator is complete in both CTAs
+          else ptx::tc_commit(&tfull[buf]);
+        }
       }
       if (*cta_abort != 0) {
         // make sure no MMA is still running when TMEM is released
-        ptx::tc_commit(drain);
+        if (PAIR) ptx::tc_commit_pair(drain);
+        else ptx::tc_commit(drain);
         uint32_t polls = 0;
         while (!ptx::mbar_try_wait(drain, 0) && ++polls < (1u << 16)) {
         }
@@ -493,7 +525,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // tile of the group's next unit (for the parameter prefetch)
     constexpr int kTileStep = kGroups / UPT;                 // tiles between two units of a group
     TileWalk walk, next;
-    walk.init(p, (int)blockIdx.x, G);
+    walk.init(p, walker, G);
     walk.advance(g / UPT);
     next = walk;
     next.advance(kTileStep);
@@ -567,7 +599,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     int reloads = 0;                        // times the slice has been (re)loaded
     for (int u = g; u < n_units; u += kGroups, ++use, walk = next, next.advance(kTileStep)) {
       const int j = u / UPT;
-      const int tm = walk.tm;
+      const int tm = strip_of(walk.tm);
       const int n0 = col0_at(walk, u);
       const uint32_t buf = j % kAcc, tpar = (j / kAcc) & 1u, upar = use & 1u;
       const int y0 = tm * kBM + qd * 32;
@@ -660,7 +692,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const int q = lane >> 2, c = lane & 3;
       const float2 xs2[4] = {make_float2(xs4[0], xs4[0]), make_float2(xs4[1], xs4[1]), make_float2(xs4[2], xs4[2]),
                              make_float2(xs4[3], xs4[3])};
-      const bool in_range = n0 < p.N;        // a unit entirely right of the matrix has nothing to compute or store
+      // a unit entirely right of the matrix (or, for the odd CTA of a pair, below it) has nothing to compute or store
+      const bool in_range = n0 < p.N && (!PAIR || tm * kBM < p.M);
       // z of one 8-column block for the thread's four rows; a = registers of lanes q, q + 8 (half 0) and of
       // lanes q + 16, q + 24 (half 1); col = first column of the block inside the unit
       // Eq. 7: the unsigned product plus the three zero-point terms, for the block's two columns and four rows
@@ -704,7 +737,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       auto release_acc = [&]() {
         ptx::tc_fence_before();
         __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&tempty[buf]);
+        if (lane == 0) {
+          if (PAIR) ptx::mbar_arrive_cluster(ptx::mapa_shared(ptx::smem_u32(&tempty[buf]), 0u));   // the even CTA issues the MMAs
+          else ptx::mbar_arrive(&tempty[buf]);
+        }
         released = true;
       };
       const int boxes_in = in_range ? ((p.N - n0 + BC - 1) / BC < kUnitN / BC ? (p.N - n0 + BC - 1) / BC : kUnitN / BC) : 0;
@@ -1160,9 +1196,14 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   __syncwarp();
   ptx::tc_fence_before();
   __syncthreads();
+  if (PAIR) {       // neither CTA leaves (or frees tensor memory) while the other may still signal it or read its tiles
+    ptx::cluster_arrive();
+    ptx::cluster_wait();
+  }
   if (warp == 1) {
     ptx::tc_fence_after();
-    ptx::tmem_dealloc(tmem_base, kTmemCols);
+    if (PAIR) ptx::tmem_dealloc_pair(tmem_base, kTmemCols);
+    else ptx::tmem_dealloc(tmem_base, kTmemCols);
   }
 }
 
@@ -1215,12 +1256,12 @@ unsigned long long timeout_ns_from_env() {
   return v;
 }
 
-template <int BN, int OUT, bool W4, bool WIDE, bool ASYM = false>
+template <int BN, int OUT, bool W4, bool WIDE, bool ASYM = false, bool PAIR = false>
 qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams prm, int grid, int res_kb,
                       cudaStream_t st) {
-  using C = Cfg<BN, OUT, W4, WIDE, ASYM>;
+  using C = Cfg<BN, OUT, W4, WIDE, ASYM, PAIR>;
   constexpr int kThreads = C::kThreads;
-  auto kern = qlinear_cwac_kernel<BN, OUT, W4, WIDE, ASYM>;
+  auto kern = qlinear_cwac_kernel<BN, OUT, W4, WIDE, ASYM, PAIR>;
   // output map: Y as a byte matrix, one staging box (32 rows x kBoxBytes, in the box's own swizzle) per copy
   CUtensorMap tmY = tmA;
   if (C::kTmaStore) {
@@ -1243,7 +1284,26 @@ qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams p
     QWT_CUDA_TRY(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448));
     if (dev >= 0 && dev < 64) attr_set[dev].store(true, std::memory_order_release);
   }
-  if (C::kInt8Out && prm.counter_target > 1u && !prm.local_pair && !prm.own_strips) {
+  const bool cooperative = C::kInt8Out && prm.counter_target > 1u && !prm.local_pair && !prm.own_strips;
+  if (PAIR) {
+    // clusters of two CTAs (and, for the row-maximum exchange, every CTA of the grid resident)
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attrs[2];
+    attrs[0].id = cudaLaunchAttributeClusterDimension;
+    attrs[0].val.clusterDim.x = 2;
+    attrs[0].val.clusterDim.y = 1;
+    attrs[0].val.clusterDim.z = 1;
+    attrs[1].id = cudaLaunchAttributeCooperative;
+    attrs[1].val.cooperative = 1;
+    cfg.attrs = attrs;
+    cfg.numAttrs = cooperative ? 2 : 1;
+    QWT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmY, prm));
+    count_launch();
+  } else if (cooperative) {
     // the row-maximum exchange needs every CTA of the grid resident
     void* args[] = {(void*)&tmA, (void*)&tmB, (void*)&tmY, (void*)&prm};
     QWT_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, smem_bytes, st));
@@ -1259,7 +1319,10 @@ qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams p
 // asks for it and at least 4 X stages remain, else the streaming layout.
 template <int BN, int OUT, bool W4>
 qwt_status launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
-                       bool want_resident, cudaStream_t st) {
+                       bool want_resident, bool pair, cudaStream_t st) {
+  if constexpr (!W4 && BN == 256 && OUT != kOutCalibStats) {
+    if (pair) return launch_cfg<BN, OUT, false, false, false, true>(tmA, tmB, prm, grid, 0, st);
+  }
   if (!W4) {
     constexpr bool kWide = BN == 256;
     using CW = Cfg<BN, OUT, false, kWide>;
@@ -1288,26 +1351,26 @@ qwt_status launch_asym(int out_mode, const CUtensorMap& tmA, const CUtensorMap& 
 
 template <int BN, bool W4>
 qwt_status launch_bn(int out_mode, const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
-                     bool want_resident, cudaStream_t st) {
+                     bool want_resident, bool pair, cudaStream_t st) {
   if (prm.w_terms != nullptr) {
     if (W4) return QWT_ERR_UNSUPPORTED;
     return launch_asym<BN>(out_mode, tmA, tmB, prm, grid, st);
   }
   switch (out_mode) {
     case QWT_OUT_INT8_PER_TOKEN:
-      return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN, W4>(tmA, tmB, prm, grid, want_resident, st);
+      return launch_inst<BN, QWT_OUT_INT8_PER_TOKEN, W4>(tmA, tmB, prm, grid, want_resident, pair, st);
     case QWT_OUT_BF16:
-      return launch_inst<BN, QWT_OUT_BF16, W4>(tmA, tmB, prm, grid, want_resident, st);
+      return launch_inst<BN, QWT_OUT_BF16, W4>(tmA, tmB, prm, grid, want_resident, pair, st);
     case QWT_OUT_FP32:
-      return launch_inst<BN, QWT_OUT_FP32, W4>(tmA, tmB, prm, grid, want_resident, st);
+      return launch_inst<BN, QWT_OUT_FP32, W4>(tmA, tmB, prm, grid, want_resident, pair, st);
     case QWT_OUT_INT32_ACC:
-      return launch_inst<BN, QWT_OUT_INT32_ACC, W4>(tmA, tmB, prm, grid, want_resident, st);
+      return launch_inst<BN, QWT_OUT_INT32_ACC, W4>(tmA, tmB, prm, grid, want_resident, pair, st);
     case QWT_OUT_INT8_STATIC:
-      return launch_inst<BN, QWT_OUT_INT8_STATIC, W4>(tmA, tmB, prm, grid, want_resident, st);
+      return launch_inst<BN, QWT_OUT_INT8_STATIC, W4>(tmA, tmB, prm, grid, want_resident, pair, st);
     case kOutCalibStats:
       // packed weights with 256-wide tiles leave no room for the per-warp sums: the plan picks 128 there
       if constexpr (W4 && BN == 256) return QWT_ERR_UNSUPPORTED;
-      else return launch_inst<BN, kOutCalibStats, W4>(tmA, tmB, prm, grid, want_resident, st);
+      else return launch_inst<BN, kOutCalibStats, W4>(tmA, tmB, prm, grid, want_resident, false, st);
   }
   return QWT_ERR_UNSUPPORTED;
 }
@@ -1374,7 +1437,22 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
       pl.grid = pl.tiles_m < sms ? pl.tiles_m : sms;
     }
   }
-  pl.fused_requant = (out_mode == QWT_OUT_INT8_PER_TOKEN) && (pl.tiles_n <= pl.grid);
+  // Long K, 256-wide tiles, int8 weights: CTA pairs (clusters of two) on two row strips of the same column tile, the
+  // MMAs of M = 256 issued by the even CTA; each CTA then loads half of the W tile per k-block (a third less through
+  // its load port and out of its shared memory per MMA), which is what the mainloop of the long-K layers waits for.
+  {
+    const char* e = getenv("QWT_PAIR");
+    const int pair_tiles = ((pl.tiles_m + 1) / 2) * pl.tiles_n;
+    const int pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
+    const bool fits = !w4 && pl.bn == 256 && !pl.w_resident && !pl.own_strips && out_mode != kOutCalibStats &&
+                      pl.tiles_m >= 2 && pl.tiles_n <= pairs;
+    // (measured: ahead by up to 7 % on layers 4096 and 11008 wide with K = 4096 and 11008, behind by 4 % on a layer
+    // 768 wide with K = 3072, whose three column tiles leave the pairs little to share)
+    const bool want = e != nullptr ? e[0] == '1' : (K >= 2048 && pl.tiles_n >= 8 && pair_tiles >= sms / 2);
+    pl.pair = fits && want;
+    if (pl.pair) pl.grid = 2 * pairs;
+  }
+  pl.fused_requant = (out_mode == QWT_OUT_INT8_PER_TOKEN) && (pl.tiles_n <= (pl.pair ? pl.grid / 2 : pl.grid));
   size_t off = 0;
   pl.ws_status_off = off;
   off += 256;
@@ -1418,9 +1496,11 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   const bool w4 = wfmt == QWT_W_INT4_PACKED;
   CUtensorMap tmA, tmB;
   const bool okA = make_byte_map(&tmA, X, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+  // (asymmetric codes and the statistics epilogue have no pair instantiation: the same grid then walks single tiles)
+  const bool pair = plan.pair && w_terms == nullptr && stats == nullptr && !w4;
   const bool okB = w4 ? make_byte_map(&tmB, W, (uint64_t)N, (uint64_t)K / 2, kBK / 2, (uint32_t)plan.bn,
                                       CU_TENSOR_MAP_SWIZZLE_NONE)
-                      : make_byte_map(&tmB, W, (uint64_t)N, (uint64_t)K, kBK, (uint32_t)plan.bn,
+                      : make_byte_map(&tmB, W, (uint64_t)N, (uint64_t)K, kBK, (uint32_t)(pair ? plan.bn / 2 : plan.bn),
                                       CU_TENSOR_MAP_SWIZZLE_128B);
   if (!okA || !okB) {
     set_cuda_error((int)cudaErrorInvalidValue);
@@ -1451,6 +1531,13 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
     prm.nl_rem = plan.tiles_m % plan.grid;
     prm.nl_mul = plan.tiles_n;
     prm.step_q = prm.step_r = 0;
+  } else if (pair) {           // pairs of CTAs take pair tiles (two row strips x one column tile) b, b + G / 2, ...
+    const int pair_tiles = ((plan.tiles_m + 1) / 2) * plan.tiles_n, pairs = plan.grid / 2;
+    prm.nl_base = pair_tiles / pairs;
+    prm.nl_rem = pair_tiles % pairs;
+    prm.nl_mul = 1;
+    prm.step_q = pairs / plan.tiles_n;
+    prm.step_r = pairs % plan.tiles_n;
   } else {                     // tiles b, b + G, ...
     prm.nl_base = prm.num_tiles / plan.grid;
     prm.nl_rem = prm.num_tiles % plan.grid;
@@ -1487,10 +1574,10 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
     prm.Y = ws + plan.ws_z_off;
   }
   qwt_status s;
-  if (w4) s = plan.bn == 256 ? launch_bn<256, true>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, st)
-                             : launch_bn<128, true>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, st);
-  else s = plan.bn == 256 ? launch_bn<256, false>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, st)
-                          : launch_bn<128, false>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, st);
+  if (w4) s = plan.bn == 256 ? launch_bn<256, true>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, false, st)
+                             : launch_bn<128, true>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, false, st);
+  else s = plan.bn == 256 ? launch_bn<256, false>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, pair, st)
+                          : launch_bn<128, false>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, false, st);
   if (s != QWT_OK) return s;
   if (mode != out_mode)
     return launch_quantize_rows(reinterpret_cast<const float*>(ws + plan.ws_z_off), M, N, N, 127,

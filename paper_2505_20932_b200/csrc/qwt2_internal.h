@@ -110,6 +110,7 @@ struct QlinearPlan {
   int strip_units;       // 128-column units of a row strip (whose row maxima the per-token INT8 exchange waits for)
   bool w_resident;       // grid is a multiple of tiles_n: a CTA's W tile can stay in shared memory
   bool own_strips;       // per-token INT8 with two column tiles per strip: a CTA takes whole strips
+  bool pair;             // CTA pairs (clusters of two, MMAs of M = 256 issued by the even CTA); the grid is even
   bool w4_expand;        // packed int4 weights are expanded to int8 in the workspace first (many rows: the GEMM is
                          // compute-bound and the int8 mainloop is twice as fast as the one that converts on chip)
   size_t ws_status_off, ws_partial_off, ws_z_off, ws_w_off, ws_total;

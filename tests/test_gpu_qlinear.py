@@ -363,3 +363,23 @@ def test_w4_both_weight_paths(H, B, M, N, K, expand, monkeypatch):
     c_ref, ys_ref = O.requant_per_token(O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb))
     assert np.allclose(ys, ys_ref, rtol=1e-5)
     assert_codes_close(codes, c_ref)
+
+
+@pytest.mark.parametrize("M,N,K", [(300, 528, 1040), (256, 256, 128), (128 * 5 + 7, 1024, 400), (3000, 2304, 512)])
+def test_cta_pairs_every_output_stage(H, B, M, N, K, monkeypatch):
+    """Clusters of two CTAs with MMAs of M = 256 (tcgen05 cta_group::2), forced on for small ragged layers: an odd
+    number of row strips (the odd CTA of the last pair then has no rows), N and K tails, several tiles per pair."""
+    monkeypatch.setenv("QWT_PAIR", "1")
+    Xq, Wq, xs, fs, fb = random_layer(M, N, K, seed=M + N + K + 5)
+    acc_ref = O.int_matmul(Xq, Wq)
+    z_ref = O.forward_folded(acc_ref, xs, fs, fb)
+    acc, _ = H.gpu_forward(Xq, None, Wq, None, None, B.QWT_OUT_INT32_ACC)
+    assert np.array_equal(acc.astype(np.int64), acc_ref)
+    z, _ = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_FP32)
+    assert_fp32_close(z, z_ref)
+    bits, _ = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_BF16)
+    assert_bf16_close(bits, z_ref, O.to_bf16_bits, O.bf16_bits_to_f32)
+    codes, ys = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_INT8_PER_TOKEN)
+    c_ref, ys_ref = O.requant_per_token(z_ref)
+    assert np.allclose(ys, ys_ref, rtol=1e-5, atol=0)
+    assert_codes_close(codes, c_ref)
