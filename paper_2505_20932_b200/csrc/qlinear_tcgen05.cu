@@ -115,7 +115,7 @@ template <int BN, int OUT, bool W4, bool WIDE, bool ASYM = false, bool PAIR = fa
 struct Cfg {
   // PAIR: two CTAs of a cluster work on two row strips of the same column tile; the even CTA issues MMAs of
   // M = 256 (tcgen05 cta_group::2) that take the A tile and half of the W tile from each CTA's shared memory
-  static_assert(!PAIR || (!W4 && !ASYM && OUT != kOutCalibStats && BN == 256), "CTA pairs: int8 weights, 256-wide tiles");
+  static_assert(!PAIR || (!ASYM && OUT != kOutCalibStats && BN == 256), "CTA pairs: symmetric codes, 256-wide tiles");
   static constexpr bool kInt8Out = OUT == QWT_OUT_INT8_PER_TOKEN;     // dynamic per-token scale: two-phase epilogue
   static constexpr bool kStatic8 = OUT == QWT_OUT_INT8_STATIC;       // Eq. 10 as printed: static multiplier + offset
   static constexpr bool kCodes = kInt8Out || kStatic8;               // one byte per output element
@@ -139,7 +139,7 @@ struct Cfg {
   static constexpr int kStagingBytes = kEpiWarps * kSlotBytes;
   static constexpr int kBRows = PAIR ? BN / 2 : BN;                   // rows of the W tile this CTA loads
   static constexpr int kBBytes = kBRows * kBK;                       // expanded (int8) W tile of one stage
-  static constexpr int kPBytes = W4 ? BN * (kBK / 2) : 0;            // packed (int4) W tile of one stage
+  static constexpr int kPBytes = W4 ? kBRows * (kBK / 2) : 0;        // packed (int4) W tile of one stage
   static constexpr int kStageBytes = kABytes + kBBytes + kPBytes;
   // per group and unit: fscale | fbias, and with asymmetric codes also the two integer column terms of Eq. 7
   static constexpr int kParamArrays = ASYM ? 4 : 2;
@@ -292,7 +292,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
     for (int i = lane; i < C::kNumBars; i += 32) {
       uint32_t count = 1;                                            // full, empty, tfull, pfull, ready, drain, wfull
-      if (i >= 2 * kMaxStages && i < 3 * kMaxStages) count = kNumConvWarps;                       // conv
+      if (i >= 2 * kMaxStages && i < 3 * kMaxStages) count = (kNumConvWarps / 2) * (PAIR ? 2 : 1);   // conv: a team
       else if (i >= 3 * kMaxStages + kAcc && i < 3 * kMaxStages + 2 * kAcc)
         count = kGroupWarps * C::kUPT * (PAIR ? 2 : 1);              // tempty (pairs: the warps of both CTAs)
       else if (i >= 3 * kMaxStages + 2 * kAcc + kGroups && i < 3 * kMaxStages + 2 * kAcc + 2 * kGroups)
@@ -358,7 +358,13 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             ok = false;
             break;
           }
-          if (PAIR) {
+          if (PAIR && W4) {
+            // packed weights: a CTA's loads are counted on its own barrier, for its own converter warps, which then
+            // report to the even CTA
+            ptx::mbar_arrive_expect_tx(&full[s], kABytes + C::kPBytes);
+            ptx::tma_load_2d(sA + s * kABytes, &tmA, kb * kBK, m0, &full[s]);
+            ptx::tma_load_2d(sP + s * C::kPBytes, &tmB, kb * (kBK / 2), n0 + (int)rank * C::kBRows, &full[s]);
+          } else if (PAIR) {
             // both CTAs' loads of the stage are counted on the even CTA's barrier, where the MMAs are issued
             const uint32_t lead_full = ptx::mapa_shared(ptx::smem_u32(&full[s]), 0u);
             if (rank == 0u) ptx::mbar_arrive_expect_tx(&full[s], 2u * (kABytes + C::kBBytes));
@@ -379,7 +385,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
       }
-      if (*cta_abort != 0 && rank == 0u) {
+      if (*cta_abort != 0 && (rank == 0u || W4)) {
         // let copies still in flight land before the CTA's shared memory is released (pairs: the even CTA's
         // barriers count the loads of both, and the odd CTA stays until the pair's final synchronisation)
         const uint32_t back = issued < (uint32_t)stages ? issued : (uint32_t)stages;
@@ -458,43 +464,51 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // 128-byte-swizzled operand tile the MMA descriptor expects.  Each nibble is moved to the HIGH half of
     // its byte, i.e. the operand holds 16 x code (|16 code| <= 112 fits int8); the factor 1/16 is exact in
     // the epilogue (fscale / 16, or an arithmetic shift of the raw accumulators).
-    const int ct = threadIdx.x - C::kConvWarp0 * 32;       // 0..127
-    uint32_t s = 0, ph = 0;
-    bool ok = true;
-    for (int jt = 0; ok && jt < n_local; ++jt) {
-      for (int kb = 0; kb < p.num_kb; ++kb) {
-        if (!ptx::mbar_wait_bounded(&full[s], ph, cta_abort, tmo)) {
-          give_up(kStWaitFull);
-          ok = false;
-          break;
-        }
-        const uint8_t* src = sP + s * C::kPBytes;
-        uint8_t* dst = sB + s * C::kBBytes;
+    // Two teams of two warps take the k-blocks alternately, so that two stages are being expanded at any time: a
+    // team's pass over a stage is mostly latency (the wait for the load, the shared-memory round trip, the proxy
+    // fence), which the other team's pass covers.
+    constexpr int kTeams = 2, kTeamThreads = 32 * kNumConvWarps / kTeams;
+    const int cw = warp - C::kConvWarp0;
+    const int team = cw / (kNumConvWarps / kTeams);
+    const int lt = threadIdx.x - (C::kConvWarp0 + team * (kNumConvWarps / kTeams)) * 32;       // 0..63 inside the team
+    uint32_t s = (uint32_t)team, ph = 0;                   // (the ring has at least three stages)
+    const int total_kb = n_local * p.num_kb;
+    for (int n = team; n < total_kb; n += kTeams) {
+      if (!ptx::mbar_wait_bounded(&full[s], ph, cta_abort, tmo)) {
+        give_up(kStWaitFull);
+        break;
+      }
+      const uint8_t* src = sP + s * C::kPBytes;
+      uint8_t* dst = sB + s * C::kBBytes;
+#pragma unroll 4
+      for (int q = lt; q < C::kBRows * 4; q += kTeamThreads) {
+        const int n_row = q >> 2, c = q & 3;               // row of the tile, 16-byte chunk of the packed row
+        const uint4 w = *reinterpret_cast<const uint4*>(src + n_row * 64 + c * 16);
+        const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+        uint32_t out[8];
 #pragma unroll
-        for (int q = ct; q < BN * 4; q += 32 * kNumConvWarps) {
-          const int n = q >> 2, c = q & 3;                 // row of the tile, 16-byte chunk of the packed row
-          const uint4 w = *reinterpret_cast<const uint4*>(src + n * 64 + c * 16);
-          const uint32_t in[4] = {w.x, w.y, w.z, w.w};
-          uint32_t out[8];
-#pragma unroll
-          for (int i = 0; i < 4; ++i) {
-            const uint32_t lo = (in[i] << 4) & 0xF0F0F0F0u;   // even elements, nibble in the high half
-            const uint32_t hi = in[i] & 0xF0F0F0F0u;          // odd elements
-            out[2 * i] = __byte_perm(lo, hi, 0x5140);         // e0 e1 e2 e3
-            out[2 * i + 1] = __byte_perm(lo, hi, 0x7362);     // e4 e5 e6 e7
-          }
-          uint8_t* row = dst + n * 128;
-          const int sw = n & 7;                              // 128-byte swizzle: chunk ^= row % 8
-          *reinterpret_cast<uint4*>(row + (((2 * c) ^ sw) << 4)) = make_uint4(out[0], out[1], out[2], out[3]);
-          *reinterpret_cast<uint4*>(row + (((2 * c + 1) ^ sw) << 4)) = make_uint4(out[4], out[5], out[6], out[7]);
+        for (int i = 0; i < 4; ++i) {
+          const uint32_t lo = (in[i] << 4) & 0xF0F0F0F0u;   // even elements, nibble in the high half
+          const uint32_t hi = in[i] & 0xF0F0F0F0u;          // odd elements
+          out[2 * i] = __byte_perm(lo, hi, 0x5140);         // e0 e1 e2 e3
+          out[2 * i + 1] = __byte_perm(lo, hi, 0x7362);     // e4 e5 e6 e7
         }
-        ptx::fence_proxy_async_smem();     // generic-proxy writes -> visible to the tensor core's async proxy
-        __syncwarp();
-        if (lane == 0) ptx::mbar_arrive(&conv[s]);
-        if (++s == (uint32_t)stages) {
-          s = 0;
-          ph ^= 1u;
-        }
+        uint8_t* row = dst + n_row * 128;
+        const int sw = n_row & 7;                            // 128-byte swizzle: chunk ^= row % 8
+        *reinterpret_cast<uint4*>(row + (((2 * c) ^ sw) << 4)) = make_uint4(out[0], out[1], out[2], out[3]);
+        *reinterpret_cast<uint4*>(row + (((2 * c + 1) ^ sw) << 4)) = make_uint4(out[4], out[5], out[6], out[7]);
+      }
+      ptx::fence_proxy_async_smem();     // generic-proxy writes -> visible to the tensor core's async proxy
+      __syncwarp();
+      if (lane == 0) {
+        // (pairs: the MMAs are issued by the even CTA, which reads this CTA's tiles as well)
+        if (PAIR) ptx::mbar_arrive_cluster(ptx::mapa_shared(ptx::smem_u32(&conv[s]), 0u));
+        else ptx::mbar_arrive(&conv[s]);
+      }
+      s += kTeams;
+      if (s >= (uint32_t)stages) {
+        s -= (uint32_t)stages;
+        ph ^= 1u;
       }
     }
   } else {
@@ -1106,10 +1120,21 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           auto stage_at = [&](int r, int b) -> uint8_t* {
             return stg + r * BOXB + ((((uint32_t)b >> 4) ^ swizzle_xor<BOXB>(r)) << 4) + (b & 15);
           };
+          // The thread's stores into the staging slot (bulk-store modes): for its row q + 8k and its column pair of an
+          // 8-column block whose bytes start at a multiple of 16, the swizzled address is a per-thread constant XOR the
+          // block's 16-byte chunk index -- one instruction per store instead of the whole swizzle arithmetic.
+          uint32_t pre[4];
+          {
+            const uint32_t cb = (uint32_t)(2 * c * C::kEsz);          // byte offset of the column pair inside a block
+#pragma unroll
+            for (int k = 0; k < 4; ++k)
+              pre[k] = ptx::smem_u32(stg) + (uint32_t)(q + 8 * k) * BOXB + (((cb >> 4) ^ swizzle_xor<BOXB>(q + 8 * k)) << 4) +
+                       (cb & 15u);
+          }
 #pragma unroll 1
           for (int bx = 0; bx < kUnitN / BC; ++bx) {
             if (n0 + bx * BC >= p.N) break;
-#pragma unroll 1
+#pragma unroll
             for (int h = 0; h < BC / LDC; ++h) {
               const int c0 = bx * BC + h * LDC;         // first column (inside the unit) of this pair of loads
               uint32_t a0[4 * NB], a1[4 * NB];
@@ -1168,13 +1193,13 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 if (h == 0) slot_free();
 #pragma unroll
                 for (int i = 0; i < NB; ++i) {
-                  const int b = (h * LDC + 8 * i + 2 * c) * C::kEsz;
+                  const uint32_t chunk = (uint32_t)((h * LDC + 8 * i) * C::kEsz) & ~15u;   // 16-byte chunk of the block
 #pragma unroll
                   for (int k = 0; k < 4; ++k) {
                     if constexpr (C::kEsz == 4)
-                      *reinterpret_cast<uint2*>(stage_at(q + 8 * k, b)) = make_uint2(ow[i * WPB + 2 * k], ow[i * WPB + 2 * k + 1]);
+                      ptx::st_shared_v2(pre[k] ^ chunk, ow[i * WPB + 2 * k], ow[i * WPB + 2 * k + 1]);
                     else
-                      *reinterpret_cast<uint32_t*>(stage_at(q + 8 * k, b)) = ow[i * WPB + k];
+                      ptx::st_shared_b32(pre[k] ^ chunk, ow[i * WPB + k]);
                   }
                 }
               }
@@ -1320,8 +1345,8 @@ qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams p
 template <int BN, int OUT, bool W4>
 qwt_status launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
                        bool want_resident, bool pair, cudaStream_t st) {
-  if constexpr (!W4 && BN == 256 && OUT != kOutCalibStats) {
-    if (pair) return launch_cfg<BN, OUT, false, false, false, true>(tmA, tmB, prm, grid, 0, st);
+  if constexpr (BN == 256 && OUT != kOutCalibStats) {
+    if (pair) return launch_cfg<BN, OUT, W4, false, false, true>(tmA, tmB, prm, grid, 0, st);
   }
   if (!W4) {
     constexpr bool kWide = BN == 256;
@@ -1385,16 +1410,28 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   // CTA and k-block holds the tensor pipe at about half its int8 rate (4 converter warps per CTA).  The weights are
   // then expanded once per call into the workspace (1.5 N K bytes of traffic) and the int8 kernel runs; with few
   // rows (weight-bandwidth-bound) the packed tile is streamed and converted on chip.
+  // CTA pairs change that: each CTA of a pair expands only its half of the W tile (128 rows per k-block), which its
+  // four converter warps do in about the time the MMAs of the k-block take, and loads 24 KB per k-block instead of
+  // 48; wherever pairs can be formed and fill the GPU the packed tile is therefore converted on chip.
+  const int sms = dev.sm_count > 0 ? dev.sm_count : kPlanSMs;
+  bool w4_pair = false;
+  if (wfmt == QWT_W_INT4_PACKED && out_mode != kOutCalibStats && N > 128 && pl.tiles_m >= 2) {
+    const char* e = getenv("QWT_PAIR");
+    const int tn = (N + 255) / 256;
+    const int pair_tiles = ((pl.tiles_m + 1) / 2) * tn;
+    const int pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
+    w4_pair = tn <= pairs && pair_tiles >= sms / 2 && !(e != nullptr && e[0] == '0');
+  }
   {
     const char* e = getenv("QWT_W4_EXPAND");
     const bool many_rows = M >= 1024;
-    pl.w4_expand = wfmt == QWT_W_INT4_PACKED && (e != nullptr ? e[0] == '1' : many_rows);
+    pl.w4_expand = wfmt == QWT_W_INT4_PACKED && (e != nullptr ? e[0] == '1' : (many_rows && !w4_pair));
+    if (pl.w4_expand) w4_pair = false;
   }
   if (pl.w4_expand) wfmt = QWT_W_INT8;        // everything below plans the int8 kernel
   // 256-wide tiles keep the tensor pipe ahead of shared-memory bandwidth and are used when the mainloop
   // dominates (long K); short-K layers are bound by the epilogue, which is organised around 128-wide tiles
   // (four accumulator buffers, so the INT8 row-maximum exchange can trail by two tiles).
-  const int sms = dev.sm_count > 0 ? dev.sm_count : kPlanSMs;
   const int phantom = out_mode == QWT_OUT_INT8_PER_TOKEN ? test_hooks().phantom_units.load(std::memory_order_relaxed) : 0;
   auto score = [&](int bn) {
     const long tn = (N + bn - 1) / bn;
@@ -1408,6 +1445,7 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   const long tiles256 = (long)pl.tiles_m * ((N + 255) / 256);
   pl.bn = (N > 128 && (tiles256 >= sms || score(256) + 0.15 >= score(128))) ? 256 : 128;
   if (out_mode == kOutCalibStats && wfmt == QWT_W_INT4_PACKED) pl.bn = 128;
+  if (w4_pair) pl.bn = 256;
   const char* force = getenv("QWT_FORCE_BN");
   if (force != nullptr) {
     const int f = atoi(force);
@@ -1444,11 +1482,12 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
     const char* e = getenv("QWT_PAIR");
     const int pair_tiles = ((pl.tiles_m + 1) / 2) * pl.tiles_n;
     const int pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
-    const bool fits = !w4 && pl.bn == 256 && !pl.w_resident && !pl.own_strips && out_mode != kOutCalibStats &&
+    const bool fits = pl.bn == 256 && !pl.w_resident && !pl.own_strips && out_mode != kOutCalibStats &&
                       pl.tiles_m >= 2 && pl.tiles_n <= pairs;
     // (measured: ahead by up to 7 % on layers 4096 and 11008 wide with K = 4096 and 11008, behind by 4 % on a layer
     // 768 wide with K = 3072, whose three column tiles leave the pairs little to share)
-    const bool want = e != nullptr ? e[0] == '1' : (K >= 2048 && pl.tiles_n >= 8 && pair_tiles >= sms / 2);
+    const bool want = e != nullptr ? e[0] == '1'
+                                   : (w4 ? w4_pair : (K >= 2048 && pl.tiles_n >= 8 && pair_tiles >= sms / 2));
     pl.pair = fits && want;
     if (pl.pair) pl.grid = 2 * pairs;
   }
@@ -1497,9 +1536,9 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   CUtensorMap tmA, tmB;
   const bool okA = make_byte_map(&tmA, X, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
   // (asymmetric codes and the statistics epilogue have no pair instantiation: the same grid then walks single tiles)
-  const bool pair = plan.pair && w_terms == nullptr && stats == nullptr && !w4;
-  const bool okB = w4 ? make_byte_map(&tmB, W, (uint64_t)N, (uint64_t)K / 2, kBK / 2, (uint32_t)plan.bn,
-                                      CU_TENSOR_MAP_SWIZZLE_NONE)
+  const bool pair = plan.pair && w_terms == nullptr && stats == nullptr;
+  const bool okB = w4 ? make_byte_map(&tmB, W, (uint64_t)N, (uint64_t)K / 2, kBK / 2,
+                                      (uint32_t)(pair ? plan.bn / 2 : plan.bn), CU_TENSOR_MAP_SWIZZLE_NONE)
                       : make_byte_map(&tmB, W, (uint64_t)N, (uint64_t)K, kBK, (uint32_t)(pair ? plan.bn / 2 : plan.bn),
                                       CU_TENSOR_MAP_SWIZZLE_128B);
   if (!okA || !okB) {
@@ -1574,7 +1613,7 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
     prm.Y = ws + plan.ws_z_off;
   }
   qwt_status s;
-  if (w4) s = plan.bn == 256 ? launch_bn<256, true>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, false, st)
+  if (w4) s = plan.bn == 256 ? launch_bn<256, true>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, pair, st)
                              : launch_bn<128, true>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, false, st);
   else s = plan.bn == 256 ? launch_bn<256, false>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, pair, st)
                           : launch_bn<128, false>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, false, st);
