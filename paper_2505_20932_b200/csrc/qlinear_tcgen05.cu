@@ -127,8 +127,25 @@ struct Cfg {
   static constexpr int kAcc = kTmemCols / BN;                        // accumulator buffers (tiles) in TMEM
   static constexpr int kUnitN = unit_cols(OUT);                      // columns of an epilogue unit
   static constexpr int kUPT = BN / kUnitN;                           // epilogue units per tile
-  static constexpr int kConvWarp0 = 2 + kEpiWarps;                   // first converter warp (W4 only)
-  static constexpr int kThreads = 32 * (2 + kEpiWarps + (W4 ? kNumConvWarps : 0));
+  // Warps in groups of four (the unit of register reallocation): warps 0-3 = TMA producer, MMA issuer and two idle
+  // warps; warps 4-19 = the four epilogue groups; warps 20-23 = the converter warps (packed weights only).
+  static constexpr int kEpiWarp0 = 4;
+  static constexpr int kConvWarp0 = kEpiWarp0 + kEpiWarps;           // first converter warp (W4 only)
+  static constexpr int kThreads = 32 * (kEpiWarp0 + kEpiWarps + (W4 ? kNumConvWarps : 0));
+  // Registers: the CTA starts with kLaunchRegs per thread (what the launch bounds allow); once the roles are known
+  // the warps that need few give theirs back to the CTA's pool (setmaxnreg.dec) and the epilogue warps take them
+  // (setmaxnreg.inc waits until the pool holds enough -- the pool is the CTA's own allocation and nothing else, so
+  // the budgets below must add up to no more than the CTA started with):
+  //   int8 weights   640 threads x 96 = 61440;  4 x 32 x 56 + 16 x 32 x 104 = 60416
+  //   packed weights 768 threads x 80: left as launched (the converter warps want their 80, measured)
+  static constexpr int kLaunchRegs = (65536 / kThreads) / 8 * 8;
+  static constexpr int kRegsService = W4 ? kLaunchRegs : 56;
+  static constexpr int kRegsConv = kLaunchRegs;
+  static constexpr int kRegsEpi = W4 ? kLaunchRegs : 104;
+  static_assert(kRegsService <= kLaunchRegs && kRegsConv <= kLaunchRegs && kRegsEpi >= kLaunchRegs, "dec / inc directions");
+  static_assert(32 * (kEpiWarp0 * kRegsService + kEpiWarps * kRegsEpi + (W4 ? kNumConvWarps * kRegsConv : 0)) <=
+                    kThreads * kLaunchRegs,
+                "register budgets exceed what the CTA was launched with: setmaxnreg.inc would wait for ever");
   // output staging: one box of 32 rows per epilogue warp, through which a warp turns "thread = row" into
   // row-contiguous global stores.  128-byte rows for 128-wide tiles; 256-wide tiles use 32-byte rows when the
   // operand ring needs the room (long K: the epilogue hides behind the mainloop) and 64-byte rows otherwise
@@ -334,6 +351,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     atomicCAS(p.status, 0u, code);
   };
 
+  // Registers move from the service (and converter) warps to the epilogue warps; each group of four warps does so at
+  // the top of its own branch, so that the compiler budgets the code below it accordingly.
+  if (warp < C::kEpiWarp0) {
+  if (C::kRegsService < C::kLaunchRegs) ptx::setmaxnreg_dec<C::kRegsService>();
   if (warp == 0) {
     // ------------------------------------------------------------------ TMA producer
     if (lane == 0) {
@@ -458,7 +479,9 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
       }
     }
+  }   // (warps 2 and 3 are idle: they fill the first group of four and wait at the end)
   } else if (W4 && warp >= C::kConvWarp0) {
+    if (C::kRegsConv < C::kLaunchRegs) ptx::setmaxnreg_dec<C::kRegsConv>();
     // ------------------------------------------------------------------ W4 -> INT8 converter warps
     // The packed tile (64 bytes per row, two's-complement nibbles, even element low) is expanded into the
     // 128-byte-swizzled operand tile the MMA descriptor expects.  Each nibble is moved to the HIGH half of
@@ -512,6 +535,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
     }
   } else {
+    if (C::kRegsEpi > C::kLaunchRegs) ptx::setmaxnreg_inc<C::kRegsEpi>();
     // ------------------------------------------------------------------ epilogue warps
     // Work item = one unit: kUnitN columns of a tile.  The CTA's units are numbered u = j * kUPT + part
     // (j = local tile); group g takes u = g, g + 4, ...  Unit u lives in its tile's accumulator buffer, part by part.
@@ -520,7 +544,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     constexpr int BOXB = C::kBoxBytes;
     constexpr int BC = C::kBC;              // columns per staging box
     constexpr int ESZ = C::kEsz;
-    const int ew = warp - 2;
+    const int ew = warp - C::kEpiWarp0;
     const int g = ew / kGroupWarps;
     const int qd = warp & 3;                // TMEM lane quadrant (hardware rule: warp % 4)
     const bool lead = qd == 0;              // stages fscale / fbias and speaks for the group to the other CTAs
@@ -1039,8 +1063,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           double S0 = 0.0, S1 = 0.0, S2 = 0.0, S3 = 0.0, K0q = 0.0, K0f = 0.0;
 #pragma unroll
           for (int qi = 0; qi < kGroupWarps; ++qi) {
-            // the slot of epilogue warp g * 4 + w holds the rows of TMEM quadrant (g * 4 + w + 2) % 4
-            const int w = (qi + 2) & 3;
+            // the slot of epilogue warp g * 4 + w holds the rows of TMEM quadrant w
+            const int w = qi;
             const int left = p.M - (tm * kBM + qi * 32);
             if (left <= 0) continue;                            // nothing of this warp is inside the matrix
             const double nw = (double)(left < 32 ? left : 32);
