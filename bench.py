@@ -735,6 +735,80 @@ def calibration_sweep(c, steps, warmup, seed):
     return rows, total_bytes, total_s, int(B.qwt_launch_count())
 
 
+RESNET50_3X3 = [   # (H = W, C = C_out) of the 3 x 3 convolution inside a bottleneck of stages 2, 3, 4; batch 32
+    (28, 128), (14, 256), (7, 512),
+]
+
+
+def conv_entry(c, steps, batch=32):
+    """CNN-shaped k x k layers: the ResNet-50 3 x 3 bottleneck convolutions (stride 1, pad 1) of the stages whose channel
+    count the implicit-GEMM path takes (C % 128 == 0), per-token (per-pixel) INT8 output, timed through
+    qwt_qconv2d_cwac_forward and, for comparison, through qwt_im2col_i8 + qwt_qlinear_cwac_forward."""
+    torch, B = c.torch, c.B
+    g = torch.Generator(device=c.device)
+    g.manual_seed(12345)
+    layers = []
+    for hw, ch in RESNET50_3X3:
+        X = torch.randn((batch, hw, hw, ch), generator=g, device=c.device)
+        Xq = (X / (X.abs().max() / 127.0)).round().clamp_(-127, 127).to(torch.int8)    # per-tensor codes (inputs only)
+        Wq = torch.randint(-127, 128, (ch, 3, 3, ch), generator=g, device=c.device, dtype=torch.int8)
+        fs = torch.rand(ch, generator=g, device=c.device) * 2e-4 + 1e-4
+        fb = torch.randn(ch, generator=g, device=c.device) * 0.01
+        M, K = batch * hw * hw, 9 * ch
+        Y = torch.empty((M, ch), dtype=torch.int8, device=c.device)
+        ys = torch.empty(M, dtype=torch.float32, device=c.device)
+        wsb = B.qwt_qconv2d_workspace_bytes(batch, hw, hw, ch, ch, 3, 3, 1, 1, B.QWT_OUT_INT8_PER_TOKEN)
+        ws = torch.empty(max(wsb, 256), dtype=torch.uint8, device=c.device)
+        P = torch.empty((M, K), dtype=torch.int8, device=c.device)
+        xs = torch.full((M,), 0.02, dtype=torch.float32, device=c.device)
+        wsb2 = B.qwt_qlinear_workspace_bytes(M, ch, K, B.QWT_W_INT8, B.QWT_OUT_INT8_PER_TOKEN)
+        ws2 = torch.empty(max(wsb2, 256), dtype=torch.uint8, device=c.device)
+        layers.append(dict(hw=hw, ch=ch, M=M, K=K, Xq=Xq, Wq=Wq, fs=fs, fb=fb, Y=Y, ys=ys, ws=ws, wsb=wsb, P=P, xs=xs,
+                           ws2=ws2, wsb2=wsb2))
+
+    def implicit(st):
+        for L in layers:
+            B.qwt_qconv2d_cwac_forward(L["Xq"], 0.02, L["Wq"], L["fs"], L["fb"], batch, L["hw"], L["hw"], L["ch"], L["ch"],
+                                       3, 3, 1, 1, B.QWT_OUT_INT8_PER_TOKEN, L["Y"], L["ys"], L["ws"], L["wsb"], st)
+
+    def patches(st):
+        for L in layers:
+            B.qwt_im2col_i8(L["Xq"], batch, L["hw"], L["hw"], L["ch"], 3, 3, 1, 1, L["P"], st)
+            B.qwt_qlinear_cwac_forward(L["P"], L["xs"], L["Wq"], B.QWT_W_INT8, L["fs"], L["fb"], L["M"], L["ch"], L["K"],
+                                       B.QWT_OUT_INT8_PER_TOKEN, L["Y"], L["ys"], L["ws2"], L["wsb2"], st)
+
+    def timed(fn):
+        for _ in range(3):
+            fn(c.stream)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(c.stream)
+        for _ in range(steps):
+            fn(c.stream)
+        e1.record(c.stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e-3 / steps
+
+    B.qwt_launch_count_reset()
+    t_imp = timed(implicit)
+    launches = B.qwt_launch_count()
+    t_pat = timed(patches)
+    for L in layers:
+        B.qwt_qlinear_check_status(L["ws"])
+    ops = sum(2 * L["M"] * L["ch"] * L["K"] for L in layers)
+    byt = sum(L["Xq"].numel() + L["Wq"].numel() + L["M"] * L["ch"] + 4 * L["M"] + 8 * L["ch"] for L in layers)
+    t_min = max(ops / (c.int8_peak * 1e12), byt / (c.peaks["hbm_gbs"] * 1e9))
+    return {"workload": "ResNet-50 shaped 3 x 3 convolutions (stride 1, pad 1; 28 x 28 x 128, 14 x 14 x 256, 7 x 7 x 512; batch 32), "
+                        "W8A8, per-tensor activation scale, per-pixel INT8 output; direct calls",
+            "layers": len(layers), "steps": steps,
+            "forward": {"tops": ops / t_imp / 1e12, "ms_per_step": t_imp * 1e3, "bound": "tensor",
+                        "frac_int8_peak_burst": ops / t_imp / 1e12 / c.int8_peak, "frac_of_roofline": t_min / t_imp,
+                        "min_time_ms": t_min * 1e3, "path": "implicit GEMM (qwt_qconv2d_cwac_forward)",
+                        "through_patch_matrix_tops": ops / t_pat / 1e12,
+                        "through_patch_matrix_ms": t_pat * 1e3},
+            "calibration": None, "gpu_launches": int(launches)}
+
+
 PER_CONFIG = [   # (workload, calibration-row cap or 0, why the cap)
     ("cfg1", 0, None),
     ("cfg2", 0, None),
@@ -765,6 +839,8 @@ def per_config_entries(c, args):
                     "gpu_launches": r["launches"]})
         del layers, r
         torch.cuda.empty_cache()
+    out.append(conv_entry(c, steps))
+    torch.cuda.empty_cache()
     if args.workload != "cfg5":
         rows, total_bytes, total_s, launches = calibration_sweep(c, steps, 3, args.seed)
         gbs = total_bytes / total_s / 1e9

@@ -304,6 +304,28 @@ qwt_status qwt_qlinear_cwac_forward_asym(const uint8_t* X, const float* x_scale,
 qwt_status qwt_im2col_i8(const int8_t* X, int32_t batch, int32_t H, int32_t W, int32_t C, int32_t kh, int32_t kw,
                          int32_t stride, int32_t pad, int8_t* patches, void* stream);
 
+/* Convolution without the patch matrix (the same layer as an implicit GEMM): the kernel of qwt_qlinear_cwac_forward
+ * reads the activations straight from the NHWC tensor -- a tile's A operand is, per filter tap and block of 128 input
+ * channels, a block of input pixels fetched by one rank-4 tensor-map copy (every `stride`-th position; positions outside
+ * the image read 0, the zero-point of the symmetric codes) -- and writes the output tensor through a rank-4 map as well.
+ *     acc[b, ho, wo, n] = sum_{i, j, c} X[b, ho*stride + i - pad, wo*stride + j - pad, c] * Wt[n, i, j, c]
+ *     z = fma((float)acc * x_scale, fscale[n], fbias[n]),  then the output stage as in qwt_qlinear_cwac_forward
+ * with ONE activation scale x_scale for the whole tensor (the paper's per-tensor S_x; a per-pixel scale would not
+ * factor out of the sum over taps) and, for QWT_OUT_INT8_PER_TOKEN, one output scale per output pixel.
+ *   X  int8 [batch, H, W, C], C % 128 == 0;   Wt int8 [Cout, kh, kw, C];   fscale, fbias float [Cout]
+ *   Y  [batch, Ho, Wo, Cout] of the output type (Ho = (H + 2 pad - kh) / stride + 1, likewise Wo)
+ *   y_scale float [batch * Ho * Wo], QWT_OUT_INT8_PER_TOKEN only
+ *   out_mode: INT8_PER_TOKEN, BF16, FP32 or INT32_ACC;   stride <= 8;   kh * kw * C <= 131072
+ *   workspace >= qwt_qconv2d_workspace_bytes(...), 256-byte aligned; status word as for the forward call.
+ * Other channel counts (C % 16 == 0) go through qwt_im2col_i8.
+ * Errors: NULL, SHAPE, UNSUPPORTED (C % 128, Cout multiple, stride, out_mode), ALIGN, WORKSPACE, ARCH, CUDA. */
+size_t qwt_qconv2d_workspace_bytes(int32_t batch, int32_t H, int32_t W, int32_t C, int32_t Cout, int32_t kh, int32_t kw,
+                                   int32_t stride, int32_t pad, int32_t out_mode);
+qwt_status qwt_qconv2d_cwac_forward(const int8_t* X, float x_scale, const int8_t* Wt, const float* fscale,
+                                    const float* fbias, int32_t batch, int32_t H, int32_t W, int32_t C, int32_t Cout,
+                                    int32_t kh, int32_t kw, int32_t stride, int32_t pad, int32_t out_mode, void* Y,
+                                    float* y_scale, void* workspace, size_t workspace_bytes, void* stream);
+
 /* ---------------------------------------------------------------------------------------------
  * Test hooks (the paper has no counterpart).  Host-side, process-wide switches that exist so that the give-up path of
  * the bounded device-side waits can be exercised without faulting or hanging a GPU; both are 0 in normal operation.

@@ -57,6 +57,8 @@ SIGNATURES = {
     "qwt_quantize_rows_i8": (_i32, [_p, _i64, _i32, _i64, _i32, _p, _p, _p]),
     "qwt_im2col_i8": (_i32, [_p, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _i32, _p, _p]),
     "qwt_pack_int4": (_i32, [_p, _i64, _i32, _p, _p]),
+    "qwt_qconv2d_workspace_bytes": (_sz, [_i32] * 10),
+    "qwt_qconv2d_cwac_forward": (_i32, [_p, C.c_float, _p, _p, _p] + [_i32] * 10 + [_p, _p, _p, _sz, _p]),
     "qwt_test_set_wait_limit_ns": (None, [C.c_uint64]),
     "qwt_test_set_phantom_units": (None, [_i32]),
     "qwt_launch_count": (_i64, []),
@@ -323,3 +325,17 @@ def qwt_test_set_wait_limit_ns(ns: int) -> None:
 
 def qwt_test_set_phantom_units(n: int) -> None:
     lib.qwt_test_set_phantom_units(int(n))
+
+
+def qwt_qconv2d_workspace_bytes(batch, H, W, C_, Cout, kh, kw, stride, pad, out_mode) -> int:
+    return lib.qwt_qconv2d_workspace_bytes(batch, H, W, C_, Cout, kh, kw, stride, pad, out_mode)
+
+
+def qwt_qconv2d_cwac_forward(X, x_scale, Wt, fscale, fbias, batch, H, W, C_, Cout, kh, kw, stride, pad, out_mode, Y, y_scale,
+                             workspace, workspace_bytes, stream=None, check=True) -> int:
+    s = lib.qwt_qconv2d_cwac_forward(_ptr(X), float(x_scale), _ptr(Wt), _ptr(fscale), _ptr(fbias), batch, H, W, C_, Cout,
+                                     kh, kw, stride, pad, out_mode, _ptr(Y), _ptr(y_scale), _ptr(workspace),
+                                     workspace_bytes, _stream(stream))
+    if check:
+        _check(s, "qwt_qconv2d_cwac_forward")
+    return s

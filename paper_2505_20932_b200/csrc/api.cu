@@ -606,6 +606,71 @@ qwt_status qwt_im2col_i8(const int8_t* X, int32_t batch, int32_t H, int32_t W, i
   return launch_im2col_i8(X, batch, H, W, C, kh, kw, stride, pad, patches, as_stream(stream));
 }
 
+namespace {
+// Geometry, plan and argument checks shared by the size query and the call.
+qwt_status qconv_setup(int32_t batch, int32_t H, int32_t W, int32_t C, int32_t Cout, int32_t kh, int32_t kw,
+                       int32_t stride, int32_t pad, int32_t out_mode, QconvArgs* cv, QlinearPlan* plan, int32_t* m_eff,
+                       int32_t* K) {
+  if (batch < 1 || H < 1 || W < 1 || C < 1 || Cout < 1 || kh < 1 || kw < 1 || stride < 1 || pad < 0) return QWT_ERR_SHAPE;
+  if (H + 2 * pad < kh || W + 2 * pad < kw) return QWT_ERR_SHAPE;
+  if (out_mode != QWT_OUT_INT8_PER_TOKEN && out_mode != QWT_OUT_BF16 && out_mode != QWT_OUT_FP32 &&
+      out_mode != QWT_OUT_INT32_ACC)
+    return QWT_ERR_UNSUPPORTED;
+  if ((C % 128) != 0 || stride > 8) return QWT_ERR_UNSUPPORTED;
+  const int nmul = out_mode == QWT_OUT_INT8_PER_TOKEN ? 16 : (out_mode == QWT_OUT_BF16 ? 8 : 4);
+  if (Cout % nmul != 0) return QWT_ERR_UNSUPPORTED;
+  const int64_t k = (int64_t)kh * kw * C;
+  if (k > 131072) return QWT_ERR_SHAPE;
+  *cv = QconvArgs{};
+  cv->B = batch; cv->H = H; cv->W = W; cv->C = C;
+  cv->Ho = (H + 2 * pad - kh) / stride + 1;
+  cv->Wo = (W + 2 * pad - kw) / stride + 1;
+  cv->kh = kh; cv->kw = kw; cv->stride = stride; cv->pad = pad;
+  qconv_tiling(batch, cv->Ho, cv->Wo, stride, cv);
+  const int64_t tiles = (int64_t)cv->tiles_w * cv->tiles_h * cv->tiles_b;
+  if (tiles * 128 >= ((int64_t)1 << 31) || tiles * 128 * (int64_t)Cout >= ((int64_t)1 << 40)) return QWT_ERR_SHAPE;
+  *m_eff = (int32_t)(tiles * 128);
+  *K = (int32_t)k;
+  DeviceInfo dev{};
+  dev.sm_count = kPlanSMs;
+  qwt_status s = qlinear_plan(*m_eff, Cout, *K, QWT_W_INT8, out_mode, dev, plan, /*plain=*/true);
+  if (s != QWT_OK) return s;
+  if (out_mode == QWT_OUT_INT8_PER_TOKEN && !plan->fused_requant) return QWT_ERR_UNSUPPORTED;   // more column tiles than CTAs
+  return QWT_OK;
+}
+}  // namespace
+
+size_t qwt_qconv2d_workspace_bytes(int32_t batch, int32_t H, int32_t W, int32_t C, int32_t Cout, int32_t kh, int32_t kw,
+                                   int32_t stride, int32_t pad, int32_t out_mode) {
+  QconvArgs cv;
+  QlinearPlan plan;
+  int32_t m_eff = 0, K = 0;
+  if (qconv_setup(batch, H, W, C, Cout, kh, kw, stride, pad, out_mode, &cv, &plan, &m_eff, &K) != QWT_OK) return 0;
+  return plan.ws_total;
+}
+
+qwt_status qwt_qconv2d_cwac_forward(const int8_t* X, float x_scale, const int8_t* Wt, const float* fscale,
+                                    const float* fbias, int32_t batch, int32_t H, int32_t W, int32_t C, int32_t Cout,
+                                    int32_t kh, int32_t kw, int32_t stride, int32_t pad, int32_t out_mode, void* Y,
+                                    float* y_scale, void* workspace, size_t workspace_bytes, void* stream) {
+  if (X == nullptr || Wt == nullptr || Y == nullptr || workspace == nullptr) return QWT_ERR_NULL;
+  if (out_mode != QWT_OUT_INT32_ACC && (fscale == nullptr || fbias == nullptr)) return QWT_ERR_NULL;
+  if (out_mode == QWT_OUT_INT8_PER_TOKEN && y_scale == nullptr) return QWT_ERR_NULL;
+  QconvArgs cv;
+  QlinearPlan plan;
+  int32_t m_eff = 0, K = 0;
+  qwt_status s = qconv_setup(batch, H, W, C, Cout, kh, kw, stride, pad, out_mode, &cv, &plan, &m_eff, &K);
+  if (s != QWT_OK) return s;
+  if (!aligned(X, 16) || !aligned(Wt, 16) || !aligned(Y, 16)) return QWT_ERR_ALIGN;
+  if (workspace_bytes < plan.ws_total || !aligned(workspace, 256)) return QWT_ERR_WORKSPACE;
+  DeviceInfo real;
+  if ((s = current_device(&real)) != QWT_OK) return s;
+  if (real.sm_count < plan.grid) return QWT_ERR_ARCH;
+  cv.x_scale = x_scale;
+  return launch_qlinear(X, nullptr, Wt, QWT_W_INT8, fscale, fbias, m_eff, Cout, K, out_mode, Y, y_scale, workspace, plan,
+                        as_stream(stream), nullptr, nullptr, nullptr, nullptr, &cv);
+}
+
 qwt_status qwt_pack_int4(const int8_t* codes, int64_t rows, int32_t cols, uint8_t* packed, void* stream) {
   if (codes == nullptr || packed == nullptr) return QWT_ERR_NULL;
   if (rows < 1 || cols < 2) return QWT_ERR_SHAPE;

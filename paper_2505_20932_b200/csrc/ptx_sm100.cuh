@@ -118,6 +118,25 @@ __device__ __forceinline__ void tma_load_2d(void* smem_dst, const CUtensorMap* t
       : "memory");
 }
 
+// The same for a rank-4 map (NHWC activations: channel bytes, w, h, image).  Out-of-range coordinates, negative ones
+// included, read the fill value; c0 must give a 16-byte aligned start.
+__device__ __forceinline__ void tma_load_4d(void* smem_dst, const CUtensorMap* tm, int32_t c0, int32_t c1, int32_t c2,
+                                            int32_t c3, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.tile.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6];"
+      ::"r"(smem_u32(smem_dst)), "l"(reinterpret_cast<uint64_t>(tm)), "r"(c0), "r"(c1), "r"(c2), "r"(c3),
+      "r"(smem_u32(bar))
+      : "memory");
+}
+// Rank-4 store of a dense box; no coordinate may be negative, the part of the box outside the tensor is not written.
+__device__ __forceinline__ void tma_store_4d(const CUtensorMap* tm, const void* smem_src, int32_t c0, int32_t c1,
+                                             int32_t c2, int32_t c3) {
+  asm volatile("cp.async.bulk.tensor.4d.global.shared::cta.tile.bulk_group [%0, {%1, %2, %3, %4}], [%5];" ::"l"(
+                   reinterpret_cast<uint64_t>(tm)),
+               "r"(c0), "r"(c1), "r"(c2), "r"(c3), "r"(smem_u32(smem_src))
+               : "memory");
+}
+
 // Shared memory -> global (tiled, 2D): the box at smem_src (dense, in the map's swizzle) is written to the tensor
 // at element coordinates (x, y); x must give a 16-byte aligned start, and neither coordinate may be negative.  The
 // part of the box outside the tensor is not written.  The shared-memory source must have been made visible

@@ -103,6 +103,18 @@ struct QlParams {
   const int* w_terms;            // [2 N]: -Z_W[n], then K Z_W[n] - sum_k W_q[n, k]
   int local_pair;                // per-token INT8: a strip is one 256-wide tile of two units, exchanged inside the CTA
   int own_strips;                // per-token INT8: a strip is two 256-wide tiles, both taken by the same CTA
+  // Convolution as an implicit GEMM (NHWC activations, rank-4 tensor maps): a tile's 128 rows are the output pixels of
+  // a block of cv_bw x cv_bh positions of cv_bn images (powers of two, product 128; row r of the tile is pixel
+  // (r % bw, (r / bw) % bh, r / (bw * bh)) of the block); a k-block is 128 input channels of one filter tap.
+  struct Conv {
+    int on;
+    int bw_log, bh_log;            // log2 of the block's width and height (the rest of the 128 rows: images)
+    int tiles_w, tiles_h;          // blocks per image row / column (row-strip index = (image block, block row, block column))
+    int Wo, Ho, B;                 // output width, height, images
+    int stride, pad, kw, cpb;      // cpb: 128-channel blocks per pixel
+    int sub_w, sub_h;              // the 32 rows of an epilogue warp as (sub_w, sub_h, 32 / (sub_w * sub_h)) positions
+    float x_scale;                 // per-tensor activation scale S_x
+  } cv;
   // calibration statistics instead of an output matrix (Section 3.3, Eq. 4-5)
   const float* F;                // [M, ldf] full-precision output of the same layer on the same rows
   long long ldf;
@@ -379,7 +391,19 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             ok = false;
             break;
           }
-          if (PAIR && W4) {
+          if (!PAIR && !W4 && p.cv.on) {
+            // implicit GEMM: the activations of one filter tap, 128 channels, for the tile's block of output pixels
+            // (zero outside the image: the zero-point of the symmetric codes)
+            const int tap = kb / p.cv.cpb, cb = kb - tap * p.cv.cpb;
+            const int fi = tap / p.cv.kw, fj = tap - fi * p.cv.kw;
+            const int tw = walk.tm % p.cv.tiles_w, t2 = walk.tm / p.cv.tiles_w;
+            const int th = t2 % p.cv.tiles_h, tb = t2 / p.cv.tiles_h;
+            ptx::mbar_arrive_expect_tx(&full[s], kABytes + C::kBBytes);
+            ptx::tma_load_4d(sA + s * kABytes, &tmA, cb * kBK, ((tw << p.cv.bw_log) * p.cv.stride) + fj - p.cv.pad,
+                             ((th << p.cv.bh_log) * p.cv.stride) + fi - p.cv.pad,
+                             tb << (7 - p.cv.bw_log - p.cv.bh_log), &full[s]);
+            ptx::tma_load_2d(sB + s * C::kBBytes, &tmB, kb * kBK, n0, &full[s]);
+          } else if (PAIR && W4) {
             // packed weights: a CTA's loads are counted on its own barrier, for its own converter warps, which then
             // report to the even CTA
             ptx::mbar_arrive_expect_tx(&full[s], kABytes + C::kPBytes);
@@ -619,11 +643,17 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     // The same box by a bulk tensor store issued by one lane: the LSU sees nothing of it and the warp goes on
     // at once.  The staging slot may be rewritten when the copy has read it: slot_free() before the next box's
     // first write (by then the copy has usually had the next box's TMEM load and arithmetic to finish reading).
+    int box_w = 0, box_h = 0, box_b = 0;             // convolution: output position of the warp's 32 rows
     auto tma_box = [&](int x_bytes, int y) {
       ptx::fence_proxy_async_smem();                 // this lane's writes to the slot, for the async proxy
       __syncwarp();
       if (lane == 0) {
-        if (y < p.M) ptx::tma_store_2d(&tmY, stg, x_bytes, y);
+        if (p.cv.on) {
+          if (box_w < p.cv.Wo && box_h < p.cv.Ho && box_b < p.cv.B)
+            ptx::tma_store_4d(&tmY, stg, x_bytes, box_w, box_h, box_b);
+        } else if (y < p.M) {
+          ptx::tma_store_2d(&tmY, stg, x_bytes, y);
+        }
         ptx::bulk_commit_group();
       }
     };
@@ -647,9 +677,24 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 #pragma unroll
         for (int k = 0; k < 4; ++k) {
           const int r = y0 + (lane >> 2) + 8 * k;
-          if (r < p.M) xs4[k] = __ldg(p.x_scale + r);
+          if (p.cv.on) xs4[k] = p.cv.x_scale;
+          else if (r < p.M) xs4[k] = __ldg(p.x_scale + r);
         }
       }
+      // convolution: the tile's block of output pixels, and where row r of the tile lies in the output
+      int cv_w0 = 0, cv_h0 = 0, cv_b0 = 0;
+      if (p.cv.on) {
+        const int tw = tm % p.cv.tiles_w, t2 = tm / p.cv.tiles_w;
+        cv_w0 = tw << p.cv.bw_log;
+        cv_h0 = (t2 % p.cv.tiles_h) << p.cv.bh_log;
+        cv_b0 = (t2 / p.cv.tiles_h) << (7 - p.cv.bw_log - p.cv.bh_log);
+      }
+      auto cv_pixel = [&](int r, int& w, int& h, int& b) {        // r = row inside the tile
+        w = cv_w0 + (r & ((1 << p.cv.bw_log) - 1));
+        h = cv_h0 + ((r >> p.cv.bw_log) & ((1 << p.cv.bh_log) - 1));
+        b = cv_b0 + (r >> (p.cv.bw_log + p.cv.bh_log));
+      };
+      if (p.cv.on) cv_pixel(qd * 32, box_w, box_h, box_b);
       // statistics: the thread's rows inside the matrix, and the first step's values of f (requested before the
       // waits below; every later step is requested one step ahead)
       constexpr int NB = 2;                   // statistics: 8-column blocks per step
@@ -947,7 +992,14 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         }
         // ---------------------------------------------------------------- phase 2: scale, codes
         const float ys = __fdiv_rn(amax_row, 127.f);
-        if (n0 == 0 && row < p.M) p.y_scale[row] = ys;
+        if (p.cv.on) {
+          int pw, ph_, pb;
+          cv_pixel(qd * 32 + my, pw, ph_, pb);
+          if (n0 == 0 && pw < p.cv.Wo && ph_ < p.cv.Ho && pb < p.cv.B)
+            p.y_scale[((size_t)pb * p.cv.Ho + ph_) * p.cv.Wo + pw] = ys;
+        } else if (n0 == 0 && row < p.M) {
+          p.y_scale[row] = ys;
+        }
         const float den_mine = ys > 0.f ? ys : 1.f;          // a zero row has z == 0 everywhere: codes 0
         const float inv_mine = __frcp_rn(den_mine);
         // a scale so small that its reciprocal overflows (never on real data): divide directly
@@ -1290,6 +1342,32 @@ bool make_byte_map(CUtensorMap* tm, const void* base, uint64_t rows, uint64_t ro
   return r == CUDA_SUCCESS;
 }
 
+// NHWC byte tensor [B, H, W, row_bytes] -> rank-4 map with a box of {box_bytes, box_w (every `stride`-th position),
+// box_h (likewise), box_b}.
+bool make_nhwc_map(CUtensorMap* tm, const void* base, uint64_t B, uint64_t H, uint64_t W, uint64_t row_bytes,
+                   uint32_t box_bytes, uint32_t box_w, uint32_t box_h, uint32_t box_b, uint32_t stride,
+                   CUtensorMapSwizzle swz) {
+  EncodeTiledFn fn = get_encode_fn();
+  if (fn == nullptr) return false;
+  cuuint64_t dims[4] = {row_bytes, W, H, B};
+  cuuint64_t strides[3] = {row_bytes, row_bytes * W, row_bytes * W * H};
+  cuuint32_t box[4] = {box_bytes, box_w * stride, box_h * stride, box_b};
+  cuuint32_t estr[4] = {1, stride, stride, 1};
+  CUresult r = fn(tm, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<void*>(base), dims, strides, box, estr,
+                  CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                  CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+  return r == CUDA_SUCCESS;
+}
+
+// Convolution: the output map is rank 4 as well; its box depends on the instantiation's staging box, so the
+// launcher builds it from this description (set by launch_qconv2d around its launch, per thread).
+struct ConvOutSpec {
+  bool on;
+  uint64_t B, Ho, Wo, row_bytes;
+  uint32_t sub_w, sub_h, sub_b;
+};
+thread_local ConvOutSpec tl_conv_out = {};
+
 unsigned long long timeout_ns_from_env() {
   const unsigned long long forced = test_hooks().wait_limit_ns.load(std::memory_order_relaxed);
   if (forced != 0ull) return forced;
@@ -1316,7 +1394,11 @@ qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams p
   if (C::kTmaStore) {
     constexpr CUtensorMapSwizzle swz = C::kBoxBytes == 32 ? CU_TENSOR_MAP_SWIZZLE_32B
                                        : (C::kBoxBytes == 64 ? CU_TENSOR_MAP_SWIZZLE_64B : CU_TENSOR_MAP_SWIZZLE_128B);
-    if (!make_byte_map(&tmY, prm.Y, (uint64_t)prm.M, (uint64_t)prm.N * C::kEsz, C::kBoxBytes, 32, swz)) {
+    const ConvOutSpec& co = tl_conv_out;
+    const bool ok = co.on ? make_nhwc_map(&tmY, prm.Y, co.B, co.Ho, co.Wo, co.row_bytes, C::kBoxBytes, co.sub_w, co.sub_h,
+                                          co.sub_b, 1, swz)
+                          : make_byte_map(&tmY, prm.Y, (uint64_t)prm.M, (uint64_t)prm.N * C::kEsz, C::kBoxBytes, 32, swz);
+    if (!ok) {
       set_cuda_error((int)cudaErrorInvalidValue);
       return QWT_ERR_CUDA;
     }
@@ -1426,8 +1508,28 @@ qwt_status launch_bn(int out_mode, const CUtensorMap& tmA, const CUtensorMap& tm
 
 }  // namespace
 
+void qconv_tiling(int B, int Ho, int Wo, int stride, QconvArgs* out) {
+  long best_tiles = -1;
+  for (int bwl = 7; bwl >= 0; --bwl) {
+    for (int bhl = 0; bwl + bhl <= 7; ++bhl) {
+      const int bw = 1 << bwl, bh = 1 << bhl, bb = 128 >> (bwl + bhl);
+      if (bw * stride > 256 || bh * stride > 256) continue;      // a box side covers at most 256 positions
+      const long tw = (Wo + bw - 1) / bw, th = (Ho + bh - 1) / bh, tb = (B + bb - 1) / bb;
+      const long tiles = tw * th * tb;
+      if (best_tiles < 0 || tiles < best_tiles) {
+        best_tiles = tiles;
+        out->bw_log = bwl;
+        out->bh_log = bhl;
+        out->tiles_w = (int)tw;
+        out->tiles_h = (int)th;
+        out->tiles_b = (int)tb;
+      }
+    }
+  }
+}
+
 qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
-                        QlinearPlan* plan) {
+                        QlinearPlan* plan, bool plain) {
   QlinearPlan pl{};
   pl.tiles_m = (M + kBM - 1) / kBM;
   // Packed int4 weights: with many rows the layer is compute-bound, and converting the W tile on chip for every
@@ -1483,7 +1585,7 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   const bool w4 = wfmt == QWT_W_INT4_PACKED;
   const long w_tile_bytes = (long)((K + kBK - 1) / kBK) * kBK * pl.bn;
   const char* nores = getenv("QWT_NO_RESIDENT_W");
-  pl.w_resident = !w4 && w_tile_bytes <= 96 * 1024 && pl.tiles_n <= sms && tiles > sms &&
+  pl.w_resident = !plain && !w4 && w_tile_bytes <= 96 * 1024 && pl.tiles_n <= sms && tiles > sms &&
                   !(nores != nullptr && nores[0] == '1');
   if (pl.w_resident) pl.grid = (sms / pl.tiles_n) * pl.tiles_n;
   // Per-token INT8 whose rows span exactly two 256-wide tiles, with at least half a grid of strips: a CTA takes
@@ -1492,7 +1594,7 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   {
     const char* e = getenv("QWT_OWN_STRIPS");
     const bool want = e != nullptr ? e[0] == '1' : true;
-    pl.own_strips = want && out_mode == QWT_OUT_INT8_PER_TOKEN && pl.tiles_n == 2 && pl.bn == 256 && !w4 &&
+    pl.own_strips = !plain && want && out_mode == QWT_OUT_INT8_PER_TOKEN && pl.tiles_n == 2 && pl.bn == 256 && !w4 &&
                     pl.tiles_m >= sms / 2 && phantom == 0;
     if (pl.own_strips) {
       pl.w_resident = false;
@@ -1506,7 +1608,7 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
     const char* e = getenv("QWT_PAIR");
     const int pair_tiles = ((pl.tiles_m + 1) / 2) * pl.tiles_n;
     const int pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
-    const bool fits = pl.bn == 256 && !pl.w_resident && !pl.own_strips && out_mode != kOutCalibStats &&
+    const bool fits = !plain && pl.bn == 256 && !pl.w_resident && !pl.own_strips && out_mode != kOutCalibStats &&
                       pl.tiles_m >= 2 && pl.tiles_n <= pairs;
     // (measured: ahead by up to 7 % on layers 4096 and 11008 wide with K = 4096 and 11008, behind by 4 % on a layer
     // 768 wide with K = 3072, whose three column tiles leave the pairs little to share)
@@ -1547,7 +1649,7 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
                           const float* fbias, int32_t M, int32_t N, int32_t K, int32_t out_mode, void* Y,
                           float* y_scale, void* workspace, const QlinearPlan& plan, cudaStream_t st,
                           const int32_t* x_zero, const int32_t* x_rowsum, const int32_t* w_terms,
-                          const QlinearStatsArgs* stats) {
+                          const QlinearStatsArgs* stats, const QconvArgs* conv) {
   uint8_t* ws = static_cast<uint8_t*>(workspace);
   if (plan.w4_expand) {
     int8_t* w8 = reinterpret_cast<int8_t*>(ws + plan.ws_w_off);
@@ -1558,7 +1660,14 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   }
   const bool w4 = wfmt == QWT_W_INT4_PACKED;
   CUtensorMap tmA, tmB;
-  const bool okA = make_byte_map(&tmA, X, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
+  // convolution: X is the NHWC activation tensor and a tile's A operand a block of its pixels (one filter tap, 128
+  // channels); M is then the number of tile rows (128 x row strips), K = kh * kw * C
+  const bool okA = conv != nullptr
+                       ? make_nhwc_map(&tmA, X, (uint64_t)conv->B, (uint64_t)conv->H, (uint64_t)conv->W, (uint64_t)conv->C,
+                                       kBK, 1u << conv->bw_log, 1u << conv->bh_log,
+                                       128u >> (conv->bw_log + conv->bh_log), (uint32_t)conv->stride,
+                                       CU_TENSOR_MAP_SWIZZLE_128B)
+                       : make_byte_map(&tmA, X, (uint64_t)M, (uint64_t)K, kBK, kBM, CU_TENSOR_MAP_SWIZZLE_128B);
   // (asymmetric codes and the statistics epilogue have no pair instantiation: the same grid then walks single tiles)
   const bool pair = plan.pair && w_terms == nullptr && stats == nullptr;
   const bool okB = w4 ? make_byte_map(&tmB, W, (uint64_t)N, (uint64_t)K / 2, kBK / 2,
@@ -1622,6 +1731,31 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   prm.counters = prm.rowmax + (size_t)plan.tiles_m * kBM;
   prm.flags = prm.counters + plan.tiles_m;
   prm.timeout_ns = timeout_ns_from_env();
+  if (conv != nullptr) {
+    prm.cv.on = 1;
+    prm.cv.bw_log = conv->bw_log;
+    prm.cv.bh_log = conv->bh_log;
+    prm.cv.tiles_w = conv->tiles_w;
+    prm.cv.tiles_h = conv->tiles_h;
+    prm.cv.Wo = conv->Wo;
+    prm.cv.Ho = conv->Ho;
+    prm.cv.B = conv->B;
+    prm.cv.stride = conv->stride;
+    prm.cv.pad = conv->pad;
+    prm.cv.kw = conv->kw;
+    prm.cv.cpb = conv->C / kBK;
+    prm.cv.x_scale = conv->x_scale;
+    const int bw = 1 << conv->bw_log, bh = 1 << conv->bh_log;
+    prm.cv.sub_w = bw < 32 ? bw : 32;
+    prm.cv.sub_h = bh < 32 / prm.cv.sub_w ? bh : 32 / prm.cv.sub_w;
+    const size_t esz = out_mode == QWT_OUT_INT8_PER_TOKEN ? 1 : (out_mode == QWT_OUT_BF16 ? 2 : 4);
+    tl_conv_out = ConvOutSpec{true, (uint64_t)conv->B, (uint64_t)conv->Ho, (uint64_t)conv->Wo, (uint64_t)N * esz,
+                              (uint32_t)prm.cv.sub_w, (uint32_t)prm.cv.sub_h,
+                              (uint32_t)(32 / (prm.cv.sub_w * prm.cv.sub_h))};
+  }
+  struct ConvOutReset {       // the description applies to this launch only
+    ~ConvOutReset() { tl_conv_out.on = false; }
+  } conv_out_reset;
   if (stats != nullptr) {
     prm.F = stats->F;
     prm.ldf = stats->ldf;

@@ -115,8 +115,19 @@ struct QlinearPlan {
                          // compute-bound and the int8 mainloop is twice as fast as the one that converts on chip)
   size_t ws_status_off, ws_partial_off, ws_z_off, ws_w_off, ws_total;
 };
+// plain: every CTA streams both operands for single tiles b, b + G, ... (no resident W tile, own strips or CTA pairs)
 qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
-                        QlinearPlan* plan);
+                        QlinearPlan* plan, bool plain = false);
+// Convolution as an implicit GEMM: geometry of the tiles (blocks of 2^bw_log x 2^bh_log output positions of
+// 128 >> (bw_log + bh_log) images) over an NHWC tensor.
+struct QconvArgs {
+  int B, H, W, C, Ho, Wo;
+  int kh, kw, stride, pad;
+  int bw_log, bh_log, tiles_w, tiles_h, tiles_b;
+  float x_scale;
+};
+// The block shape that wastes the fewest tile rows for this output size (ties: the widest block).
+void qconv_tiling(int B, int Ho, int Wo, int stride, QconvArgs* out);
 // Internal output mode of the forward kernel: no output matrix, the per-channel sums of Eq. 4-5 instead.
 constexpr int kOutCalibStats = 5;
 struct QlinearStatsArgs {
@@ -129,7 +140,8 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
                           const float* fbias, int32_t M, int32_t N, int32_t K, int32_t out_mode, void* Y,
                           float* y_scale, void* workspace, const QlinearPlan& plan, cudaStream_t st,
                           const int32_t* x_zero = nullptr, const int32_t* x_rowsum = nullptr,
-                          const int32_t* w_terms = nullptr, const QlinearStatsArgs* stats = nullptr);
+                          const int32_t* w_terms = nullptr, const QlinearStatsArgs* stats = nullptr,
+                          const QconvArgs* conv = nullptr);
 qwt_status launch_quantize_rows_u8(const float* X, int64_t rows, int32_t cols, int64_t ld, uint8_t* Xq, float* scale,
                                    int32_t* zero, int32_t* rowsum, cudaStream_t st);
 qwt_status launch_asym_weight_terms(const uint8_t* W, const int32_t* w_zero, int32_t N, int32_t K, int32_t* w_terms,
