@@ -1532,27 +1532,26 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
                         QlinearPlan* plan, bool plain) {
   QlinearPlan pl{};
   pl.tiles_m = (M + kBM - 1) / kBM;
-  // Packed int4 weights: with many rows the layer is compute-bound, and converting the W tile on chip for every
-  // CTA and k-block holds the tensor pipe at about half its int8 rate (4 converter warps per CTA).  The weights are
-  // then expanded once per call into the workspace (1.5 N K bytes of traffic) and the int8 kernel runs; with few
-  // rows (weight-bandwidth-bound) the packed tile is streamed and converted on chip.
-  // CTA pairs change that: each CTA of a pair expands only its half of the W tile (128 rows per k-block), which its
-  // four converter warps do in about the time the MMAs of the k-block take, and loads 24 KB per k-block instead of
-  // 48; wherever pairs can be formed and fill the GPU the packed tile is therefore converted on chip.
+  // Packed int4 weights are expanded to int8 on chip, tile by tile, by four converter warps; with CTA pairs each CTA
+  // expands only its half of the W tile (128 rows per k-block) and loads 24 KB per k-block instead of 48.  With many
+  // rows the layer is compute-bound and the converting mainloop still trails the int8 one (ViT-B shapes at 25 216 rows,
+  // BF16 out: 0.86-0.98 of it for K = 768, 0.85 for K = 3072; single CTAs: 0.65-0.75), so by default the weights are
+  // then expanded once per call into the workspace (1.5 N K bytes of traffic) and the int8 kernel runs; with few rows
+  // (weight-bandwidth-bound) the packed tile is streamed and converted on chip.  QWT_W4_EXPAND=0 / 1 forces either.
   const int sms = dev.sm_count > 0 ? dev.sm_count : kPlanSMs;
+  {
+    const char* e = getenv("QWT_W4_EXPAND");
+    const bool many_rows = M >= 1024;
+    pl.w4_expand = wfmt == QWT_W_INT4_PACKED && (e != nullptr ? e[0] == '1' : many_rows);
+  }
+  // on chip: pairs wherever they can be formed and fill the GPU
   bool w4_pair = false;
-  if (wfmt == QWT_W_INT4_PACKED && out_mode != kOutCalibStats && N > 128 && pl.tiles_m >= 2) {
+  if (wfmt == QWT_W_INT4_PACKED && !pl.w4_expand && out_mode != kOutCalibStats && N > 128 && pl.tiles_m >= 2) {
     const char* e = getenv("QWT_PAIR");
     const int tn = (N + 255) / 256;
     const int pair_tiles = ((pl.tiles_m + 1) / 2) * tn;
     const int pairs = pair_tiles < sms / 2 ? pair_tiles : sms / 2;
     w4_pair = tn <= pairs && pair_tiles >= sms / 2 && !(e != nullptr && e[0] == '0');
-  }
-  {
-    const char* e = getenv("QWT_W4_EXPAND");
-    const bool many_rows = M >= 1024;
-    pl.w4_expand = wfmt == QWT_W_INT4_PACKED && (e != nullptr ? e[0] == '1' : (many_rows && !w4_pair));
-    if (pl.w4_expand) w4_pair = false;
   }
   if (pl.w4_expand) wfmt = QWT_W_INT8;        // everything below plans the int8 kernel
   // 256-wide tiles keep the tensor pipe ahead of shared-memory bandwidth and are used when the mainloop

@@ -105,20 +105,19 @@ def test_config4_layers_sampled_rows(B, layer):
     assert bool((ys > 0).all()) and bool((Y.abs().amax(dim=1) == 127).all())
 
 
-@pytest.mark.parametrize("w4_path", ["default", "single_cta", "workspace"])
+@pytest.mark.parametrize("w4_path", ["default", "pairs", "single_cta"])
 @pytest.mark.parametrize("layer", [0, 1, 2, 3])
 def test_config3_layers_sampled_rows_w4_bf16(B, layer, w4_path, monkeypatch):
     """ViT-B block at 128 x 197 tokens, packed 4-bit weights, BF16 output, through the three weight paths: the plan's
-    own choice for these shapes (nibbles expanded in shared memory by the converter warps of CTA pairs, each CTA its
-    half of the W tile), the same expansion by single CTAs (QWT_PAIR=0, QWT_W4_EXPAND=0), and the weights expanded
-    once per call into the workspace (QWT_W4_EXPAND=1)."""
+    own choice for this many rows (the weights expanded once per call into the workspace), nibbles expanded in shared
+    memory by the converter warps of CTA pairs, each CTA its half of the W tile (QWT_W4_EXPAND=0), and the same
+    expansion by single CTAs (QWT_W4_EXPAND=0, QWT_PAIR=0)."""
     monkeypatch.delenv("QWT_W4_EXPAND", raising=False)
     monkeypatch.delenv("QWT_PAIR", raising=False)
-    if w4_path == "single_cta":
+    if w4_path != "default":
         monkeypatch.setenv("QWT_W4_EXPAND", "0")
+    if w4_path == "single_cta":
         monkeypatch.setenv("QWT_PAIR", "0")
-    elif w4_path == "workspace":
-        monkeypatch.setenv("QWT_W4_EXPAND", "1")
     spec = WL.config_layers(3)[layer]
     Xq, xs, W, Wq, fs, fb = recipe_layer(B, spec, seed=30 + layer)
     Y, _ = run_forward(B, Xq, xs, W, fs, fb, B.QWT_OUT_BF16, B.QWT_W_INT4_PACKED, spec.K)
