@@ -92,6 +92,13 @@ __device__ __forceinline__ void st_shared_v2(uint32_t addr, uint32_t v0, uint32_
   asm volatile("st.shared.v2.b32 [%0], {%1, %2};" ::"r"(addr), "r"(v0), "r"(v1) : "memory");
 }
 
+// ---------------------------------------------------------------- programmatic dependent launch
+// When the kernel was launched with programmatic stream serialization it may start while the kernel before it in the
+// stream is still running; this waits until that kernel has finished and its memory is visible (a no-op otherwise).
+__device__ __forceinline__ void grid_dependency_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+// Lets the kernel behind this one in the stream start launching (it will wait, as above, before it touches memory).
+__device__ __forceinline__ void grid_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // ---------------------------------------------------------------- registers
 // Per-thread register budget of the calling group of four warps (all four must execute it); a multiple of 8.
 template <int N>

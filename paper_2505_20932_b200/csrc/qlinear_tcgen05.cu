@@ -351,6 +351,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
   }
   ptx::tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
+  // Everything above touched only this CTA's shared and tensor memory.  From here on global memory is read and written:
+  // with a programmatic launch (the kernel may have started under the tail of the one before it in the stream) wait for
+  // that kernel to finish first.
+  ptx::grid_dependency_wait();
 
   // Without the INT8 exchange nothing else in the workspace is used: the first CTA clears the status word
   // (a wait can only give up seconds later).
@@ -383,6 +387,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       TileWalk walk;
       walk.init(p, walker, G);
       for (int jt = 0; ok && jt < n_local; ++jt, walk.advance()) {
+        // With its last tile under way this CTA lets the kernel behind this one in the stream begin: that kernel's CTAs
+        // take the SMs as they fall free, do their set-up and wait for this kernel's end before they touch global
+        // memory.  (Earlier would be no use, a waiting CTA only holds an SM that another stream's kernel could work on.)
+        if (jt + 1 >= n_local) ptx::grid_launch_dependents();
         const int m0 = strip_of(walk.tm) * kBM;
         const int n0 = walk.tn * BN;
         for (int kb = 0; kb < p.num_kb; ++kb, ++issued) {
@@ -1368,6 +1376,20 @@ struct ConvOutSpec {
 };
 thread_local ConvOutSpec tl_conv_out = {};
 
+// Programmatic dependent launch of the non-cooperative forward kernels (QWT_PDL=1; off by default).  In a single
+// stream it takes about 1 us off every call that follows another kernel (DeiT-S shapes, BF16 out, graph replay:
+// 13.1 -> 12.1, 8.5 -> 7.6, 15.3 -> 14.1, 17.3 -> 16.2 us).  With several streams it can cost more than it gives: a
+// dependent kernel's CTAs take SMs as they fall free and then wait there, which keeps a cooperative kernel of another
+// stream (the per-token INT8 exchange needs its whole grid resident) from starting (DeiT-S stack over two streams:
+// 787 -> 652 TOPS).
+bool programmatic_launch_enabled() {
+  static const bool on = [] {
+    const char* e = getenv("QWT_PDL");
+    return e != nullptr && e[0] == '1';
+  }();
+  return on;
+}
+
 unsigned long long timeout_ns_from_env() {
   const unsigned long long forced = test_hooks().wait_limit_ns.load(std::memory_order_relaxed);
   if (forced != 0ull) return forced;
@@ -1428,10 +1450,15 @@ qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams p
     attrs[0].val.clusterDim.x = 2;
     attrs[0].val.clusterDim.y = 1;
     attrs[0].val.clusterDim.z = 1;
-    attrs[1].id = cudaLaunchAttributeCooperative;
-    attrs[1].val.cooperative = 1;
+    if (cooperative) {
+      attrs[1].id = cudaLaunchAttributeCooperative;
+      attrs[1].val.cooperative = 1;
+    } else {
+      attrs[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+      attrs[1].val.programmaticStreamSerializationAllowed = 1;
+    }
     cfg.attrs = attrs;
-    cfg.numAttrs = cooperative ? 2 : 1;
+    cfg.numAttrs = (cooperative || programmatic_launch_enabled()) ? 2 : 1;
     QWT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmY, prm));
     count_launch();
   } else if (cooperative) {
@@ -1440,8 +1467,20 @@ qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams p
     QWT_CUDA_TRY(cudaLaunchCooperativeKernel((const void*)kern, dim3(grid), dim3(kThreads), args, smem_bytes, st));
     count_launch();
   } else {
-    kern<<<grid, kThreads, smem_bytes, st>>>(tmA, tmB, tmY, prm);
-    QWT_LAUNCH_CHECK();
+    // plain launch, allowed to begin (barrier set-up, tensor-memory allocation) while the kernel before it in the stream
+    // is still finishing; the kernel itself waits for that kernel before it touches global memory
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = dim3(grid);
+    cfg.blockDim = dim3(kThreads);
+    cfg.dynamicSmemBytes = (size_t)smem_bytes;
+    cfg.stream = st;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = programmatic_launch_enabled() ? 1 : 0;
+    QWT_CUDA_TRY(cudaLaunchKernelEx(&cfg, kern, tmA, tmB, tmY, prm));
+    count_launch();
   }
   return QWT_OK;
 }
