@@ -123,7 +123,7 @@ struct QlParams {
 };
 
 // Compile-time geometry of one instantiation.
-template <int BN, int OUT, bool W4, bool WIDE, bool ASYM = false, bool PAIR = false>
+template <int BN, int OUT, bool W4, int WIDE, bool ASYM = false, bool PAIR = false>
 struct Cfg {
   // PAIR: two CTAs of a cluster work on two row strips of the same column tile; the even CTA issues MMAs of
   // M = 256 (tcgen05 cta_group::2) that take the A tile and half of the W tile from each CTA's shared memory
@@ -162,7 +162,7 @@ struct Cfg {
   // row-contiguous global stores.  128-byte rows for 128-wide tiles; 256-wide tiles use 32-byte rows when the
   // operand ring needs the room (long K: the epilogue hides behind the mainloop) and 64-byte rows otherwise
   // (statistics: the slot holds the warp's four sums and two shifts of the unit's 128 columns, 3 KB)
-  static constexpr int kBoxBytes = kStats ? 96 : (BN == 128 ? (kStatic8 && kUnitN < 128 ? 64 : 128) : (WIDE ? 64 : 32));
+  static constexpr int kBoxBytes = kStats ? 96 : (BN == 128 ? (kStatic8 && kUnitN < 128 ? 64 : 128) : (WIDE == 1 ? 64 : 32));
   static constexpr int kBC = kBoxBytes / kEsz;                       // columns per box
   static constexpr int kSlotBytes = 32 * kBoxBytes;
   static constexpr int kStagingBytes = kEpiWarps * kSlotBytes;
@@ -264,7 +264,7 @@ struct TileWalk {
   }
 };
 
-template <int BN, int OUT, bool W4, bool WIDE, bool ASYM, bool PAIR>
+template <int BN, int OUT, bool W4, int WIDE, bool ASYM, bool PAIR>
 __global__ void __launch_bounds__((Cfg<BN, OUT, W4, WIDE, ASYM, PAIR>::kThreads), 1)
 qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmY, const QlParams p) {
@@ -378,9 +378,17 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // With a grid that is a multiple of tiles_n every tile of this CTA has the same column tile: its W
         // tile is loaded once and the ring below streams X only (half the bytes per tile through the SM's
         // load port, which is what bounds short-K layers).
-        const int n0 = ((int)blockIdx.x % p.tiles_n) * BN;      // (one modulo per call)
-        ptx::mbar_arrive_expect_tx(wfull, (uint32_t)(p.res_kb * C::kBBytes));
-        for (int kb = 0; kb < p.res_kb; ++kb) ptx::tma_load_2d(sWres + kb * C::kBBytes, &tmB, kb * kBK, n0, wfull);
+        const int n0 = (walker % p.tiles_n) * BN + (int)rank * C::kBRows;      // (one modulo per call)
+        if (PAIR) {
+          // each CTA keeps its half of the pair's W tile; both halves are counted on the even CTA's barrier
+          const uint32_t lead_wfull = ptx::mapa_shared(ptx::smem_u32(wfull), 0u);
+          if (rank == 0u) ptx::mbar_arrive_expect_tx(wfull, 2u * (uint32_t)(p.res_kb * C::kBBytes));
+          for (int kb = 0; kb < p.res_kb; ++kb)
+            ptx::tma_load_2d_pair(sWres + kb * C::kBBytes, &tmB, kb * kBK, n0, lead_wfull);
+        } else {
+          ptx::mbar_arrive_expect_tx(wfull, (uint32_t)(p.res_kb * C::kBBytes));
+          for (int kb = 0; kb < p.res_kb; ++kb) ptx::tma_load_2d(sWres + kb * C::kBBytes, &tmB, kb * kBK, n0, wfull);
+        }
       }
       uint32_t issued = 0, s = 0, ph = 0;
       bool ok = true;
@@ -420,9 +428,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           } else if (PAIR) {
             // both CTAs' loads of the stage are counted on the even CTA's barrier, where the MMAs are issued
             const uint32_t lead_full = ptx::mapa_shared(ptx::smem_u32(&full[s]), 0u);
-            if (rank == 0u) ptx::mbar_arrive_expect_tx(&full[s], 2u * (kABytes + C::kBBytes));
+            if (rank == 0u) ptx::mbar_arrive_expect_tx(&full[s], 2u * (kABytes + (resident ? 0 : C::kBBytes)));
             ptx::tma_load_2d_pair(sA + s * kABytes, &tmA, kb * kBK, m0, lead_full);
-            ptx::tma_load_2d_pair(sB + s * C::kBBytes, &tmB, kb * kBK, n0 + (int)rank * C::kBRows, lead_full);
+            if (!resident)
+              ptx::tma_load_2d_pair(sB + s * C::kBBytes, &tmB, kb * kBK, n0 + (int)rank * C::kBRows, lead_full);
           } else if (resident) {
             ptx::mbar_arrive_expect_tx(&full[s], kABytes);
             ptx::tma_load_2d(sA + s * kABytes, &tmA, kb * kBK, m0, &full[s]);
@@ -1405,7 +1414,7 @@ unsigned long long timeout_ns_from_env() {
   return v;
 }
 
-template <int BN, int OUT, bool W4, bool WIDE, bool ASYM = false, bool PAIR = false>
+template <int BN, int OUT, bool W4, int WIDE, bool ASYM = false, bool PAIR = false>
 qwt_status launch_cfg(const CUtensorMap& tmA, const CUtensorMap& tmB, QlParams prm, int grid, int res_kb,
                       cudaStream_t st) {
   using C = Cfg<BN, OUT, W4, WIDE, ASYM, PAIR>;
@@ -1491,15 +1500,25 @@ template <int BN, int OUT, bool W4>
 qwt_status launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const QlParams& prm, int grid,
                        bool want_resident, bool pair, cudaStream_t st) {
   if constexpr (BN == 256 && OUT != kOutCalibStats) {
-    if (pair) return launch_cfg<BN, OUT, W4, false, false, true>(tmA, tmB, prm, grid, 0, st);
+    if (pair) {
+      if constexpr (!W4) {
+        // short K: each CTA of a pair keeps its half of the W tile for the whole call; the ring then carries X only
+        // (64-byte staging boxes while at least four X stages remain, else 32-byte ones)
+        if (want_resident && Cfg<BN, OUT, false, 1, false, true>::stages_for(prm.num_kb) >= 4)
+          return launch_cfg<BN, OUT, false, 1, false, true>(tmA, tmB, prm, grid, prm.num_kb, st);
+        if (want_resident && Cfg<BN, OUT, false, 0, false, true>::stages_for(prm.num_kb) >= 4)
+          return launch_cfg<BN, OUT, false, 0, false, true>(tmA, tmB, prm, grid, prm.num_kb, st);
+      }
+      return launch_cfg<BN, OUT, W4, 0, false, true>(tmA, tmB, prm, grid, 0, st);
+    }
   }
   if (!W4) {
-    constexpr bool kWide = BN == 256;
+    constexpr int kWide = BN == 256 ? 1 : 0;
     using CW = Cfg<BN, OUT, false, kWide>;
     if (want_resident && CW::stages_for(prm.num_kb) >= 4)
       return launch_cfg<BN, OUT, false, kWide>(tmA, tmB, prm, grid, prm.num_kb, st);
   }
-  return launch_cfg<BN, OUT, W4, false>(tmA, tmB, prm, grid, 0, st);
+  return launch_cfg<BN, OUT, W4, 0>(tmA, tmB, prm, grid, 0, st);
 }
 
 // Asymmetric (unsigned) codes: int8 weights only, streaming operand ring.
@@ -1654,6 +1673,26 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
                                    : (w4 ? w4_pair : (K >= 2048 && pl.tiles_n >= 8 && pair_tiles >= sms / 2));
     pl.pair = fits && want;
     if (pl.pair) pl.grid = 2 * pairs;
+    // Short K whose 256-wide W tile is too large to stay in one CTA's shared memory: as a pair, with half of the tile
+    // resident in each CTA (at most 8 k-blocks = 128 KB) and a number of pairs that is a multiple of tiles_n, so that
+    // every tile of a pair has the same column tile.  What a CTA then moves per tile is its X tile and the output: the
+    // W tile no longer goes through its port to L2 once per tile.  Measured at 25 216 rows, K = 768 (BF16 / FP32 /
+    // static INT8 / raw accumulators out): 2304 wide 47.1 -> 43.4, 64.0 -> 55.1, 47.9 -> 46.9, 62.2 -> 53.4 us; 3072
+    // wide 61.8 -> 55.1, 84.0 -> 71.0, 62.9 -> 59.4, 81.4 -> 68.3 us; 16 % at 50 432 rows, 14 % at K = 512, 2 % at
+    // K = 1024; a layer 768 wide (three column tiles, 72 of 74 pairs used) loses 1-10 %, and per-token INT8 output,
+    // whose pace the row-maximum exchange sets, gains nothing: both keep the single-CTA streaming kernel.
+    const char* pr = getenv("QWT_PAIR_RESIDENT");
+    const int num_kb = (K + kBK - 1) / kBK;
+    const int res_pairs = pl.tiles_n > 0 ? (sms / 2 / pl.tiles_n) * pl.tiles_n : 0;
+    const bool res_fits = !plain && !w4 && pl.bn == 256 && !pl.w_resident && !pl.own_strips &&
+                          out_mode != kOutCalibStats && pl.tiles_m >= 2 && num_kb <= 8 && res_pairs > 0 &&
+                          pair_tiles >= 2 * res_pairs;
+    const bool res_want = pr != nullptr ? pr[0] == '1' : (pl.tiles_n >= 6 && out_mode != QWT_OUT_INT8_PER_TOKEN);
+    if (res_fits && res_want) {
+      pl.pair = true;
+      pl.w_resident = true;
+      pl.grid = 2 * res_pairs;
+    }
   }
   pl.fused_requant = (out_mode == QWT_OUT_INT8_PER_TOKEN) && (pl.tiles_n <= (pl.pair ? pl.grid / 2 : pl.grid));
   size_t off = 0;

@@ -383,3 +383,27 @@ def test_cta_pairs_every_output_stage(H, B, M, N, K, monkeypatch):
     c_ref, ys_ref = O.requant_per_token(z_ref)
     assert np.allclose(ys, ys_ref, rtol=1e-5, atol=0)
     assert_codes_close(codes, c_ref)
+
+
+@pytest.mark.parametrize("M,N,K,force", [(6221, 1536, 400, "1"), (5117, 1552, 1024, "1"), (6221, 1536, 400, None)])
+def test_cta_pairs_with_resident_w_halves(H, B, M, N, K, force, monkeypatch):
+    """Short K, many rows, at least six column tiles: every CTA of a pair keeps its half of the pair's W tile in shared
+    memory for the whole call and streams X only (a number of pairs that is a multiple of the column tiles, so that a
+    pair never changes its column tile).  Ragged M, N and K; K = 1024 takes the instantiation with the narrow staging
+    boxes.  Forced on, the per-token INT8 exchange runs over the pairs as well; left to the plan (force None), the
+    other output modes take the path by themselves."""
+    if force is not None:
+        monkeypatch.setenv("QWT_PAIR_RESIDENT", force)
+    Xq, Wq, xs, fs, fb = random_layer(M, N, K, seed=M + N + K + 9)
+    acc_ref = O.int_matmul(Xq, Wq)
+    z_ref = O.forward_folded(acc_ref, xs, fs, fb)
+    acc, _ = H.gpu_forward(Xq, None, Wq, None, None, B.QWT_OUT_INT32_ACC)
+    assert np.array_equal(acc.astype(np.int64), acc_ref)
+    z, _ = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_FP32)
+    assert_fp32_close(z, z_ref)
+    bits, _ = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_BF16)
+    assert_bf16_close(bits, z_ref, O.to_bf16_bits, O.bf16_bits_to_f32)
+    codes, ys = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_INT8_PER_TOKEN)
+    c_ref, ys_ref = O.requant_per_token(z_ref)
+    assert np.allclose(ys, ys_ref, rtol=1e-5, atol=0)
+    assert_codes_close(codes, c_ref)
