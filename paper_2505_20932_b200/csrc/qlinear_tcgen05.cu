@@ -89,6 +89,11 @@ struct QlParams {
   int nl_base, nl_rem, nl_mul, step_q, step_r;
   int stages;           // depth of the operand ring in shared memory
   int res_kb;           // > 0: the CTA's W tile (all res_kb k-blocks) stays resident, the ring holds X only
+  // Packed int4 weights with a resident W tile (CTA pairs): the tile arrives packed, once, and the epilogue warps expand
+  // it into the resident buffer before their first unit; the operands then hold 16 x code and the epilogue divides
+  // by 16 (w4_mul = 1/16 on fscale, offsets x 16, raw accumulators >> 4), exactly as with the converter warps.
+  int w4_res;
+  float w4_mul;
   uint32_t* status;
   unsigned long long* partial;   // [tiles_m][units per strip][128]: (tag, row maximum of the unit), zero = not yet there
   uint32_t counter_target;       // units of a row strip that lie inside the matrix
@@ -322,6 +327,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     for (int i = lane; i < C::kNumBars; i += 32) {
       uint32_t count = 1;                                            // full, empty, tfull, pfull, ready, drain, wfull
       if (i >= 2 * kMaxStages && i < 3 * kMaxStages) count = (kNumConvWarps / 2) * (PAIR ? 2 : 1);   // conv: a team
+      // packed resident tile: conv[0] counts the packed tile's bytes, conv[1] this CTA's expanding warps (the ring is
+      // free for X), conv[2] (even CTA) the expanding warps of both CTAs (the MMAs may start)
+      if (!W4 && p.w4_res && i >= 2 * kMaxStages && i < 2 * kMaxStages + 3)
+        count = i == 2 * kMaxStages ? 1 : (i == 2 * kMaxStages + 1 ? kEpiWarps : 2 * kEpiWarps);
       else if (i >= 3 * kMaxStages + kAcc && i < 3 * kMaxStages + 2 * kAcc)
         count = kGroupWarps * C::kUPT * (PAIR ? 2 : 1);              // tempty (pairs: the warps of both CTAs)
       else if (i >= 3 * kMaxStages + 2 * kAcc + kGroups && i < 3 * kMaxStages + 2 * kAcc + 2 * kGroups)
@@ -379,7 +388,15 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         // tile is loaded once and the ring below streams X only (half the bytes per tile through the SM's
         // load port, which is what bounds short-K layers).
         const int n0 = (walker % p.tiles_n) * BN + (int)rank * C::kBRows;      // (one modulo per call)
-        if (PAIR) {
+        if (PAIR && !W4 && p.w4_res) {
+          // the packed half tile (64 bytes per row and k-block) lands in the top end of the still unused X ring; the
+          // stages it covers are filled with X only when the epilogue warps have expanded it into the resident buffer
+          // (the first X loads, into the stages below it, are under way meanwhile)
+          constexpr int kPackedKb = C::kBRows * (kBK / 2);
+          uint8_t* const packed = sA + stages * kABytes - p.res_kb * kPackedKb;
+          ptx::mbar_arrive_expect_tx(&conv[0], (uint32_t)(p.res_kb * kPackedKb));
+          for (int kb = 0; kb < p.res_kb; ++kb) ptx::tma_load_2d(packed + kb * kPackedKb, &tmB, kb * (kBK / 2), n0, &conv[0]);
+        } else if (PAIR) {
           // each CTA keeps its half of the pair's W tile; both halves are counted on the even CTA's barrier
           const uint32_t lead_wfull = ptx::mapa_shared(ptx::smem_u32(wfull), 0u);
           if (rank == 0u) ptx::mbar_arrive_expect_tx(wfull, 2u * (uint32_t)(p.res_kb * C::kBBytes));
@@ -392,6 +409,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       }
       uint32_t issued = 0, s = 0, ph = 0;
       bool ok = true;
+      // packed resident tile: first ring stage that overlaps the packed tile's landing area
+      const uint32_t held_from = (PAIR && !W4 && p.w4_res)
+                                     ? (uint32_t)((stages * kABytes - p.res_kb * C::kBRows * (kBK / 2)) / kABytes)
+                                     : 0xffffffffu;
       TileWalk walk;
       walk.init(p, walker, G);
       for (int jt = 0; ok && jt < n_local; ++jt, walk.advance()) {
@@ -404,6 +425,11 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         for (int kb = 0; kb < p.num_kb; ++kb, ++issued) {
           if (!ptx::mbar_wait_bounded(&empty[s], ph ^ 1u, cta_abort, tmo)) {
             give_up(kStWaitEmpty);
+            ok = false;
+            break;
+          }
+          if (issued == held_from && !ptx::mbar_wait_bounded(&conv[1], 0, cta_abort, tmo)) {
+            give_up(kStWaitFull);
             ok = false;
             break;
           }
@@ -447,6 +473,11 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           }
         }
       }
+      if (*cta_abort != 0 && !W4 && p.w4_res) {      // the packed tile's copies (counted in this CTA)
+        uint32_t polls = 0;
+        while (!ptx::mbar_try_wait(&conv[0], 0) && ++polls < (1u << 16)) {
+        }
+      }
       if (*cta_abort != 0 && (rank == 0u || W4)) {
         // let copies still in flight land before the CTA's shared memory is released (pairs: the even CTA's
         // barriers count the loads of both, and the odd CTA stays until the pair's final synchronisation)
@@ -458,7 +489,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           while (!ptx::mbar_try_wait(&full[n % stages], (n / stages) & 1u) && ++polls < (1u << 16)) {
           }
         }
-        if (resident) {
+        if (resident && !(!W4 && p.w4_res)) {
           uint32_t polls = 0;
           while (!ptx::mbar_try_wait(wfull, 0) && ++polls < (1u << 16)) {
           }
@@ -472,7 +503,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       const uint32_t a_base = ptx::smem_u32(sA), b_base = ptx::smem_u32(sB), w_base = ptx::smem_u32(sWres);
       uint32_t s = 0, ph = 0, it = 0;
       bool ok = true;
-      if (resident && !ptx::mbar_wait_bounded(wfull, 0, cta_abort, tmo)) {
+      if (resident && !ptx::mbar_wait_bounded((!W4 && p.w4_res) ? &conv[2] : wfull, 0, cta_abort, tmo)) {
         give_up(kStWaitFull);
         ok = false;
       }
@@ -620,10 +651,10 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           pre_cd[i] = c < p.N ? __ldg(p.w_terms + p.N + c) : 0;
         }
         if (!C::kHasParams) continue;
-        pre_fs[i] = c < p.N ? __ldg(p.fscale + c) * (W4 ? 0.0625f : 1.0f) : 0.f;   // W4 operands hold 16 x code
+        pre_fs[i] = c < p.N ? __ldg(p.fscale + c) * (W4 ? 0.0625f : p.w4_mul) : 0.f;   // W4 operands hold 16 x code
         if (C::kStatic8) {   // integer accumulator offsets travel as bit patterns (x16 with the x16 W4 operands)
           const int o = c < p.N ? __ldg(reinterpret_cast<const int*>(p.fbias) + c) : 0;
-          pre_fb[i] = __int_as_float(W4 ? o * 16 : o);
+          pre_fb[i] = __int_as_float((W4 || p.w4_res) ? o * 16 : o);
         } else {
           pre_fb[i] = (c < p.N && p.fbias != nullptr) ? __ldg(p.fbias + c) : 0.f;   // statistics: no bias = 0
         }
@@ -678,6 +709,48 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
       if (lane == 0) ptx::bulk_wait_read_all();
       __syncwarp();
     };
+
+    if (PAIR && !W4 && p.w4_res) {
+      // Packed resident tile: all sixteen epilogue warps expand this CTA's half (two's-complement nibbles, even element
+      // low, each moved to the HIGH half of its byte: the operand holds 16 x code) from the X ring, where it landed,
+      // into the resident buffer in the 128-byte-swizzled layout of the MMA descriptor; then the ring is free for X
+      // and, once both CTAs are through, the even CTA's MMAs may start.
+      bool fine = ptx::mbar_wait_bounded(&conv[0], 0, cta_abort, tmo);
+      if (fine) {
+        constexpr int kPackedKb = C::kBRows * (kBK / 2);
+        const uint8_t* const packed = sA + stages * kABytes - p.res_kb * kPackedKb;    // top end of the X ring
+        const int t = (int)threadIdx.x - C::kEpiWarp0 * 32;
+        const int items = p.res_kb * C::kBRows * 4;          // 16-byte chunks of the packed tile
+        for (int it = t; it < items; it += kEpiWarps * 32) {
+          const int kb = it / (C::kBRows * 4), rem = it - kb * (C::kBRows * 4);
+          const int n_row = rem >> 2, ch = rem & 3;
+          const uint4 w = *reinterpret_cast<const uint4*>(packed + kb * kPackedKb + n_row * 64 + ch * 16);
+          const uint32_t in[4] = {w.x, w.y, w.z, w.w};
+          uint32_t out[8];
+#pragma unroll
+          for (int i = 0; i < 4; ++i) {
+            const uint32_t lo = (in[i] << 4) & 0xF0F0F0F0u;   // even elements, nibble in the high half
+            const uint32_t hi = in[i] & 0xF0F0F0F0u;          // odd elements
+            out[2 * i] = __byte_perm(lo, hi, 0x5140);
+            out[2 * i + 1] = __byte_perm(lo, hi, 0x7362);
+          }
+          uint8_t* row = sWres + kb * C::kBBytes + n_row * 128;
+          const int sw = n_row & 7;
+          *reinterpret_cast<uint4*>(row + (((2 * ch) ^ sw) << 4)) = make_uint4(out[0], out[1], out[2], out[3]);
+          *reinterpret_cast<uint4*>(row + (((2 * ch + 1) ^ sw) << 4)) = make_uint4(out[4], out[5], out[6], out[7]);
+        }
+        ptx::fence_proxy_async_smem();     // generic-proxy writes -> visible to the tensor core's async proxy
+      }
+      __syncwarp();
+      if (lane == 0) {
+        if (fine) {
+          ptx::mbar_arrive(&conv[1]);
+          ptx::mbar_arrive_cluster(ptx::mapa_shared(ptx::smem_u32(&conv[2]), 0u));
+        } else {
+          give_up(kStWaitFull);
+        }
+      }
+    }
 
     int use = 0;                            // units this group has handled
     int slice_n0 = -1;                      // first column of the unit whose parameters are in the group's slice
@@ -1244,7 +1317,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 if (ASYM) asym_fix(a0 + 4 * i, a1 + 4 * i, c0 + 8 * i);
                 if constexpr (OUT == QWT_OUT_INT32_ACC) {
                   // W4: every term is a multiple of 16, the shift is exact
-                  auto fix = [](uint32_t v) { return W4 ? (uint32_t)((int)v >> 4) : v; };
+                  const bool sixteenfold = W4 || p.w4_res != 0;
+                  auto fix = [&](uint32_t v) { return sixteenfold ? (uint32_t)((int)v >> 4) : v; };
 #pragma unroll
                   for (int k = 0; k < 4; ++k) {
                     ow[i * WPB + 2 * k] = fix(k < 2 ? a0[4 * i + 2 * k] : a1[4 * i + 2 * k - 4]);
@@ -1508,6 +1582,7 @@ qwt_status launch_inst(const CUtensorMap& tmA, const CUtensorMap& tmB, const QlP
           return launch_cfg<BN, OUT, false, 1, false, true>(tmA, tmB, prm, grid, prm.num_kb, st);
         if (want_resident && Cfg<BN, OUT, false, 0, false, true>::stages_for(prm.num_kb) >= 4)
           return launch_cfg<BN, OUT, false, 0, false, true>(tmA, tmB, prm, grid, prm.num_kb, st);
+        if (prm.w4_res) return QWT_ERR_UNSUPPORTED;     // (the plan checks the same conditions: not reached)
       }
       return launch_cfg<BN, OUT, W4, 0, false, true>(tmA, tmB, prm, grid, 0, st);
     }
@@ -1586,8 +1661,51 @@ void qconv_tiling(int B, int Ho, int Wo, int stride, QconvArgs* out) {
   }
 }
 
+namespace {
+// Whether the pair kernel with resident W halves has room for its X ring (the conditions launch_inst applies).
+template <int OUT>
+constexpr bool pair_resident_has_room(int num_kb) {
+  return Cfg<256, OUT, false, 1, false, true>::stages_for(num_kb) >= 4 ||
+         Cfg<256, OUT, false, 0, false, true>::stages_for(num_kb) >= 4;
+}
+bool pair_resident_fits(int out_mode, int num_kb) {
+  switch (out_mode) {
+    case QWT_OUT_INT8_PER_TOKEN: return pair_resident_has_room<QWT_OUT_INT8_PER_TOKEN>(num_kb);
+    case QWT_OUT_BF16: return pair_resident_has_room<QWT_OUT_BF16>(num_kb);
+    case QWT_OUT_FP32: return pair_resident_has_room<QWT_OUT_FP32>(num_kb);
+    case QWT_OUT_INT32_ACC: return pair_resident_has_room<QWT_OUT_INT32_ACC>(num_kb);
+    case QWT_OUT_INT8_STATIC: return pair_resident_has_room<QWT_OUT_INT8_STATIC>(num_kb);
+  }
+  return false;
+}
+qwt_status qlinear_plan_impl(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
+                             QlinearPlan* plan, bool plain);
+}  // namespace
+
 qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
                         QlinearPlan* plan, bool plain) {
+  // Packed int4 weights: where the int8 kernel would run as CTA pairs with resident W halves, the packed tile is
+  // expanded on chip, once per CTA, into that resident buffer -- the weights cross HBM as N K / 2 bytes and no
+  // workspace copy is made.  QWT_W4_EXPAND=1 keeps the workspace expansion.
+  // Measured on the ViT-B shapes at 25 216 rows (BF16 out) against the workspace expansion in front of the same pair
+  // kernel: 2304 x 768 43.6 -> 42.4 us, 3072 x 768 55.3 -> 52.8 us; level over the 48-layer stack on two streams (there the
+  // expansion kernels of one stream hide under the other stream's GEMMs).
+  const char* e = getenv("QWT_W4_EXPAND");
+  if (wfmt == QWT_W_INT4_PACKED && !plain && out_mode != kOutCalibStats && !(e != nullptr && e[0] == '1')) {
+    QlinearPlan t{};
+    const qwt_status s = qlinear_plan_impl(M, N, K, QWT_W_INT8, out_mode, dev, &t, plain);
+    if (s == QWT_OK && t.pair && t.w_resident && pair_resident_fits(out_mode, (K + kBK - 1) / kBK)) {
+      t.w4_res = true;
+      *plan = t;
+      return QWT_OK;
+    }
+  }
+  return qlinear_plan_impl(M, N, K, wfmt, out_mode, dev, plan, plain);
+}
+
+namespace {
+qwt_status qlinear_plan_impl(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t out_mode, const DeviceInfo& dev,
+                             QlinearPlan* plan, bool plain) {
   QlinearPlan pl{};
   pl.tiles_m = (M + kBM - 1) / kBM;
   // Packed int4 weights are expanded to int8 on chip, tile by tile, by four converter warps; with CTA pairs each CTA
@@ -1687,7 +1805,8 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
     const bool res_fits = !plain && !w4 && pl.bn == 256 && !pl.w_resident && !pl.own_strips &&
                           out_mode != kOutCalibStats && pl.tiles_m >= 2 && num_kb <= 8 && res_pairs > 0 &&
                           pair_tiles >= 2 * res_pairs;
-    const bool res_want = pr != nullptr ? pr[0] == '1' : (pl.tiles_n >= 6 && out_mode != QWT_OUT_INT8_PER_TOKEN);
+    const bool res_want = pr != nullptr ? pr[0] == '1'
+                                        : (pl.tiles_n >= 6 && out_mode != QWT_OUT_INT8_PER_TOKEN);
     if (res_fits && res_want) {
       pl.pair = true;
       pl.w_resident = true;
@@ -1721,6 +1840,7 @@ qwt_status qlinear_plan(int32_t M, int32_t N, int32_t K, int32_t wfmt, int32_t o
   *plan = pl;
   return QWT_OK;
 }
+}  // namespace
 
 qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, int32_t wfmt, const float* fscale,
                           const float* fbias, int32_t M, int32_t N, int32_t K, int32_t out_mode, void* Y,
@@ -1736,6 +1856,8 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
     wfmt = QWT_W_INT8;
   }
   const bool w4 = wfmt == QWT_W_INT4_PACKED;
+  // (the packed resident tile exists for the symmetric pair kernel only; the plan asks for it for nothing else)
+  if (plan.w4_res && (!w4 || w_terms != nullptr || stats != nullptr || conv != nullptr)) return QWT_ERR_UNSUPPORTED;
   CUtensorMap tmA, tmB;
   // convolution: X is the NHWC activation tensor and a tile's A operand a block of its pixels (one filter tap, 128
   // channels); M is then the number of tile rows (128 x row strips), K = kh * kw * C
@@ -1808,6 +1930,8 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
   prm.counters = prm.rowmax + (size_t)plan.tiles_m * kBM;
   prm.flags = prm.counters + plan.tiles_m;
   prm.timeout_ns = timeout_ns_from_env();
+  prm.w4_res = plan.w4_res ? 1 : 0;
+  prm.w4_mul = plan.w4_res ? 0.0625f : 1.0f;
   if (conv != nullptr) {
     prm.cv.on = 1;
     prm.cv.bw_log = conv->bw_log;
@@ -1848,7 +1972,7 @@ qwt_status launch_qlinear(const int8_t* X, const float* x_scale, const void* W, 
     prm.Y = ws + plan.ws_z_off;
   }
   qwt_status s;
-  if (w4) s = plan.bn == 256 ? launch_bn<256, true>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, pair, st)
+  if (w4 && !plan.w4_res) s = plan.bn == 256 ? launch_bn<256, true>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, pair, st)
                              : launch_bn<128, true>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, false, st);
   else s = plan.bn == 256 ? launch_bn<256, false>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, pair, st)
                           : launch_bn<128, false>(mode, tmA, tmB, prm, plan.grid, plan.w_resident, false, st);

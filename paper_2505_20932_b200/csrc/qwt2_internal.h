@@ -113,6 +113,8 @@ struct QlinearPlan {
   bool pair;             // CTA pairs (clusters of two, MMAs of M = 256 issued by the even CTA); the grid is even
   bool w4_expand;        // packed int4 weights are expanded to int8 in the workspace first (many rows: the GEMM is
                          // compute-bound and the int8 mainloop is twice as fast as the one that converts on chip)
+  bool w4_res;           // packed int4 weights, CTA pairs with resident W halves: every CTA expands its half once, on
+                         // chip, and the int8 pair kernel runs on the resident operand (no workspace copy of W)
   size_t ws_status_off, ws_partial_off, ws_z_off, ws_w_off, ws_total;
 };
 // plain: every CTA streams both operands for single tiles b, b + G, ... (no resident W tile, own strips or CTA pairs)

@@ -407,3 +407,26 @@ def test_cta_pairs_with_resident_w_halves(H, B, M, N, K, force, monkeypatch):
     c_ref, ys_ref = O.requant_per_token(z_ref)
     assert np.allclose(ys, ys_ref, rtol=1e-5, atol=0)
     assert_codes_close(codes, c_ref)
+
+
+@pytest.mark.parametrize("M,N,K", [(6221, 1536, 416), (5117, 1552, 1024)])
+def test_w4_resident_halves_expanded_on_chip(H, B, M, N, K):
+    """Packed weights, many rows, at least six column tiles, short K: the plan runs the int8 pair kernel on W halves that
+    every CTA expands once, on chip, from the packed tile (no workspace copy of W).  Ragged M, N and K (a last k-block
+    of 32 elements); extreme nibbles in the first rows; every output stage against the oracle."""
+    Xq, Wq, Wp, xs, fs, fb = random_w4_layer(M, N, K, seed=M + N + K + 13)
+    Wq[:3, :] = np.array([[-7], [7], [0]], np.int8)
+    Wq[1, 1::2] = -7                                       # even and odd nibbles differ
+    Wp = O.pack_int4(Wq)
+    acc_ref = O.int_matmul(Xq, Wq)
+    z_ref = O.forward_folded(acc_ref, xs, fs, fb)
+    acc, _ = H.gpu_forward(Xq, None, Wp, None, None, B.QWT_OUT_INT32_ACC, wfmt=B.QWT_W_INT4_PACKED, K=K)
+    assert np.array_equal(acc.astype(np.int64), acc_ref)
+    z, _ = H.gpu_forward(Xq, xs, Wp, fs, fb, B.QWT_OUT_FP32, wfmt=B.QWT_W_INT4_PACKED, K=K)
+    assert_fp32_close(z, z_ref)
+    bits, _ = H.gpu_forward(Xq, xs, Wp, fs, fb, B.QWT_OUT_BF16, wfmt=B.QWT_W_INT4_PACKED, K=K)
+    assert_bf16_close(bits, z_ref, O.to_bf16_bits, O.bf16_bits_to_f32)
+    codes, ys = H.gpu_forward(Xq, xs, Wp, fs, fb, B.QWT_OUT_INT8_PER_TOKEN, wfmt=B.QWT_W_INT4_PACKED, K=K)
+    c_ref, ys_ref = O.requant_per_token(z_ref)
+    assert np.allclose(ys, ys_ref, rtol=1e-5, atol=0)
+    assert_codes_close(codes, c_ref)

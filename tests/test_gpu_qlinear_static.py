@@ -84,3 +84,13 @@ def test_static_with_packed_int4_weights(H, B):
     mult, off = H.gpu_fold_static(ws, bias, a, b, S_x, S_r)
     codes, _ = H.gpu_forward(Xq, None, O.pack_int4(Wq), mult, off, B.QWT_OUT_INT8_STATIC, wfmt=B.QWT_W_INT4_PACKED, K=K)
     assert np.array_equal(codes, O.requant_static(O.int_matmul(Xq, Wq), mult, off))
+
+
+def test_static_with_packed_int4_weights_resident_halves(H, B):
+    """The same through the pair kernel whose W halves are expanded on chip once per CTA (many rows, six column tiles):
+    the integer offsets are then sixteenfold like the operands."""
+    M, N, K = 6200, 1536, 416
+    Xq, Wq, ws, bias, a, b, S_x, S_r = layer(M, N, K, seed=6, w_bits=4)
+    mult, off = H.gpu_fold_static(ws, bias, a, b, S_x, S_r)
+    codes, _ = H.gpu_forward(Xq, None, O.pack_int4(Wq), mult, off, B.QWT_OUT_INT8_STATIC, wfmt=B.QWT_W_INT4_PACKED, K=K)
+    assert np.array_equal(codes, O.requant_static(O.int_matmul(Xq, Wq), mult, off))
