@@ -190,8 +190,9 @@ qwt_status qwt_cwac_fold_static(const float* w_scale, const float* bias, const f
  *                           (reinterpreted); x_scale and y_scale are not used (NULL).  No workspace traffic.
  *
  *   X [M, K] int8; x_scale [M] float (may be NULL for INT32_ACC)
- *   W [N, K] int8, or [N, K/2] packed int4 (expanded to int8 on chip tile by tile; with 1024 rows or more, once per
- *     call into the workspace, which is sized for it)
+ *   W [N, K] int8, or [N, K/2] packed int4 (expanded to int8 on chip: tile by tile, or once per CTA where the layer
+ *     runs on CTA pairs that keep their W halves in shared memory; otherwise, with 1024 rows or more, once per call
+ *     into the workspace, which qwt_qlinear_workspace_bytes sizes for it)
  *   fscale, fbias [N] float (may be NULL for INT32_ACC)
  *   Y [M, N] of the output type; y_scale [M] float out, INT8 mode only (else NULL)
  *   K % 16 == 0 (int8) or K % 32 == 0 (packed int4); X, W, Y bases 16-byte aligned;
