@@ -1,4 +1,4 @@
-"""GPU parity on seeded random layer shapes: the forward plan has many branches (tile width, resident W tile, own strips,
+"""GPU parity on seeded random layer shapes and calibration problems: the forward plan has many branches (tile width, resident W tile, own strips,
 CTA pairs, resident W halves, packed weights on chip or through the workspace, the three row-maximum exchanges, the
 two-kernel fallback), chosen from M, N, K, the weight format and the output mode; shapes drawn at random, ragged in every
 dimension, walk through them without anybody having picked the edges by hand.  Every case is checked against the oracle."""
@@ -6,7 +6,7 @@ import numpy as np
 import pytest
 
 from oracle import qwt_oracle as O
-from tolerances import assert_bf16_close, assert_codes_close, assert_fp32_close
+from tolerances import assert_ab_close, assert_bf16_close, assert_codes_close, assert_fp32_close
 
 pytestmark = pytest.mark.gpu
 
@@ -72,3 +72,39 @@ def test_random_shape_against_the_oracle(H, B, M, N, K, w4, mode):
         c_ref, ys_ref = O.requant_per_token(z_ref)
         assert np.allclose(ys, ys_ref, rtol=1e-5, atol=0)
         assert_codes_close(codes, c_ref)
+
+
+def draw_calibrations(n, seed):
+    rng = np.random.default_rng(seed)
+    out = []
+    for i in range(n):
+        rows = int(rng.integers(1, 300)) if i % 4 == 0 else int(rng.integers(300, 60_000))
+        C = int(rng.integers(1, 700))
+        ld = 4 * ((C + 3) // 4) + 4 * int(rng.integers(0, 3))        # rows of 16-byte multiples, sometimes padded
+        out.append((rows, C, ld, int(rng.integers(0, 1 << 30))))
+    return out
+
+
+@pytest.mark.parametrize("rows,C,ld,seed", draw_calibrations(24, seed=5))
+def test_random_calibration_against_the_oracle(H, rows, C, ld, seed):
+    """Random lengths, channel counts (ragged against the 128-channel slabs) and leading dimensions; per channel a random
+    mean (up to a thousand spreads away), spread, slope and noise level, and a few constant channels (Eq. 4's degenerate
+    case).  (a, b) and the degenerate count against the oracle's centred two-pass fit."""
+    rng = np.random.default_rng(seed)
+    mean = rng.standard_normal(C) * 10.0 ** rng.uniform(-2, 3, C)
+    spread = 10.0 ** rng.uniform(-2, 1, C)
+    q = np.full((rows, ld), 7e29, np.float32)                        # the padding columns must not matter
+    f = np.full((rows, ld), -3e29, np.float32)
+    q[:, :C] = (mean[None, :] + spread[None, :] * rng.standard_normal((rows, C))).astype(np.float32)
+    slope = 1 + 0.1 * rng.standard_normal(C)
+    noise = spread * 10.0 ** rng.uniform(-3, -1, C)
+    f[:, :C] = (slope[None, :] * q[:, :C].astype(np.float64) + rng.standard_normal(C)[None, :] * spread[None, :] +
+                noise[None, :] * rng.standard_normal((rows, C))).astype(np.float32)
+    dead = rng.random(C) < 0.03
+    q[:, :C][:, dead] = q[0, :C][dead][None, :]
+    a, b, nd = H.gpu_calibrate(f, q, channels=C)
+    a_ref, b_ref, nd_ref = O.cwac_fit(f[:, :C], q[:, :C])
+    assert nd == nd_ref
+    f64 = f[:, :C].astype(np.float64)
+    assert_ab_close(a, b, a_ref, b_ref, np.maximum(np.abs(f64.mean(0)), f64.std(0)))
+
