@@ -753,6 +753,8 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     }
 
     int use = 0;                            // units this group has handled
+    int xuse = 0;                           // ... of which through the counter exchange (phases of pub / ready there:
+                                            // a unit right of the matrix handles nothing and arrives on neither)
     int slice_n0 = -1;                      // first column of the unit whose parameters are in the group's slice
     int reloads = 0;                        // times the slice has been (re)loaded
     for (int u = g; u < n_units; u += kGroups, ++use, walk = next, next.advance(kTileStep)) {
@@ -1044,7 +1046,7 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
           if (lead) {
             // the lead warp counts the unit once the whole group has published, then waits for the strip
             if (lane == 0) {
-              int fine = ptx::mbar_wait_bounded(&pub[g], upar, cta_abort, tmo) ? 1 : 0;
+              int fine = ptx::mbar_wait_bounded(&pub[g], (uint32_t)xuse & 1u, cta_abort, tmo) ? 1 : 0;
               if (fine) {
                 __threadfence();
                 const uint32_t old = atomicAdd(p.counters + tm, 1u);
@@ -1073,8 +1075,9 @@ qlinear_cwac_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
             __syncwarp();     // the other lanes wait here, not in a spin loop beside lane 0
           }
-          if (!ptx::mbar_wait_bounded(&ready[g], upar, cta_abort, tmo)) good = 0;
+          if (!ptx::mbar_wait_bounded(&ready[g], (uint32_t)xuse & 1u, cta_abort, tmo)) good = 0;
           else amax_row = row < p.M ? __uint_as_float(__ldcg(p.rowmax + row)) : 0.f;
+          ++xuse;
         }
         if (!__all_sync(0xffffffffu, good)) {
           if (lane == 0) give_up(kStWaitStrip);

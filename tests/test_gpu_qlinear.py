@@ -430,3 +430,17 @@ def test_w4_resident_halves_expanded_on_chip(H, B, M, N, K):
     c_ref, ys_ref = O.requant_per_token(z_ref)
     assert np.allclose(ys, ys_ref, rtol=1e-5, atol=0)
     assert_codes_close(codes, c_ref)
+
+
+@pytest.mark.parametrize("M,N,K", [(2600, 4112, 128), (10916, 4112, 800)])
+def test_counter_exchange_with_half_empty_last_column_tile(H, B, M, N, K):
+    """Per-token INT8 over more than 32 units per row strip (the counter-and-flag exchange) with a last column tile whose
+    second unit lies right of the matrix: a group that was handed such a unit takes no part in that exchange, and the
+    phases of its exchange barriers must not count it (they once did: the group's next exchange then waited on the
+    wrong phase and ran into the wait limit)."""
+    Xq, Wq, xs, fs, fb = random_layer(M, N, K, seed=M + N + K + 21)
+    z_ref = O.forward_folded(O.int_matmul(Xq, Wq), xs, fs, fb)
+    codes, ys = H.gpu_forward(Xq, xs, Wq, fs, fb, B.QWT_OUT_INT8_PER_TOKEN)
+    c_ref, ys_ref = O.requant_per_token(z_ref)
+    assert np.allclose(ys, ys_ref, rtol=1e-5, atol=0)
+    assert_codes_close(codes, c_ref)
